@@ -1,0 +1,373 @@
+"""Pins the fp64 oracle to things other than itself.
+
+Each test re-derives a result by a different route (explicit Python loops over the
+definition, a brute-force full-matrix gradient that never forms u, central finite
+differences of an independently written loss, a closed form, an SVD) so that a dropped
+term, a wrong sign or index, or a transposed operand in the oracle fails at least one.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import sfb_oracle as orc
+from sfbgen import make_inputs, scaled
+
+RNG = np.random.default_rng(12345)
+
+
+# ----------------------------------------------------------------------------- helpers
+def loop_softmax(z):
+    m = max(z)
+    e = [math.exp(v - m) for v in z]
+    s = sum(e)
+    return [v / s for v in e]
+
+
+def loop_matvec(W, a):
+    return [sum(W[j][d] * a[d] for d in range(len(a))) for j in range(len(W))]
+
+
+def loop_mlr_loss(W, X, y):
+    tot = 0.0
+    for i in range(len(X)):
+        z = loop_matvec(W, X[i])
+        m = max(z)
+        tot += m + math.log(sum(math.exp(v - m) for v in z)) - z[y[i]]
+    return tot
+
+
+def loop_dml_loss(L, Xa, Xb, sim, margin):
+    tot = 0.0
+    for i in range(len(Xa)):
+        d = [float(np.float32(Xa[i][k]) - np.float32(Xb[i][k])) for k in range(len(Xa[i]))]
+        z = loop_matvec(L, d)
+        n = sum(v * v for v in z)
+        tot += 0.5 * n if sim[i] else 0.5 * max(0.0, margin - n)
+    return tot
+
+
+def loop_sc_loss(W, A, X):
+    tot = 0.0
+    for i in range(len(A)):
+        z = loop_matvec(W, A[i])
+        tot += 0.5 * sum((z[j] - X[i][j]) ** 2 for j in range(len(z)))
+    return tot
+
+
+def central_fd(loss, W, h=1e-5):
+    W = np.array(W, dtype=np.float64)
+    G = np.zeros_like(W)
+    for j in range(W.shape[0]):
+        for d in range(W.shape[1]):
+            w0 = W[j, d]
+            W[j, d] = w0 + h
+            lp = loss(W.tolist())
+            W[j, d] = w0 - h
+            lm = loss(W.tolist())
+            W[j, d] = w0
+            G[j, d] = (lp - lm) / (2 * h)
+    return G
+
+
+def dense_to_csr(A):
+    rowptr, idx, val = [0], [], []
+    for row in A:
+        nz = np.nonzero(row)[0]
+        idx.extend(nz.tolist())
+        val.extend(row[nz].tolist())
+        rowptr.append(len(idx))
+    return np.array(rowptr, np.uint32), np.array(idx, np.uint32), np.array(val, np.float32)
+
+
+def tiny_mlr(J=5, D=7, K=6):
+    W = RNG.normal(0, 0.5, (J, D)).astype(np.float32)
+    X = RNG.normal(0, 1, (K, D)).astype(np.float32)
+    y = RNG.integers(0, J, K).astype(np.int32)
+    return W, X, y
+
+
+# ----------------------------------------------------------------------------- MLR
+def test_mlr_u_matches_definition_by_loops():
+    W, X, y = tiny_mlr()
+    U, V = orc.mlr_factors(W, X, y)
+    for i in range(len(X)):
+        p = loop_softmax(loop_matvec(W.astype(np.float64).tolist(), X[i].astype(np.float64).tolist()))
+        p[y[i]] -= 1.0
+        assert np.allclose(U[i], p, rtol=0, atol=1e-14)
+    assert np.array_equal(V, X.astype(np.float64))
+
+
+def test_mlr_sf_update_equals_bruteforce_gradient():
+    # G[j][d] = sum_i softmax(z_i)[j] x_i[d]  -  sum_{i: y_i = j} x_i[d]   (never forms u)
+    W, X, y = tiny_mlr(J=6, D=9, K=11)
+    U, V = orc.mlr_factors(W, X, y)
+    W64, X64 = W.astype(np.float64), X.astype(np.float64)
+    G = np.zeros_like(W64)
+    for i in range(len(X)):
+        p = loop_softmax(loop_matvec(W64.tolist(), X64[i].tolist()))
+        for j in range(W.shape[0]):
+            G[j] += p[j] * X64[i]
+    for i in range(len(X)):
+        G[y[i]] -= X64[i]
+    assert orc.rel_fro(orc.delta_w(U, V), G) <= 1e-12
+
+
+def test_mlr_gradient_by_finite_differences_c0():
+    # The whole tiny workload C0 (10 x 64, K = 32): 640 parameters.
+    cfg = scaled("C0")
+    inp = make_inputs(cfg)
+    W, X, y = inp["W"], inp["X"][0], inp["labels"][0]
+    U, V = orc.mlr_factors(W, X, y)
+    X64, yl = X.astype(np.float64).tolist(), y.tolist()
+    G = central_fd(lambda Wl: loop_mlr_loss(Wl, X64, yl), W)
+    assert orc.rel_fro(orc.delta_w(U, V), G) <= 1e-7
+    # the oracle's own loss agrees with the loop loss
+    assert abs(orc.mlr_loss(W, X, y) - loop_mlr_loss(W.astype(np.float64).tolist(), X64, yl)) <= 1e-10
+
+
+def test_mlr_u_rows_sum_to_zero_and_rank_bounds():
+    cfg = scaled("C0")
+    inp = make_inputs(cfg)
+    U, V = orc.mlr_factors(inp["W"], inp["X"][0], inp["labels"][0])
+    assert np.abs(U.sum(axis=1)).max() <= 1e-14
+    # C0 has J = 10 < K = 32: 1^T dW = 0 gives rank <= J - 1 = 9
+    s = np.linalg.svd(orc.delta_w(U, V), compute_uv=False)
+    assert s[9] <= 1e-12 * s[0]
+    # K = 4 < min(J, D): rank <= K
+    s4 = np.linalg.svd(orc.delta_w(U[:4], V[:4]), compute_uv=False)
+    assert s4[3] > 1e-8 * s4[0]
+    assert s4[4] <= 1e-12 * s4[0]
+
+
+def test_mlr_closed_form_at_w_zero():
+    J, D, K = 7, 5, 9
+    X = RNG.normal(0, 1, (K, D)).astype(np.float32)
+    y = RNG.integers(0, J, K).astype(np.int32)
+    U, V = orc.mlr_factors(np.zeros((J, D), np.float32), X, y)
+    expect = np.tile(X.astype(np.float64).sum(axis=0) / J, (J, 1))
+    for i in range(K):
+        expect[y[i]] -= X[i].astype(np.float64)
+    assert np.allclose(orc.delta_w(U, V), expect, rtol=0, atol=1e-13)
+
+
+def test_mlr_two_classes_is_binary_logistic_regression():
+    W, X, y = tiny_mlr(J=2, D=4, K=8)
+    U, _ = orc.mlr_factors(W, X, y)
+    Z = X.astype(np.float64) @ W.astype(np.float64).T
+    sig = 1.0 / (1.0 + np.exp(-(Z[:, 0] - Z[:, 1])))
+    assert np.allclose(U[:, 0], sig - (y == 0), atol=1e-14)
+    assert np.allclose(U[:, 1], -U[:, 0], atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- DML
+def tiny_dml(J=6, D=16, K=12, scale=0.25):
+    L = RNG.normal(0, scale / math.sqrt(D), (J, D)).astype(np.float32)
+    Xa = RNG.normal(0, 1, (K, D)).astype(np.float32)
+    Xb = RNG.normal(0, 1, (K, D)).astype(np.float32)
+    sim = (np.arange(K) % 2 == 0).astype(np.uint8)
+    return L, Xa, Xb, sim
+
+
+def test_dml_gradient_by_finite_differences_and_scatter_matrix():
+    L, Xa, Xb, sim = tiny_dml()
+    U, V, n, active = orc.dml_factors(L, Xa, Xb, sim, 1.0)
+    dis = ~sim.astype(bool)
+    assert active[dis].any() and (~active[dis]).any()           # both hinge branches exercised
+    assert np.abs(n[dis] - 1.0).min() > 1e-3                      # away from the kink
+    G_fd = central_fd(lambda Ll: loop_dml_loss(Ll, Xa.tolist(), Xb.tolist(), sim.tolist(), 1.0), L)
+    assert orc.rel_fro(orc.delta_w(U, V), G_fd) <= 1e-7
+    # brute force through the D x D scatter matrices: G = L (sum_sim d d^T - sum_{dis, active} d d^T)
+    Dm = (Xa - Xb).astype(np.float64)
+    S = np.zeros((Dm.shape[1], Dm.shape[1]))
+    for i in range(len(Dm)):
+        if sim[i]:
+            S += np.outer(Dm[i], Dm[i])
+        elif sum(v * v for v in loop_matvec(L.astype(np.float64).tolist(), Dm[i].tolist())) < 1.0:
+            S -= np.outer(Dm[i], Dm[i])
+    assert orc.rel_fro(orc.delta_w(U, V), L.astype(np.float64) @ S) <= 1e-12
+    assert np.array_equal(V, Dm)
+
+
+def test_dml_special_cases():
+    L, Xa, Xb, sim = tiny_dml()
+    # L = 0 -> U = 0 -> L unchanged
+    U0, V0, _, _ = orc.dml_factors(np.zeros_like(L), Xa, Xb, sim)
+    assert not U0.any()
+    assert np.array_equal(orc.apply_dense(np.zeros_like(L), U0, V0, 0.3), np.zeros(L.shape))
+    # all similar -> dL = L (D^T D)
+    allsim = np.ones(len(Xa), np.uint8)
+    U, V, _, _ = orc.dml_factors(L, Xa, Xb, allsim)
+    Dm = (Xa - Xb).astype(np.float64)
+    assert orc.rel_fro(orc.delta_w(U, V), L.astype(np.float64) @ (Dm.T @ Dm)) <= 1e-13
+    # a dissimilar pair beyond the margin contributes nothing; strictness at equality
+    big = np.float32(50.0)
+    Ud, _, nd, act = orc.dml_factors(L, Xa * big, Xb * big, np.zeros(len(Xa), np.uint8))
+    assert (nd >= 1.0).all() and not act.any() and not Ud.any()
+    L1 = np.array([[1.0, 0.0]], np.float32)
+    _, _, n1, a1 = orc.dml_factors(L1, np.array([[1.0, 0.0]], np.float32), np.zeros((1, 2), np.float32), [0])
+    assert n1[0] == 1.0 and not a1[0]
+    # scaling a similar pair's difference by c scales its contribution by c^2 (c a power of two: exact)
+    U1, V1, _, _ = orc.dml_factors(L, Xa[:1], Xb[:1], [1])
+    U2, V2, _, _ = orc.dml_factors(L, Xa[:1] * np.float32(2), Xb[:1] * np.float32(2), [1])
+    assert np.allclose(orc.delta_w(U2, V2), 4.0 * orc.delta_w(U1, V1), rtol=1e-15)
+    # sign of an active dissimilar pair is the opposite of a similar one
+    small = np.float32(1e-3)
+    Us, _, _, _ = orc.dml_factors(L, Xa[:1] * small, Xb[:1] * small, [1])
+    Un, _, _, an = orc.dml_factors(L, Xa[:1] * small, Xb[:1] * small, [0])
+    assert an[0] and np.array_equal(Un, -Us)
+
+
+# ----------------------------------------------------------------------------- SC
+def tiny_sc(J=8, D=20, K=6, density=0.3):
+    W = RNG.normal(0, 1, (J, D)).astype(np.float32)
+    A = (RNG.normal(0, 1, (K, D)) * (RNG.random((K, D)) < density)).astype(np.float32)
+    X = RNG.normal(0, 1, (K, J)).astype(np.float32)
+    return W, A, X
+
+
+def test_sc_gradient_fd_gram_route_and_sparse_equals_dense():
+    W, A, X = tiny_sc()
+    rowptr, idx, val = dense_to_csr(A)
+    U = orc.sc_factors(W, rowptr, idx, val, X)
+    W64, A64, X64 = (m.astype(np.float64) for m in (W, A, X))
+    for i in range(len(A)):
+        z = loop_matvec(W64.tolist(), A64[i].tolist())
+        assert np.allclose(U[i], np.array(z) - X64[i], atol=1e-13)
+    dW = orc.delta_w(U, orc.csr_to_dense(rowptr, idx, val, W.shape[1]))
+    assert orc.rel_fro(dW, W64 @ (A64.T @ A64) - X64.T @ A64) <= 1e-12        # Gram-matrix route
+    G_fd = central_fd(lambda Wl: loop_sc_loss(Wl, A64.tolist(), X64.tolist()), W)
+    assert orc.rel_fro(dW, G_fd) <= 1e-7
+    Wn_sparse = orc.apply_sparse(W, U, rowptr, idx, val, 0.01)
+    assert np.allclose(Wn_sparse, W64 - 0.01 * dW, rtol=0, atol=1e-14)
+    assert abs(orc.sc_loss(W, rowptr, idx, val, X) - loop_sc_loss(W64.tolist(), A64.tolist(), X64.tolist())) < 1e-10
+
+
+def test_sc_special_cases():
+    W, A, X = tiny_sc()
+    rowptr, idx, val = dense_to_csr(A)
+    # fixed point: x_i = W a_i exactly -> u = 0 -> W unchanged
+    Xfix = (A.astype(np.float64) @ W.astype(np.float64).T)
+    U = orc.sc_factors(W, rowptr, idx, val, Xfix)
+    assert np.abs(U).max() <= 1e-14
+    # one-hot code a = c e_j: only column j changes, W[:,j] <- W[:,j] - eta c (c W[:,j] - x)
+    j, c, eta = 3, 1.5, 0.2
+    rp1, ix1, vl1 = np.array([0, 1], np.uint32), np.array([j], np.uint32), np.array([c], np.float32)
+    x = X[:1]
+    U1 = orc.sc_factors(W, rp1, ix1, vl1, x)
+    Wn = orc.apply_sparse(W, U1, rp1, ix1, vl1, eta)
+    expect = W.astype(np.float64)
+    expect[:, j] -= eta * c * (c * W[:, j].astype(np.float64) - x[0])
+    assert np.allclose(Wn, expect, atol=1e-15)
+    # with c = 1 and eta = 1 the column becomes x exactly
+    vl1[0] = 1.0
+    Wn1 = orc.apply_sparse(W, orc.sc_factors(W, rp1, ix1, vl1, x), rp1, ix1, vl1, 1.0)
+    assert np.allclose(Wn1[:, j], x[0].astype(np.float64), atol=1e-15)
+    # columns of atoms no code uses are bit-identical before and after
+    used = np.zeros(W.shape[1], bool)
+    used[idx] = True
+    Wn2 = orc.apply_sparse(W, orc.sc_factors(W, rowptr, idx, val, X), rowptr, idx, val, 0.1)
+    assert (~used).any()
+    assert np.array_equal(Wn2[:, ~used], W.astype(np.float64)[:, ~used])
+
+
+# ----------------------------------------------------------------------------- apply
+def test_apply_is_the_sum_of_outer_products_and_is_additive_linear_permutation_invariant():
+    J, D, K = 5, 7, 9
+    W = RNG.normal(0, 1, (J, D))
+    U = RNG.normal(0, 1, (K, J))
+    V = RNG.normal(0, 1, (K, D))
+    # apply-to-zero with eta = -1 is U^T V; checked by the triple loop of the definition
+    T = orc.apply_dense(np.zeros((J, D)), U, V, -1.0)
+    ref = np.zeros((J, D))
+    for i in range(K):
+        for j in range(J):
+            for d in range(D):
+                ref[j, d] += U[i, j] * V[i, d]
+    assert np.allclose(T, ref, atol=1e-14)
+    full = orc.apply_dense(W, U, V, 0.3)
+    assert np.allclose(full, W - 0.3 * ref, atol=1e-14)
+    # additivity over a split of the SFs (how workers' streams are applied)
+    half = orc.apply_dense(orc.apply_dense(W, U[:4], V[:4], 0.3), U[4:], V[4:], 0.3)
+    assert np.allclose(half, full, atol=1e-14)
+    # eta-linearity and permutation invariance
+    two = orc.apply_dense(orc.apply_dense(W, U, V, 0.1), U, V, 0.2)
+    assert np.allclose(two, full, atol=1e-14)
+    perm = RNG.permutation(K)
+    assert np.allclose(orc.apply_dense(W, U[perm], V[perm], 0.3), full, atol=1e-14)
+
+
+def test_step_is_independent_of_the_worker_split_and_lowers_the_loss():
+    cfg = scaled("C0")
+    inp = make_inputs(cfg)
+    batch = dict(X=inp["X"][0], labels=inp["labels"][0])
+    W1, U, V = orc.step(orc.MODEL_MLR, inp["W"], batch, cfg["eta"] / cfg["K"])
+    # the same K pairs split as (P,B) = (1,32), (4,8), (32,1) unpack to identical factors
+    for P, B in ((1, 32), (4, 8), (32, 1)):
+        buf = orc.pack(orc.MODEL_MLR, orc.DTYPE_F32, cfg["J"], cfg["D"], P, B, U, V)
+        _, U2, V2 = orc.unpack(buf)
+        assert np.array_equal(U2, U.astype(np.float32)) and np.array_equal(V2, V.astype(np.float32))
+    assert orc.mlr_loss(W1, batch["X"], batch["labels"]) < orc.mlr_loss(inp["W"], batch["X"], batch["labels"])
+
+
+# ----------------------------------------------------------------------------- pack
+def test_pack_header_directory_and_alignment():
+    J, D, P, B = 10, 64, 4, 8
+    U = RNG.normal(0, 1, (P * B, J))
+    V = RNG.normal(0, 1, (P * B, D))
+    buf = orc.pack(orc.MODEL_MLR, orc.DTYPE_F32, J, D, P, B, U, V, clock=7)
+    h = orc.parse_header(buf)
+    assert h["magic"] == 0x31424653 and bytes(buf[:4]) == b"SFB1"
+    assert (h["version"], h["model"], h["dtype"], h["flags"]) == (1, 0, 0, 0)
+    assert (h["P"], h["B"], h["J"], h["D"], h["clock"]) == (P, B, J, D, 7)
+    assert h["ldu"] == 12 and h["ldv"] == 64            # 10 floats -> 48 bytes = 3 x 16
+    assert h["total_bytes"] == buf.size
+    assert h["streams_off"] == 128 + 128 and h["stream_stride"] % 128 == 0
+    assert h["stream_stride"] == 384 + 2048             # B*ldu*4 = 384 ; B*ldv*4 = 2048
+    for p in range(P):
+        e = np.frombuffer(bytes(buf[128 + 32 * p:160 + 32 * p]), dtype=np.uint32)
+        assert (e[0], e[1], e[2], e[3]) == (p, B, 7, 0)
+        u_off, v_off = np.frombuffer(bytes(buf[128 + 32 * p + 16:160 + 32 * p]), dtype=np.uint64)
+        assert u_off == h["streams_off"] + p * h["stream_stride"] and v_off == u_off + 384
+        row = buf[int(u_off):int(u_off) + 48].view(np.float32)
+        assert np.array_equal(row[:10], U[p * B].astype(np.float32)) and not row[10:].any()
+        vrow = buf[int(v_off) + 256:int(v_off) + 512].view(np.float32)          # second v row of the worker
+        assert np.array_equal(vrow, V[p * B + 1].astype(np.float32))
+    _, U2, V2 = orc.unpack(buf)
+    assert np.array_equal(U2, U.astype(np.float32)) and np.array_equal(V2, V.astype(np.float32))
+
+
+def test_pack_bf16_rounds_to_nearest_even():
+    # 1 + 2^-8 is a tie between 1.0 and 1 + 2^-7 -> even mantissa (1.0); 1 + 3*2^-8 ties up to 1 + 2^-6
+    vals = np.array([[1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -2.5, 0.0, 3.0e-5, 7.0]])
+    buf = orc.pack(orc.MODEL_MLR, orc.DTYPE_BF16, 8, 8, 1, 1, vals, vals)
+    h, U, V = orc.unpack(buf)
+    assert h["ldu"] == 8 and h["dtype"] == 1
+    assert U[0, 0] == 1.0 and U[0, 1] == 1.0 and U[0, 2] == 1.0 + 2.0 ** -6 and U[0, 3] == 1.0 + 2.0 ** -7
+    assert U[0, 4] == -2.5 and U[0, 5] == 0.0 and U[0, 7] == 7.0
+    assert abs(U[0, 6] - 3.0e-5) <= 3.0e-5 * 2.0 ** -8
+    raw = buf[h["streams_off"]:h["streams_off"] + 16].view(np.uint16)
+    assert raw[0] == 0x3F80 and raw[4] == 0xC020
+
+
+def test_pack_sparse_v_roundtrip():
+    cfg = scaled("C3", J=16, D=40, P=2, B=3, density=0.2)
+    inp = make_inputs(cfg)
+    rowptr, idx, val = inp["rowptr"][0], inp["idx"][0], inp["val"][0]
+    K = cfg["K"]
+    for i in range(K):
+        seg = idx[rowptr[i]:rowptr[i + 1]]
+        assert (np.diff(seg.astype(np.int64)) > 0).all()               # strictly ascending
+    U = RNG.normal(0, 1, (K, cfg["J"]))
+    buf = orc.pack(orc.MODEL_SC, orc.DTYPE_F32, cfg["J"], cfg["D"], cfg["P"], cfg["B"], U,
+                   csr=(rowptr, idx, val), clock=3, nnz_capacity=inp["nnz_capacity"])
+    h, U2, (rp2, ix2, vl2) = orc.unpack(buf)
+    assert h["flags"] == 1 and h["cap_p"] == inp["nnz_capacity"] // cfg["P"]
+    assert np.array_equal(rp2, rowptr) and np.array_equal(ix2, idx) and np.array_equal(vl2, val)
+    assert np.array_equal(U2, U.astype(np.float32))
+    for p in range(cfg["P"]):
+        nnz_p = np.frombuffer(bytes(buf[128 + 32 * p + 12:128 + 32 * p + 16]), dtype=np.uint32)[0]
+        assert nnz_p == rowptr[(p + 1) * cfg["B"]] - rowptr[p * cfg["B"]]
+    with pytest.raises(ValueError):
+        orc.pack(orc.MODEL_SC, orc.DTYPE_F32, cfg["J"], cfg["D"], cfg["P"], cfg["B"], U,
+                 csr=(rowptr, idx, val), nnz_capacity=cfg["P"])
