@@ -1,0 +1,158 @@
+/*
+ * sfb.h -- C ABI of the sufficient-factor (SF) hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library computes, for matrix-parametrised models min_W (1/N) sum_i f_i(W a_i) + h(W)
+ * (paper Section 2, problem (P), W in R^{J x D}), the two stages of Sufficient Factor
+ * Broadcasting that touch W:
+ *
+ *   1. per-sample sufficient factors (u_i, v_i) with  grad_i = u_i v_i^T,
+ *      u_i = d f_i / d (W a_i),  v_i = a_i                       (Section 2.1, "Proximal SGD");
+ *   2. the rank-K update from the factors of all P workers,
+ *      W <- W - eta * sum_{i<K} u_i v_i^T,  K = P*B               (Section 3, incl. "Mini-batch").
+ *
+ * Between the two sits the SF buffer: the message the P workers would broadcast, laid out as P
+ * worker streams in one device buffer (Section 4.2: write_u / write_v / commit; Section 4.4:
+ * input/output SF queues).  No network is involved; the P workers are simulated in one buffer.
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer owned by the caller and 128-byte aligned.  The
+ *     library never frees or reallocates caller memory; it allocates only its own workspace, in
+ *     sfb_create, and frees it in sfb_destroy.
+ *   - All calls enqueue work on the CUDA stream given to sfb_create and return without
+ *     synchronising, except sfb_status and sfb_destroy.
+ *   - Return value: 0 (SFB_OK) or a negative SFB_ERR_* code found on the host before anything was
+ *     launched (no partial effect).  Conditions only the device can see (label out of range, CSR
+ *     index out of range or unsorted, SF-buffer header not matching the descriptor, CSR capacity
+ *     exceeded) set bits of a sticky device status word and make the kernel that found them skip
+ *     the affected writes; nothing traps.  Read the word with sfb_status.
+ *   - W is J x D, row-major fp32, updated in place.  Samples are rows: X is [K][D].
+ *   - Sample i belongs to worker p = i / B, slot i % B.
+ *
+ * Arithmetic paths (sfb_desc.path)
+ *   SFB_PATH_F32   fp32 FMA on CUDA cores; X, U, V fp32.
+ *   SFB_PATH_TF32  tensor cores (tcgen05, kind::tf32), fp32 accumulate; X, U, V fp32 in memory.
+ *   SFB_PATH_BF16  tensor cores (tcgen05, kind::f16 with bf16 inputs), fp32 accumulate; X, U, V
+ *                  bf16 in memory; W stays an fp32 master and the context keeps a bf16 shadow of
+ *                  it that the apply refreshes.
+ *
+ * SF buffer wire format (little-endian; every offset a multiple of 128 bytes)
+ *   header, 128 bytes:
+ *      0 u32 magic 0x31424653 ("SFB1")   4 u16 version 1   6 u8 model   7 u8 value dtype (0 f32, 1 bf16)
+ *      8 u32 flags (bit 0: v is sparse)  12 u32 P  16 u32 B  20 u32 J  24 u32 D
+ *     28 u32 clock (iteration number)    32 u32 ldu  36 u32 ldv
+ *     40 u64 stream_stride  48 u64 total_bytes  56 u64 streams_off  64 u32 cap_p   rest zero
+ *   directory at 128: P entries of 32 bytes {u32 worker, u32 n_sf (= B), u32 clock, u32 nnz,
+ *      u64 u_off, u64 v_off}, padded to 128 bytes.
+ *   worker stream p at streams_off + p * stream_stride:
+ *      U block: B rows of ldu values, row r = u of sample p*B + r, pad values zero, padded to 128 B;
+ *      V block: dense: B rows of ldv values; sparse (CSR): u32 rowptr[B+1] (local, starts at 0),
+ *               u32 idx[cap_p], value val[cap_p], each padded to 128 B, unused tail zero.
+ *   ldu (ldv) is J (D) rounded up so that a row is a whole number of 16-byte units.
+ *   cap_p = nnz_capacity / P.  bf16 values are fp32 rounded to nearest even.
+ */
+#ifndef SFB_H_
+#define SFB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sfb_ctx sfb_ctx; /* opaque: workspace, cached tensor maps, device status word */
+
+enum { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2 };
+enum { SFB_PATH_F32 = 0, SFB_PATH_TF32 = 1, SFB_PATH_BF16 = 2 };
+
+enum {
+  SFB_OK = 0,
+  SFB_ERR_ARG = -1,         /* null pointer, misaligned pointer, K not a whole number of worker streams */
+  SFB_ERR_SHAPE = -2,       /* non-positive or unsupported sizes */
+  SFB_ERR_UNSUPPORTED = -3, /* model/path combination not provided, or not an sm_100 device */
+  SFB_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed */
+  SFB_ERR_ALLOC = -5        /* workspace allocation failed */
+};
+
+/* bits of the device status word */
+enum {
+  SFB_DEV_BAD_LABEL = 1,    /* MLR label outside [0, J): that sample's u is written as zeros */
+  SFB_DEV_BAD_INDEX = 2,    /* CSR column >= D or not strictly ascending: that entry is skipped */
+  SFB_DEV_BAD_HEADER = 4,   /* SF buffer header does not match the descriptor: apply leaves W untouched */
+  SFB_DEV_CAPACITY = 8,     /* a worker's nonzeros exceed cap_p: that stream's codes are truncated */
+  SFB_DEV_TIMEOUT = 16      /* a bounded device-side wait ran out */
+};
+
+typedef struct sfb_desc {
+  int32_t model;         /* SFB_MLR / SFB_DML / SFB_SC */
+  int32_t path;          /* SFB_PATH_* */
+  int32_t J, D;          /* W is J x D (SC: J = feature dimension, D = number of atoms) */
+  int32_t P, B;          /* simulated workers, SF pairs per worker; K = P*B */
+  int32_t v_sparse;      /* 1: v is CSR (required for SFB_SC), 0: dense */
+  float margin;          /* DML hinge margin on the squared distance */
+  uint64_t nnz_capacity; /* total CSR capacity (a multiple of 32*P) when v_sparse */
+} sfb_desc;
+
+/* Per-model side inputs of the factor computation (device pointers; unused ones NULL). */
+typedef struct sfb_aux {
+  const int32_t* labels;  /* MLR: class of each sample, [K] */
+  const void* Xb;         /* DML: second element of each pair, [K][D], same type as X (X is the first) */
+  const uint8_t* similar; /* DML: 1 = similar pair, 0 = dissimilar, [K] */
+  const uint32_t* rowptr; /* SC: CSR row pointers of the codes, [K+1], rowptr[0] = 0 */
+  const uint32_t* idx;    /* SC: atom index of each nonzero, strictly ascending within a row */
+  const void* val;        /* SC: value of each nonzero (fp32) */
+  const void* Xdata;      /* SC: data vectors x_i, [K][J] fp32 */
+} sfb_aux;
+
+/* Creates a context for one (model, path, shape).  `cuda_stream` is a cudaStream_t (NULL = the
+ * legacy default stream).  Allocates the workspace the chosen path needs.  (No paper counterpart
+ * beyond the constructor sfb_app(J, D, staleness) of Section 4.2.) */
+int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out);
+
+/* Synchronises the stream and frees the workspace. */
+int sfb_destroy(sfb_ctx* ctx);
+
+/* Bytes the caller must allocate for the SF buffer of `desc` (0 on a bad descriptor). */
+size_t sfb_sf_buffer_bytes(const sfb_desc* desc);
+
+/* Padded row lengths (in values) of U and V rows; caller-side U / V arrays use them too. */
+int sfb_ld(const sfb_desc* desc, int32_t* ldu, int32_t* ldv);
+
+/* Sufficient factors of K = P*B samples (Section 2.1; Figures 2 and 3):
+ *   MLR  z = W x,           u = softmax(z) - onehot(label),              v = x
+ *   DML  d = x - xb, z = W d, u = +z (similar) | -z*[|z|^2 < margin] (dissimilar), v = d
+ *   SC   z = W a (a = CSR code), u = z - xdata,                          v = a (not copied here)
+ * W [J][D] fp32; X [K][D] (fp32, or bf16 on SFB_PATH_BF16); U out [K][ldu]; V out [K][ldv]
+ * (V may be NULL for SC and is ignored).  Pad columns of U and V are written as zeros. */
+int sfb_compute_factors(sfb_ctx* ctx, const void* W, const void* X, const sfb_aux* aux, void* U, void* V);
+
+/* Lays K (u, v) pairs out as P worker streams with header and directory: what the workers would
+ * broadcast after commit() (Section 4.2).  U [K][ldu], V [K][ldv] in the path's value type; for
+ * sparse v pass V = NULL and the CSR arrays through `aux`.  Pure data movement. */
+int sfb_pack(sfb_ctx* ctx, const void* U, const void* V, const sfb_aux* aux, void* sf_buf, uint32_t clock);
+
+/* Rank-K update W <- W - eta * sum_{i<K} u_i v_i^T from the first K/B worker streams of the SF
+ * buffer (Section 3: every worker applies the factors of all workers).  K must be a positive
+ * multiple of B and at most P*B.  The sum order is fixed, so results are bit-reproducible. */
+int sfb_apply(sfb_ctx* ctx, void* W, const void* sf_buf, float eta, int32_t K);
+
+/* One iteration: factors written straight into the SF buffer (header and directory included, with
+ * the given clock), then the apply of the first K slots.  K as in sfb_apply. */
+int sfb_step(sfb_ctx* ctx, void* W, const void* X, const sfb_aux* aux, void* sf_buf, float eta, int32_t K,
+             uint32_t clock);
+
+/* Tells the context that W was changed by someone else, so a cached bf16 shadow is stale. */
+int sfb_invalidate(sfb_ctx* ctx);
+
+/* Synchronises the stream, returns the sticky device status word in *device_status and clears it. */
+int sfb_status(sfb_ctx* ctx, int32_t* device_status);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t sfb_launch_count(const sfb_ctx* ctx);
+
+const char* sfb_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SFB_H_ */

@@ -1,0 +1,178 @@
+"""ctypes binding of the C ABI in include/sfb.h: same names, argument marshalling only.
+
+Every step of the path runs inside libsfb.so's CUDA kernels.  If the library is missing or cannot
+be loaded this module raises; there is no Python or CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+from .build import LIB_PATH
+
+SFB_MLR, SFB_DML, SFB_SC = 0, 1, 2
+SFB_PATH_F32, SFB_PATH_TF32, SFB_PATH_BF16 = 0, 1, 2
+SFB_OK = 0
+SFB_DEV_BAD_LABEL, SFB_DEV_BAD_INDEX, SFB_DEV_BAD_HEADER, SFB_DEV_CAPACITY, SFB_DEV_TIMEOUT = 1, 2, 4, 8, 16
+
+MODELS = {"mlr": SFB_MLR, "dml": SFB_DML, "sc": SFB_SC}
+PATHS = {"f32": SFB_PATH_F32, "tf32": SFB_PATH_TF32, "bf16": SFB_PATH_BF16}
+
+# Every entry point include/sfb.h declares (checked by the CPU test-suite against the built library).
+EXPORTS = (
+    "sfb_create", "sfb_destroy", "sfb_sf_buffer_bytes", "sfb_ld", "sfb_compute_factors", "sfb_pack",
+    "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
+)
+
+
+class sfb_desc(C.Structure):
+    _fields_ = [("model", C.c_int32), ("path", C.c_int32), ("J", C.c_int32), ("D", C.c_int32),
+                ("P", C.c_int32), ("B", C.c_int32), ("v_sparse", C.c_int32), ("margin", C.c_float),
+                ("nnz_capacity", C.c_uint64)]
+
+
+class sfb_aux(C.Structure):
+    _fields_ = [("labels", C.c_void_p), ("Xb", C.c_void_p), ("similar", C.c_void_p), ("rowptr", C.c_void_p),
+                ("idx", C.c_void_p), ("val", C.c_void_p), ("Xdata", C.c_void_p)]
+
+
+class SfbError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> C.CDLL:
+    """Loads libsfb.so (built in-tree by `build.build_library`) and declares the signatures."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise FileNotFoundError(f"{path} not found: build it first (python -m paper_1511_08486_b200.build)")
+    lib = C.CDLL(path)
+    vp = C.c_void_p
+    lib.sfb_create.argtypes = [C.POINTER(sfb_desc), vp, C.POINTER(vp)]
+    lib.sfb_create.restype = C.c_int
+    lib.sfb_destroy.argtypes = [vp]
+    lib.sfb_destroy.restype = C.c_int
+    lib.sfb_sf_buffer_bytes.argtypes = [C.POINTER(sfb_desc)]
+    lib.sfb_sf_buffer_bytes.restype = C.c_size_t
+    lib.sfb_ld.argtypes = [C.POINTER(sfb_desc), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.sfb_ld.restype = C.c_int
+    lib.sfb_compute_factors.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, vp]
+    lib.sfb_compute_factors.restype = C.c_int
+    lib.sfb_pack.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, C.c_uint32]
+    lib.sfb_pack.restype = C.c_int
+    lib.sfb_apply.argtypes = [vp, vp, vp, C.c_float, C.c_int32]
+    lib.sfb_apply.restype = C.c_int
+    lib.sfb_step.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, C.c_float, C.c_int32, C.c_uint32]
+    lib.sfb_step.restype = C.c_int
+    lib.sfb_invalidate.argtypes = [vp]
+    lib.sfb_invalidate.restype = C.c_int
+    lib.sfb_status.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.sfb_status.restype = C.c_int
+    lib.sfb_launch_count.argtypes = [vp]
+    lib.sfb_launch_count.restype = C.c_int64
+    lib.sfb_strerror.argtypes = [C.c_int]
+    lib.sfb_strerror.restype = C.c_char_p
+    if path == LIB_PATH:
+        _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().sfb_strerror(code).decode()
+
+
+def make_desc(model, path, J, D, P, B, v_sparse=0, margin=1.0, nnz_capacity=0) -> sfb_desc:
+    return sfb_desc(MODELS.get(model, model), PATHS.get(path, path), J, D, P, B, int(v_sparse), float(margin),
+                    int(nnz_capacity))
+
+
+def _ptr(t) -> int | None:
+    """Device pointer of a torch tensor (or None)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def make_aux(labels=None, Xb=None, similar=None, rowptr=None, idx=None, val=None, Xdata=None) -> sfb_aux:
+    return sfb_aux(_ptr(labels), _ptr(Xb), _ptr(similar), _ptr(rowptr), _ptr(idx), _ptr(val), _ptr(Xdata))
+
+
+def sfb_sf_buffer_bytes(desc: sfb_desc) -> int:
+    return int(load_library().sfb_sf_buffer_bytes(C.byref(desc)))
+
+
+def sfb_ld(desc: sfb_desc) -> tuple[int, int]:
+    ldu, ldv = C.c_int32(0), C.c_int32(0)
+    r = load_library().sfb_ld(C.byref(desc), C.byref(ldu), C.byref(ldv))
+    if r != SFB_OK:
+        raise SfbError(r, "sfb_ld")
+    return ldu.value, ldv.value
+
+
+class Context:
+    """Owns one sfb_ctx.  Methods carry the C names without the prefix and raise SfbError on a negative code."""
+
+    def __init__(self, desc: sfb_desc, stream: int | None = None):
+        self._lib = load_library()
+        self.desc = desc
+        if stream is None:
+            import torch
+            stream = torch.cuda.current_stream().cuda_stream
+        h = C.c_void_p(None)
+        r = self._lib.sfb_create(C.byref(desc), C.c_void_p(stream), C.byref(h))
+        if r != SFB_OK:
+            raise SfbError(r, "sfb_create")
+        self._h = h
+        self.ldu, self.ldv = sfb_ld(desc)
+        self.sf_buffer_bytes = sfb_sf_buffer_bytes(desc)
+        self.K = desc.P * desc.B
+
+    def _chk(self, r: int, what: str):
+        if r != SFB_OK:
+            raise SfbError(r, what)
+
+    def compute_factors(self, W, X, aux: sfb_aux, U, V=None):
+        self._chk(self._lib.sfb_compute_factors(self._h, _ptr(W), _ptr(X), C.byref(aux), _ptr(U), _ptr(V)),
+                  "sfb_compute_factors")
+
+    def pack(self, U, V, aux: sfb_aux | None, sf_buf, clock: int = 0):
+        a = C.byref(aux) if aux is not None else None
+        self._chk(self._lib.sfb_pack(self._h, _ptr(U), _ptr(V), a, _ptr(sf_buf), clock), "sfb_pack")
+
+    def apply(self, W, sf_buf, eta: float, K: int | None = None):
+        self._chk(self._lib.sfb_apply(self._h, _ptr(W), _ptr(sf_buf), eta, self.K if K is None else K), "sfb_apply")
+
+    def step(self, W, X, aux: sfb_aux, sf_buf, eta: float, K: int | None = None, clock: int = 0):
+        self._chk(self._lib.sfb_step(self._h, _ptr(W), _ptr(X), C.byref(aux), _ptr(sf_buf), eta,
+                                     self.K if K is None else K, clock), "sfb_step")
+
+    def invalidate(self):
+        self._chk(self._lib.sfb_invalidate(self._h), "sfb_invalidate")
+
+    def status(self) -> int:
+        s = C.c_int32(0)
+        self._chk(self._lib.sfb_status(self._h, C.byref(s)), "sfb_status")
+        return s.value
+
+    def launch_count(self) -> int:
+        return int(self._lib.sfb_launch_count(self._h))
+
+    def destroy(self):
+        if self._h is not None and self._h.value:
+            self._lib.sfb_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -1,0 +1,318 @@
+// Host side of the C ABI declared in include/sfb.h: argument checks, workspace, kernel sequencing.
+// Every step of the path runs in the CUDA kernels of this library; there is no CPU fallback.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "umma_api.cuh"
+
+using namespace sfb;
+
+struct sfb_ctx {
+  sfb_desc d;
+  Layout l;
+  cudaStream_t stream;
+  int K;
+  int* dev_status;          // sticky device status word
+  float* z_ws;              // fp32 products z = W a, [K][ldz], when u is stored in another type (bf16 path)
+  int ldz;
+  float* wt_ws;             // SC: atom-major copy of W for the forward
+  __nv_bfloat16* w_shadow;  // bf16 path: bf16 copy of W, refreshed by the apply
+  const void* shadow_of;    // W pointer the shadow currently mirrors (nullptr = stale)
+  UmmaPlan* umma;           // tensor-core plan (tensor maps), TF32 / BF16 paths
+  int64_t launches;
+};
+
+namespace {
+
+bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int check_desc(const sfb_desc* d) {
+  if (d == nullptr) return SFB_ERR_ARG;
+  if (d->model < SFB_MLR || d->model > SFB_SC) return SFB_ERR_ARG;
+  if (d->path < SFB_PATH_F32 || d->path > SFB_PATH_BF16) return SFB_ERR_ARG;
+  if (d->J <= 0 || d->D <= 0 || d->P <= 0 || d->B <= 0) return SFB_ERR_SHAPE;
+  if ((long long)d->P * d->B > (1 << 24)) return SFB_ERR_SHAPE;
+  if (d->model == SFB_SC) {
+    if (!d->v_sparse) return SFB_ERR_UNSUPPORTED;          // dictionary updates take CSR codes
+    if (d->path != SFB_PATH_F32) return SFB_ERR_UNSUPPORTED;
+    if (d->nnz_capacity == 0 || d->nnz_capacity % (32ull * d->P) != 0) return SFB_ERR_SHAPE;
+    if (d->nnz_capacity / d->P > (1ull << 30)) return SFB_ERR_SHAPE;
+  } else if (d->v_sparse) {
+    return SFB_ERR_UNSUPPORTED;
+  }
+  if (d->path == SFB_PATH_BF16 && d->model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (d->path == SFB_PATH_BF16 && (d->D % 8) != 0) return SFB_ERR_SHAPE;   // 16-byte rows of bf16 X and W shadow
+  if (d->path == SFB_PATH_TF32 && (d->D % 4) != 0) return SFB_ERR_SHAPE;   // 16-byte rows of fp32 X and W
+  if (d->model == SFB_DML && !(d->margin > 0.f)) return SFB_ERR_ARG;
+  return SFB_OK;
+}
+
+RowMap caller_rows(const void* base, int ld, int B, int es) {
+  RowMap m;
+  m.base = const_cast<char*>(reinterpret_cast<const char*>(base));
+  m.worker_stride = (long long)B * ld * es;
+  m.ld = ld; m.B = B; m.es = es;
+  return m;
+}
+RowMap stream_u(const sfb_ctx* c, const void* sf_buf) {
+  RowMap m;
+  m.base = const_cast<char*>(reinterpret_cast<const char*>(sf_buf)) + c->l.streams_off;
+  m.worker_stride = c->l.stream_stride;
+  m.ld = c->l.ldu; m.B = c->d.B; m.es = c->l.es;
+  return m;
+}
+RowMap stream_v(const sfb_ctx* c, const void* sf_buf) {
+  RowMap m = stream_u(c, sf_buf);
+  m.base += c->l.u_bytes;
+  m.ld = c->l.ldv;
+  return m;
+}
+RowMap z_rows(const sfb_ctx* c) { return caller_rows(c->z_ws, c->ldz, c->d.B, 4); }
+
+CsrView global_codes(const sfb_aux* a, int B) {
+  CsrView v;
+  memset(&v, 0, sizeof(v));
+  v.rowptr = a->rowptr; v.idx = a->idx; v.val = reinterpret_cast<const float*>(a->val); v.B = B;
+  return v;
+}
+CsrView stream_codes(const sfb_ctx* c, const void* sf_buf) {
+  CsrView v;
+  memset(&v, 0, sizeof(v));
+  v.base = reinterpret_cast<const char*>(sf_buf);
+  v.streams_off = c->l.streams_off; v.stream_stride = c->l.stream_stride; v.v_off = c->l.u_bytes;
+  v.rp_bytes = c->l.rp_bytes; v.idx_bytes = c->l.idx_bytes; v.B = c->d.B;
+  return v;
+}
+
+int check_aux(const sfb_ctx* c, const sfb_aux* a) {
+  if (a == nullptr) return SFB_ERR_ARG;
+  switch (c->d.model) {
+    case SFB_MLR: return (a->labels != nullptr && aligned(a->labels, 4)) ? SFB_OK : SFB_ERR_ARG;
+    case SFB_DML: return (a->Xb != nullptr && a->similar != nullptr && aligned(a->Xb, 16)) ? SFB_OK : SFB_ERR_ARG;
+    default:
+      return (a->rowptr && a->idx && a->val && a->Xdata && aligned(a->rowptr, 4) && aligned(a->idx, 4) &&
+              aligned(a->val, 4) && aligned(a->Xdata, 4)) ? SFB_OK : SFB_ERR_ARG;
+  }
+}
+
+#define ACC(expr)                  \
+  do {                             \
+    const int r_ = (expr);         \
+    if (r_ < 0) return r_;         \
+    c->launches += r_;             \
+  } while (0)
+
+// Refreshes the bf16 shadow of W if it does not mirror this W.
+int ensure_shadow(sfb_ctx* c, const void* W) {
+  if (c->d.path != SFB_PATH_BF16 || c->shadow_of == W) return SFB_OK;
+  ACC(launch_cast_bf16(c->stream, reinterpret_cast<const float*>(W), c->w_shadow, (long long)c->d.J * c->d.D));
+  c->shadow_of = W;
+  return SFB_OK;
+}
+
+// Factors of one minibatch written through the row maps u / v (v.base == nullptr: v not wanted).
+int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, RowMap u, RowMap v, CsrView codes) {
+  const sfb_desc& d = c->d;
+  const float* Wf = reinterpret_cast<const float*>(W);
+  if (d.model == SFB_SC) {
+    ACC(launch_sc_forward_ws(c->stream, Wf, c->wt_ws, codes, reinterpret_cast<const float*>(aux->Xdata), u, c->K, d.J,
+                             d.D, c->dev_status));
+    return SFB_OK;
+  }
+  if (d.path == SFB_PATH_F32) {
+    const float* Xb = (d.model == SFB_DML) ? reinterpret_cast<const float*>(aux->Xb) : nullptr;
+    ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, c->K, d.J, d.D, u, v));
+    if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, u, u, aux->labels, c->K, d.J, c->dev_status));
+    else ACC(launch_finish_dml(c->stream, u, u, aux->similar, d.margin, c->K, d.J));
+    return SFB_OK;
+  }
+  // tensor-core paths
+  if (d.path == SFB_PATH_BF16) {
+    const int r = ensure_shadow(c, W);
+    if (r < 0) return r;
+  }
+  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, z_rows(c), c->dev_status));
+  return SFB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sfb_strerror(int code) {
+  switch (code) {
+    case SFB_OK: return "ok";
+    case SFB_ERR_ARG: return "bad argument (null or misaligned pointer, bad enum, K not a whole number of worker streams)";
+    case SFB_ERR_SHAPE: return "unsupported sizes";
+    case SFB_ERR_UNSUPPORTED: return "model/path combination not provided, or not an sm_100 device";
+    case SFB_ERR_CUDA: return "a CUDA call failed";
+    case SFB_ERR_ALLOC: return "workspace allocation failed";
+    default: return "unknown error";
+  }
+}
+
+size_t sfb_sf_buffer_bytes(const sfb_desc* desc) {
+  if (check_desc(desc) != SFB_OK) return 0;
+  return (size_t)make_layout(*desc).total_bytes;
+}
+
+int sfb_ld(const sfb_desc* desc, int32_t* ldu, int32_t* ldv) {
+  const int r = check_desc(desc);
+  if (r != SFB_OK) return r;
+  const Layout l = make_layout(*desc);
+  if (ldu) *ldu = l.ldu;
+  if (ldv) *ldv = l.ldv;
+  return SFB_OK;
+}
+
+int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
+  if (out == nullptr) return SFB_ERR_ARG;
+  *out = nullptr;
+  const int r = check_desc(desc);
+  if (r != SFB_OK) return r;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SFB_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SFB_ERR_CUDA;
+  if (major != 10) return SFB_ERR_UNSUPPORTED;   // kernels are built for sm_100a only
+  sfb_ctx* c = new (std::nothrow) sfb_ctx();
+  if (c == nullptr) return SFB_ERR_ALLOC;
+  memset(c, 0, sizeof(*c));
+  c->d = *desc;
+  c->l = make_layout(*desc);
+  c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  c->K = desc->P * desc->B;
+  bool ok = cudaMalloc(&c->dev_status, 256) == cudaSuccess;
+  if (ok) ok = cudaMemsetAsync(c->dev_status, 0, 256, c->stream) == cudaSuccess;
+  if (ok && desc->model == SFB_SC) ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
+  if (ok && desc->path != SFB_PATH_F32) {
+    c->ldz = (int)pad_to(desc->J, 4);
+    ok = cudaMalloc(&c->z_ws, (size_t)c->K * c->ldz * 4) == cudaSuccess;
+  }
+  if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    sfb_destroy(c);
+    return SFB_ERR_ALLOC;
+  }
+  if (desc->path != SFB_PATH_F32) {
+    const int ur = umma_plan_create(c->d, c->l, c->z_ws, c->ldz, c->w_shadow, &c->umma);
+    if (ur != SFB_OK) {
+      sfb_destroy(c);
+      return ur;
+    }
+  }
+  *out = c;
+  return SFB_OK;
+}
+
+int sfb_destroy(sfb_ctx* c) {
+  if (c == nullptr) return SFB_ERR_ARG;
+  cudaStreamSynchronize(c->stream);
+  if (c->umma) umma_plan_destroy(c->umma);
+  if (c->dev_status) cudaFree(c->dev_status);
+  if (c->z_ws) cudaFree(c->z_ws);
+  if (c->wt_ws) cudaFree(c->wt_ws);
+  if (c->w_shadow) cudaFree(c->w_shadow);
+  delete c;
+  return SFB_OK;
+}
+
+int sfb_invalidate(sfb_ctx* c) {
+  if (c == nullptr) return SFB_ERR_ARG;
+  c->shadow_of = nullptr;
+  return SFB_OK;
+}
+
+int64_t sfb_launch_count(const sfb_ctx* c) { return c ? c->launches : 0; }
+
+int sfb_status(sfb_ctx* c, int32_t* device_status) {
+  if (c == nullptr || device_status == nullptr) return SFB_ERR_ARG;
+  int32_t h = 0;
+  if (cudaMemcpyAsync(&h, c->dev_status, 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  if (cudaMemsetAsync(c->dev_status, 0, 4, c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  *device_status = h;
+  return SFB_OK;
+}
+
+int sfb_compute_factors(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, void* U, void* V) {
+  if (c == nullptr || W == nullptr || U == nullptr) return SFB_ERR_ARG;
+  if (!aligned(W, 16) || !aligned(U, 16) || (V != nullptr && !aligned(V, 16))) return SFB_ERR_ARG;
+  int r = check_aux(c, aux);
+  if (r != SFB_OK) return r;
+  if (c->d.model != SFB_SC && (X == nullptr || !aligned(X, 16))) return SFB_ERR_ARG;
+  RowMap u = caller_rows(U, c->l.ldu, c->d.B, c->l.es);
+  RowMap v = caller_rows(c->d.model == SFB_SC ? nullptr : V, c->l.ldv, c->d.B, c->l.es);
+  return factors_into(c, W, X, aux, u, v, c->d.model == SFB_SC ? global_codes(aux, c->d.B) : CsrView());
+}
+
+int sfb_pack(sfb_ctx* c, const void* U, const void* V, const sfb_aux* aux, void* sf_buf, uint32_t clock) {
+  if (c == nullptr || U == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
+  if (!aligned(U, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
+  const sfb_desc& d = c->d;
+  const uint32_t* rowptr = nullptr;
+  if (d.v_sparse) {
+    if (aux == nullptr || aux->rowptr == nullptr || aux->idx == nullptr || aux->val == nullptr) return SFB_ERR_ARG;
+    rowptr = aux->rowptr;
+  } else if (V == nullptr || !aligned(V, 16)) {
+    return SFB_ERR_ARG;
+  }
+  ACC(launch_copy_rows(c->stream, caller_rows(U, c->l.ldu, d.B, c->l.es), stream_u(c, sf_buf), c->K, d.J));
+  if (d.v_sparse)
+    ACC(launch_pack_csr(c->stream, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
+                        c->dev_status));
+  else
+    ACC(launch_copy_rows(c->stream, caller_rows(V, c->l.ldv, d.B, c->l.es), stream_v(c, sf_buf), c->K, d.D));
+  ACC(launch_write_header(c->stream, sf_buf, d, c->l, clock, rowptr));
+  return SFB_OK;
+}
+
+static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check) {
+  const sfb_desc& d = c->d;
+  if (check) ACC(launch_check_header(c->stream, sf_buf, d, c->l, c->dev_status));
+  if (d.v_sparse) {
+    ACC(launch_sc_apply(c->stream, reinterpret_cast<float*>(W), stream_codes(c, sf_buf), stream_u(c, sf_buf), K, d.J,
+                        d.D, eta, c->dev_status, c->dev_status));
+  } else if (d.path == SFB_PATH_F32) {
+    ACC(launch_apply_f32(c->stream, reinterpret_cast<float*>(W), stream_u(c, sf_buf), stream_v(c, sf_buf), K, d.J, d.D,
+                         eta, c->dev_status));
+  } else {
+    ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, sf_buf, eta, K, c->dev_status));
+    if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
+  }
+  return SFB_OK;
+}
+
+int sfb_apply(sfb_ctx* c, void* W, const void* sf_buf, float eta, int32_t K) {
+  if (c == nullptr || W == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
+  if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
+  if (K <= 0 || K > c->K || (K % c->d.B) != 0) return SFB_ERR_ARG;
+  if (c->d.path == SFB_PATH_BF16 && c->shadow_of != W) c->shadow_of = nullptr;
+  return apply_from(c, W, sf_buf, eta, K, true);
+}
+
+int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_buf, float eta, int32_t K,
+             uint32_t clock) {
+  if (c == nullptr || W == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
+  if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
+  if (K <= 0 || K > c->K || (K % c->d.B) != 0) return SFB_ERR_ARG;
+  int r = check_aux(c, aux);
+  if (r != SFB_OK) return r;
+  const sfb_desc& d = c->d;
+  if (d.model != SFB_SC && (X == nullptr || !aligned(X, 16))) return SFB_ERR_ARG;
+  CsrView codes;
+  memset(&codes, 0, sizeof(codes));
+  if (d.v_sparse) {
+    ACC(launch_pack_csr(c->stream, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
+                        c->dev_status));
+    codes = stream_codes(c, sf_buf);   // the forward reads the codes it just committed to the buffer
+  }
+  r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes);
+  if (r < 0) return r;
+  ACC(launch_write_header(c->stream, sf_buf, d, c->l, clock, d.v_sparse ? aux->rowptr : nullptr));
+  return apply_from(c, W, sf_buf, eta, K, false);
+}
+
+}  // extern "C"

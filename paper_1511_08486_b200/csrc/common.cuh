@@ -1,0 +1,112 @@
+// Shared declarations of the SF hot-path kernels (internal; the public boundary is include/sfb.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sfb.h"
+
+namespace sfb {
+
+// Where the K factor rows of one operand live: row i of worker p = i / B sits at
+// base + p * worker_stride + (i % B) * ld * elem_size.  Covers both caller-side [K][ld] arrays
+// (worker_stride = B * ld * elem_size) and the U / V blocks of the SF buffer's worker streams.
+struct RowMap {
+  char* base;
+  long long worker_stride;  // bytes
+  int ld;                   // values per row (padded)
+  int B;                    // rows per worker
+  int es;                   // bytes per value (4 = fp32, 2 = bf16)
+  __host__ __device__ __forceinline__ char* row(int i) const {
+    return base + (long long)(i / B) * worker_stride + (long long)(i % B) * ld * es;
+  }
+};
+
+// Byte layout of the SF buffer for one descriptor (see the wire format in include/sfb.h).
+struct Layout {
+  int es, ldu, ldv, cap_p;
+  long long u_bytes, v_bytes, rp_bytes, idx_bytes, val_bytes;
+  long long stream_stride, streams_off, total_bytes;
+};
+
+static inline long long pad_to(long long n, long long a) { return (n + a - 1) / a * a; }
+
+static inline Layout make_layout(const sfb_desc& d) {
+  Layout l;
+  l.es = (d.path == SFB_PATH_BF16) ? 2 : 4;
+  const int unit = 16 / l.es;
+  l.ldu = (int)pad_to(d.J, unit);
+  l.ldv = (int)pad_to(d.D, unit);
+  l.cap_p = d.v_sparse ? (int)(d.nnz_capacity / (uint64_t)d.P) : 0;
+  l.u_bytes = pad_to((long long)d.B * l.ldu * l.es, 128);
+  if (d.v_sparse) {
+    l.rp_bytes = pad_to((long long)(d.B + 1) * 4, 128);
+    l.idx_bytes = pad_to((long long)l.cap_p * 4, 128);
+    l.val_bytes = pad_to((long long)l.cap_p * l.es, 128);
+    l.v_bytes = l.rp_bytes + l.idx_bytes + l.val_bytes;
+  } else {
+    l.rp_bytes = l.idx_bytes = l.val_bytes = 0;
+    l.v_bytes = pad_to((long long)d.B * l.ldv * l.es, 128);
+  }
+  l.stream_stride = l.u_bytes + l.v_bytes;
+  l.streams_off = 128 + pad_to((long long)d.P * 32, 128);
+  l.total_bytes = l.streams_off + (long long)d.P * l.stream_stride;
+  return l;
+}
+
+// ---- kernel launchers (each returns the number of kernels it launched, or a negative SFB_ERR_*) ----
+
+// Z[i][j] = sum_d A[i][d] * W[j][d] on fp32 CUDA cores, written as fp32 rows through `z`.
+// A = X, or X - Xb (element-wise fp32 subtraction) when Xb != nullptr.  When `v` has a base, the
+// operand rows (X, or the difference) are also written there (the factor v), pad columns zero.
+int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
+                       RowMap z, RowMap v);
+
+// W[j][d] -= eta * sum_{i<K} U[i][j] * V[i][d] on fp32 CUDA cores (fixed summation order).
+int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J, int D, float eta,
+                     const int* dev_status);
+
+// MLR epilogue: u = softmax(z) - onehot(label).  z rows are fp32; u rows fp32 or bf16 (u.es).
+int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status);
+
+// DML epilogue: u = +z (similar) or -z * [|z|^2 < margin] (dissimilar).
+int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J);
+
+// Copies K rows of `cols` values from src to dst rows (same value type), zero-filling dst pad columns.
+int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols);
+
+// Writes header and directory of the SF buffer.  `rowptr` (global CSR row pointers) only for sparse v.
+int launch_write_header(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, uint32_t clock,
+                        const uint32_t* rowptr);
+
+// Copies the CSR codes of every worker into its stream (local row pointers, zero-filled tail).
+int launch_pack_csr(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, const uint32_t* rowptr,
+                    const uint32_t* idx, const float* val, int* dev_status);
+
+// Sets SFB_DEV_BAD_HEADER in *dev_status unless the buffer's header matches the descriptor.
+int launch_check_header(cudaStream_t s, const void* sf_buf, const sfb_desc& d, const Layout& l, int* dev_status);
+
+// SC forward: u_i = sum_{(d,a) in code i} a * W[:, d] - x_i, codes read from CSR arrays whose row
+// pointers are either global ([K+1]) or per worker stream inside the SF buffer.
+struct CsrView {
+  const char* base;          // SF buffer base, or nullptr for caller-side global arrays
+  const uint32_t* rowptr;    // global arrays (base == nullptr)
+  const uint32_t* idx;
+  const float* val;
+  long long streams_off, stream_stride, v_off, rp_bytes, idx_bytes;  // stream-relative offsets (base != nullptr)
+  int B;
+};
+// Wt is a caller-provided workspace of sc_forward_workspace_bytes(J, D) bytes (atom-major copy of W).
+long long sc_forward_workspace_bytes(int J, int D);
+int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView codes, const float* Xdata, RowMap u, int K,
+                         int J, int D, int* dev_status);
+
+// SC apply: W[:, d] -= eta * sum_{i: a_id != 0} a_id * u_i (sparse-v scatter, no float atomics).
+int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
+                    const int* dev_status_ro, int* dev_status);
+
+// W (fp32) -> bf16 shadow, round to nearest even.
+int launch_cast_bf16(cudaStream_t s, const float* W, __nv_bfloat16* Wb, long long n);
+
+}  // namespace sfb

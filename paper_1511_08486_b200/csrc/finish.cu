@@ -1,0 +1,260 @@
+// Bandwidth-bound passes of the factor computation: the model epilogues that turn the products
+// z_i = W a_i into the factor u_i, row copies, and the fp32 -> bf16 cast of W.
+//
+//   MLR  u_i = softmax(z_i) - onehot(y_i)   (chain rule on the multiclass logistic loss; Section 2.1)
+//   DML  u_i = +z_i (similar pair) | -z_i * [|z_i|^2 < margin] (dissimilar pair)   (Section 2, DML)
+//
+// One thread block per sample row; the row is staged once in shared memory (when it fits) so HBM
+// sees one read and one write per value; reductions over the J entries use warp shuffles.
+#include "common.cuh"
+
+namespace sfb {
+namespace {
+
+constexpr int FIN_THREADS = 256;
+constexpr int ROW_CACHE_FLOATS = 48 * 1024;   // 192 KB of dynamic shared memory
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+// Block-wide reductions with a fixed combination order (bit-reproducible).
+__device__ float block_max(float v, float* red) {
+  v = warp_max(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) red[w] = v;
+  __syncthreads();
+  float r = (l < (int)(blockDim.x >> 5)) ? red[l] : -INFINITY;
+  return warp_max(r);
+}
+__device__ float block_sum(float v, float* red) {
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) red[w] = v;
+  __syncthreads();
+  float r = (l < (int)(blockDim.x >> 5)) ? red[l] : 0.f;
+  return warp_sum(r);
+}
+
+// Stores 4 consecutive values starting at column j (j % 4 == 0, j + 3 < ld).
+__device__ __forceinline__ void store_u4(char* row, int j, float4 v, int es) {
+  if (es == 4) {
+    *reinterpret_cast<float4*>(row + (size_t)j * 4) = v;
+  } else {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 p;
+    p.x = *reinterpret_cast<uint32_t*>(&lo);
+    p.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(row + (size_t)j * 2) = p;
+  }
+}
+
+// z rows are fp32 with ld a multiple of 4; values beyond J inside the last float4 are ignored.
+__global__ void __launch_bounds__(FIN_THREADS) finish_mlr_kernel(RowMap z, RowMap u, const int32_t* __restrict__ labels,
+                                                                 int K, int J, int cache_floats, int* dev_status) {
+  extern __shared__ __align__(16) float cache[];
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  if (i >= K) return;
+  const float* zr = reinterpret_cast<const float*>(z.row(i));
+  char* ur = u.row(i);
+  const int J4 = (J + 3) >> 2;
+  const bool cached = (J4 * 4) <= cache_floats;
+  const float kLog2e = 1.4426950408889634f;
+
+  float m = -INFINITY;
+  for (int q = threadIdx.x; q < J4; q += FIN_THREADS) {
+    float4 t = *reinterpret_cast<const float4*>(zr + q * 4);
+    const int j = q * 4;
+    if (j + 1 >= J) t.y = -INFINITY;
+    if (j + 2 >= J) t.z = -INFINITY;
+    if (j + 3 >= J) t.w = -INFINITY;
+    if (cached) *reinterpret_cast<float4*>(cache + j) = t;
+    m = fmaxf(fmaxf(fmaxf(m, t.x), fmaxf(t.y, t.z)), t.w);
+  }
+  m = block_max(m, red);
+
+  float s = 0.f;
+  const float mb = m * kLog2e;
+  for (int q = threadIdx.x; q < J4; q += FIN_THREADS) {
+    const int j = q * 4;
+    float4 t;
+    if (cached) {
+      t = *reinterpret_cast<const float4*>(cache + j);
+    } else {
+      t = *reinterpret_cast<const float4*>(zr + j);
+      if (j + 1 >= J) t.y = -INFINITY;
+      if (j + 2 >= J) t.z = -INFINITY;
+      if (j + 3 >= J) t.w = -INFINITY;
+    }
+    t.x = exp2f(fmaf(t.x, kLog2e, -mb)); t.y = exp2f(fmaf(t.y, kLog2e, -mb));
+    t.z = exp2f(fmaf(t.z, kLog2e, -mb)); t.w = exp2f(fmaf(t.w, kLog2e, -mb));
+    if (cached) *reinterpret_cast<float4*>(cache + j) = t;
+    s += (t.x + t.y) + (t.z + t.w);
+  }
+  s = block_sum(s, red);
+  const float inv = 1.0f / s;
+
+  const int y = labels[i];
+  const bool bad = (y < 0) || (y >= J);
+  if (bad && threadIdx.x == 0) atomicOr(dev_status, SFB_DEV_BAD_LABEL);
+  const int ld4 = u.ld >> 2;   // u.ld is a multiple of 4 (fp32) or 8 (bf16)
+  for (int q = threadIdx.x; q < ld4; q += FIN_THREADS) {
+    const int j = q * 4;
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q < J4 && !bad) {
+      if (cached) {
+        t = *reinterpret_cast<const float4*>(cache + j);
+      } else {
+        t = *reinterpret_cast<const float4*>(zr + j);
+        t.x = exp2f(fmaf(t.x, kLog2e, -mb)); t.y = exp2f(fmaf(t.y, kLog2e, -mb));
+        t.z = exp2f(fmaf(t.z, kLog2e, -mb)); t.w = exp2f(fmaf(t.w, kLog2e, -mb));
+      }
+      t.x *= inv; t.y *= inv; t.z *= inv; t.w *= inv;
+      if (y == j) t.x -= 1.f;
+      if (y == j + 1) t.y -= 1.f;
+      if (y == j + 2) t.z -= 1.f;
+      if (y == j + 3) t.w -= 1.f;
+      if (j + 1 >= J) t.y = 0.f;
+      if (j + 2 >= J) t.z = 0.f;
+      if (j + 3 >= J) t.w = 0.f;
+    }
+    store_u4(ur, j, t, u.es);
+  }
+}
+
+__global__ void __launch_bounds__(FIN_THREADS) finish_dml_kernel(RowMap z, RowMap u, const uint8_t* __restrict__ similar,
+                                                                 float margin, int K, int J, int cache_floats) {
+  extern __shared__ __align__(16) float cache[];
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  if (i >= K) return;
+  const float* zr = reinterpret_cast<const float*>(z.row(i));
+  char* ur = u.row(i);
+  const int J4 = (J + 3) >> 2;
+  const bool cached = (J4 * 4) <= cache_floats;
+
+  float n = 0.f;
+  for (int q = threadIdx.x; q < J4; q += FIN_THREADS) {
+    float4 t = *reinterpret_cast<const float4*>(zr + q * 4);
+    const int j = q * 4;
+    if (j + 1 >= J) t.y = 0.f;
+    if (j + 2 >= J) t.z = 0.f;
+    if (j + 3 >= J) t.w = 0.f;
+    if (cached) *reinterpret_cast<float4*>(cache + j) = t;
+    n += (t.x * t.x + t.y * t.y) + (t.z * t.z + t.w * t.w);
+  }
+  n = block_sum(n, red);
+  const bool sim = similar[i] != 0;
+  const float g = sim ? 1.f : ((n < margin) ? -1.f : 0.f);   // strict hinge: inactive at equality
+
+  const int ld4 = u.ld >> 2;
+  for (int q = threadIdx.x; q < ld4; q += FIN_THREADS) {
+    const int j = q * 4;
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q < J4 && g != 0.f) {
+      t = cached ? *reinterpret_cast<const float4*>(cache + j) : *reinterpret_cast<const float4*>(zr + j);
+      t.x *= g; t.y *= g; t.z *= g; t.w *= g;
+      if (j + 1 >= J) t.y = 0.f;
+      if (j + 2 >= J) t.z = 0.f;
+      if (j + 3 >= J) t.w = 0.f;
+    }
+    store_u4(ur, j, t, u.es);
+  }
+}
+
+// 16-byte-vectorised row copy; rows are whole numbers of 16-byte units on both sides.
+__global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, int K, int cols) {
+  const int units_dst = dst.ld * dst.es / 16;
+  const int per = 16 / dst.es;
+  const long long total = (long long)K * units_dst;
+  for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
+       g += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(g / units_dst), q = (int)(g % units_dst);
+    const int c = q * per;
+    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+    if (c < cols && c < src.ld) {
+      val = *reinterpret_cast<const uint4*>(src.row(i) + (size_t)q * 16);
+      if (c + per > cols) {   // mask the tail beyond `cols`
+        if (dst.es == 4) {
+          uint32_t* w = reinterpret_cast<uint32_t*>(&val);
+          for (int e = 0; e < 4; ++e)
+            if (c + e >= cols) w[e] = 0u;
+        } else {
+          uint16_t* h = reinterpret_cast<uint16_t*>(&val);
+          for (int e = 0; e < 8; ++e)
+            if (c + e >= cols) h[e] = 0;
+        }
+      }
+    }
+    *reinterpret_cast<uint4*>(dst.row(i) + (size_t)q * 16) = val;
+  }
+}
+
+__global__ void __launch_bounds__(256) cast_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wb,
+                                                        long long n4) {
+  for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n4; g += (long long)gridDim.x * blockDim.x) {
+    const float4 t = reinterpret_cast<const float4*>(W)[g];
+    __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
+    uint2 p;
+    p.x = *reinterpret_cast<uint32_t*>(&lo);
+    p.y = *reinterpret_cast<uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(Wb)[g] = p;
+  }
+}
+
+int fin_cache_floats(int J) {
+  const int need = ((J + 3) / 4) * 4;
+  return need <= ROW_CACHE_FLOATS ? need : 0;
+}
+
+}  // namespace
+
+int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status) {
+  const int cf = fin_cache_floats(J);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(finish_mlr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
+    cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
+    attr_done = true;
+  }
+  finish_mlr_kernel<<<K, FIN_THREADS, (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J) {
+  const int cf = fin_cache_floats(J);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(finish_mlr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
+    cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
+    attr_done = true;
+  }
+  finish_dml_kernel<<<K, FIN_THREADS, (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols) {
+  const long long total = (long long)K * (dst.ld * dst.es / 16);
+  if (total == 0) return 0;
+  const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
+  copy_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, K, cols);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_cast_bf16(cudaStream_t s, const float* W, __nv_bfloat16* Wb, long long n) {
+  const long long n4 = n / 4;   // J*D is a multiple of 4 on the bf16 path (D % 8 == 0 is required there)
+  const int blocks = (int)((n4 + 255) / 256 < 148LL * 16 ? (n4 + 255) / 256 : 148LL * 16);
+  cast_bf16_kernel<<<blocks, 256, 0, s>>>(W, Wb, n4);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+}  // namespace sfb

@@ -1,0 +1,243 @@
+// fp32 CUDA-core contractions of the SF hot path.
+//
+//   forward:  Z[i][j] = sum_d A[i][d] * W[j][d]      (z_i = W a_i for every sample; Section 2, (P))
+//   apply  :  W[j][d] -= eta * sum_i U[i][j] * V[i][d]  (W <- W - eta * sum_i u_i v_i^T; Section 3)
+//
+// Both are register-blocked shared-memory SGEMMs: 256 threads, a (64*MI) x (64*NI) output tile, a
+// reduction step of 16, operands staged k-major in shared memory so that every inner-loop read is
+// a conflict-free 16-byte load, global loads prefetched into registers one step ahead.  The
+// summation order is fixed (ascending reduction index inside one thread), so results are
+// bit-reproducible run to run.
+#include "common.cuh"
+
+namespace sfb {
+namespace {
+
+constexpr int BK = 16;
+
+__device__ __forceinline__ float4 ld4_guard(const float* row, int c, int cols, bool vec_ok) {
+  // row: start of a row; c: first column (multiple of 4); cols: valid columns
+  if (vec_ok && c + 3 < cols) return *reinterpret_cast<const float4*>(row + c);
+  float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c < cols) r.x = row[c];
+  if (c + 1 < cols) r.y = row[c + 1];
+  if (c + 2 < cols) r.z = row[c + 2];
+  if (c + 3 < cols) r.w = row[c + 3];
+  return r;
+}
+
+template <int MI, int NI>
+__device__ __forceinline__ void mma_tile(const float (*As)[64 * MI + 4], const float (*Bs)[64 * NI + 4], int ty,
+                                         int tx, float (&acc)[4 * MI][4 * NI]) {
+#pragma unroll
+  for (int k = 0; k < BK; ++k) {
+    float a[4 * MI], b[4 * NI];
+#pragma unroll
+    for (int mi = 0; mi < MI; ++mi) {
+      float4 t = *reinterpret_cast<const float4*>(&As[k][mi * 64 + ty * 4]);
+      a[mi * 4 + 0] = t.x; a[mi * 4 + 1] = t.y; a[mi * 4 + 2] = t.z; a[mi * 4 + 3] = t.w;
+    }
+#pragma unroll
+    for (int ni = 0; ni < NI; ++ni) {
+      float4 t = *reinterpret_cast<const float4*>(&Bs[k][ni * 64 + tx * 4]);
+      b[ni * 4 + 0] = t.x; b[ni * 4 + 1] = t.y; b[ni * 4 + 2] = t.z; b[ni * 4 + 3] = t.w;
+    }
+#pragma unroll
+    for (int m = 0; m < 4 * MI; ++m)
+#pragma unroll
+      for (int n = 0; n < 4 * NI; ++n) acc[m][n] = fmaf(a[m], b[n], acc[m][n]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ forward
+// Tile rows = samples i (BM = 64*MI), tile columns = classes j (BN = 64*NI), reduction over d.
+// Both operands are contiguous along d, so tiles are transposed while being stored to shared memory.
+template <int MI, int NI>
+__global__ void __launch_bounds__(256) forward_f32_kernel(const float* __restrict__ W, const float* __restrict__ X,
+                                                          const float* __restrict__ Xb, int K, int J, int D,
+                                                          RowMap z, RowMap v) {
+  constexpr int BM = 64 * MI, BN = 64 * NI;
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int i0 = blockIdx.y * BM, j0 = blockIdx.x * BN;
+  const bool vec_ok = (D & 3) == 0;
+  const bool write_v = (v.base != nullptr) && (blockIdx.x == 0);
+  const int lr = tid >> 2, lc = (tid & 3) * 4;   // loader: row within 64, first of 4 reduction columns
+
+  float acc[4 * MI][4 * NI];
+#pragma unroll
+  for (int m = 0; m < 4 * MI; ++m)
+#pragma unroll
+    for (int n = 0; n < 4 * NI; ++n) acc[m][n] = 0.f;
+
+  float4 pa[MI], pb[NI];
+  auto fetch = [&](int d0) {
+#pragma unroll
+    for (int q = 0; q < MI; ++q) {
+      const int i = i0 + lr + 64 * q;
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < K) {
+        a = ld4_guard(X + (size_t)i * D, d0 + lc, D, vec_ok);
+        if (Xb != nullptr) {
+          const float4 b = ld4_guard(Xb + (size_t)i * D, d0 + lc, D, vec_ok);
+          a.x = __fsub_rn(a.x, b.x); a.y = __fsub_rn(a.y, b.y); a.z = __fsub_rn(a.z, b.z); a.w = __fsub_rn(a.w, b.w);
+        }
+        if (write_v && d0 + lc < v.ld) *reinterpret_cast<float4*>(v.row(i) + (size_t)(d0 + lc) * 4) = a;
+      }
+      pa[q] = a;
+    }
+#pragma unroll
+    for (int q = 0; q < NI; ++q) {
+      const int j = j0 + lr + 64 * q;
+      pb[q] = (j < J) ? ld4_guard(W + (size_t)j * D, d0 + lc, D, vec_ok) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int q = 0; q < MI; ++q) {
+      As[lc + 0][lr + 64 * q] = pa[q].x; As[lc + 1][lr + 64 * q] = pa[q].y;
+      As[lc + 2][lr + 64 * q] = pa[q].z; As[lc + 3][lr + 64 * q] = pa[q].w;
+    }
+#pragma unroll
+    for (int q = 0; q < NI; ++q) {
+      Bs[lc + 0][lr + 64 * q] = pb[q].x; Bs[lc + 1][lr + 64 * q] = pb[q].y;
+      Bs[lc + 2][lr + 64 * q] = pb[q].z; Bs[lc + 3][lr + 64 * q] = pb[q].w;
+    }
+  };
+
+  fetch(0);
+  for (int d0 = 0; d0 < D; d0 += BK) {
+    stash();
+    __syncthreads();
+    if (d0 + BK < D) fetch(d0 + BK);
+    mma_tile<MI, NI>(As, Bs, ty, tx, acc);
+    __syncthreads();
+  }
+  // The factor v has pad columns [D, ldv): the last loader step wrote zeros there only when
+  // D..ldv falls inside a fetched float4, which holds because ldv = D rounded up to 4.
+
+#pragma unroll
+  for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int i = i0 + mi * 64 + ty * 4 + a;
+      if (i >= K) continue;
+      float* zr = reinterpret_cast<float*>(z.row(i));
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni) {
+        const int j = j0 + ni * 64 + tx * 4;
+        if (j < z.ld)   // ld is a multiple of 4, so the whole float4 is inside the row; columns >= J hold 0
+          *reinterpret_cast<float4*>(zr + j) = make_float4(acc[mi * 4 + a][ni * 4 + 0], acc[mi * 4 + a][ni * 4 + 1],
+                                                           acc[mi * 4 + a][ni * 4 + 2], acc[mi * 4 + a][ni * 4 + 3]);
+      }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ apply
+// Tile rows = rows j of W (BM), tile columns = columns d of W (BN), reduction over the K factors.
+// U rows are contiguous along j and V rows along d: tiles go to shared memory as they are.
+template <int MI, int NI>
+__global__ void __launch_bounds__(256) apply_f32_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
+                                                        int D, float eta, const int* __restrict__ dev_status) {
+  constexpr int BM = 64 * MI, BN = 64 * NI;
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
+  if (dev_status != nullptr && (*dev_status & SFB_DEV_BAD_HEADER)) return;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int j0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
+  const int lr = tid >> 4, lc = (tid & 15) * 4;   // loader: factor row within 16, first of 4 columns
+
+  float acc[4 * MI][4 * NI];
+#pragma unroll
+  for (int m = 0; m < 4 * MI; ++m)
+#pragma unroll
+    for (int n = 0; n < 4 * NI; ++n) acc[m][n] = 0.f;
+
+  float4 pa[MI], pb[NI];
+  auto fetch = [&](int k0) {
+    const int i = k0 + lr;
+#pragma unroll
+    for (int q = 0; q < MI; ++q) {
+      const int j = j0 + lc + 64 * q;
+      pa[q] = (i < K) ? ld4_guard(reinterpret_cast<const float*>(u.row(i)), j, J, true)
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int q = 0; q < NI; ++q) {
+      const int d = d0 + lc + 64 * q;
+      pb[q] = (i < K) ? ld4_guard(reinterpret_cast<const float*>(v.row(i)), d, D, true)
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int q = 0; q < MI; ++q) *reinterpret_cast<float4*>(&As[lr][lc + 64 * q]) = pa[q];
+#pragma unroll
+    for (int q = 0; q < NI; ++q) *reinterpret_cast<float4*>(&Bs[lr][lc + 64 * q]) = pb[q];
+  };
+
+  fetch(0);
+  for (int k0 = 0; k0 < K; k0 += BK) {
+    stash();
+    __syncthreads();
+    if (k0 + BK < K) fetch(k0 + BK);
+    mma_tile<MI, NI>(As, Bs, ty, tx, acc);
+    __syncthreads();
+  }
+
+  const bool vec_ok = (D & 3) == 0;
+#pragma unroll
+  for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int j = j0 + mi * 64 + ty * 4 + a;
+      if (j >= J) continue;
+      float* wr = W + (size_t)j * D;
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni) {
+        const int d = d0 + ni * 64 + tx * 4;
+        const float* c = acc[mi * 4 + a] + ni * 4;
+        if (vec_ok && d + 3 < D) {
+          float4 w = *reinterpret_cast<float4*>(wr + d);
+          w.x = fmaf(-eta, c[0], w.x); w.y = fmaf(-eta, c[1], w.y);
+          w.z = fmaf(-eta, c[2], w.z); w.w = fmaf(-eta, c[3], w.w);
+          *reinterpret_cast<float4*>(wr + d) = w;
+        } else {
+#pragma unroll
+          for (int b = 0; b < 4; ++b)
+            if (d + b < D) wr[d + b] = fmaf(-eta, c[b], wr[d + b]);
+        }
+      }
+    }
+}
+
+}  // namespace
+
+int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
+                       RowMap z, RowMap v) {
+  const long long big_tiles = (long long)((K + 127) / 128) * ((J + 127) / 128);
+  if (big_tiles >= 148) {
+    dim3 grid((J + 127) / 128, (K + 127) / 128);
+    forward_f32_kernel<2, 2><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, z, v);
+  } else {
+    dim3 grid((J + 63) / 64, (K + 63) / 64);
+    forward_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, z, v);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J, int D, float eta,
+                     const int* dev_status) {
+  const long long big_tiles = (long long)((J + 127) / 128) * ((D + 127) / 128);
+  if (big_tiles >= 148) {
+    dim3 grid((D + 127) / 128, (J + 127) / 128);
+    apply_f32_kernel<2, 2><<<grid, 256, 0, s>>>(W, u, v, K, J, D, eta, dev_status);
+  } else {
+    dim3 grid((D + 63) / 64, (J + 63) / 64);
+    apply_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, u, v, K, J, D, eta, dev_status);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+}  // namespace sfb

@@ -1,0 +1,250 @@
+// Sparse-code paths of the sparse-coding dictionary update (Section 2, "Sparse coding"; Figure 3):
+//
+//   forward:  u_i = W a_i - x_i = sum_{(d,a) in code i} a * W[:, d] - x_i     (a_i given as a CSR row)
+//   apply  :  W[:, d] -= eta * sum_{i : a_id != 0} a_id * u_i                 (only touched atoms move)
+//
+// W is J x D row-major, so an atom (column d) is strided in memory.  The forward therefore works on
+// an atom-major copy W^T (one coalesced J-vector per nonzero), rebuilt from W by a tiled transpose.
+// The apply gives every thread block a slab of 8 consecutive atoms (32-byte sectors of every row of
+// W) held in shared memory; the block walks all samples in order, finds each sample's nonzeros
+// inside its slab by binary search in the sorted CSR row, and applies them in (sample, atom) order.
+// No floating-point atomics: every element of W is owned by one block and updated in a fixed order,
+// so the result is bit-reproducible; atoms no code uses are written back unchanged.
+#include "common.cuh"
+
+namespace sfb {
+namespace {
+
+struct CsrRow {
+  const uint32_t* idx;
+  const float* val;
+  int len;
+};
+
+__device__ __forceinline__ CsrRow csr_row(const CsrView& c, int i) {
+  CsrRow r;
+  if (c.base == nullptr) {
+    const uint32_t s = c.rowptr[i], e = c.rowptr[i + 1];
+    r.idx = c.idx + s;
+    r.val = c.val + s;
+    r.len = (int)(e - s);
+  } else {
+    const int p = i / c.B, l = i % c.B;
+    const char* vb = c.base + c.streams_off + (long long)p * c.stream_stride + c.v_off;
+    const uint32_t* rp = reinterpret_cast<const uint32_t*>(vb);
+    const uint32_t s = rp[l], e = rp[l + 1];
+    r.idx = reinterpret_cast<const uint32_t*>(vb + c.rp_bytes) + s;
+    r.val = reinterpret_cast<const float*>(vb + c.rp_bytes + c.idx_bytes) + s;
+    r.len = (int)(e - s);
+  }
+  return r;
+}
+
+// Wt[d][j] = W[j][d]; Wt rows have ldt values (J rounded up to 4), pad columns zero.
+__global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict__ W, float* __restrict__ Wt, int J, int D,
+                                                        int ldt) {
+  __shared__ float tile[32][33];
+  const int d0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+#pragma unroll
+  for (int r = 0; r < 32; r += 8) {
+    const int j = j0 + ty + r, d = d0 + tx;
+    tile[ty + r][tx] = (j < J && d < D) ? W[(size_t)j * D + d] : 0.f;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 32; r += 8) {
+    const int d = d0 + ty + r, j = j0 + tx;
+    if (d < D && j < ldt) Wt[(size_t)d * ldt + j] = tile[tx][ty + r];
+  }
+}
+
+// grid = (K samples, ceil(ldt / 1024)); each thread owns 4 consecutive rows j of W.
+__global__ void __launch_bounds__(256) sc_forward_kernel(const float* __restrict__ Wt, int ldt, CsrView codes,
+                                                         const float* __restrict__ Xdata, RowMap u, int K, int J, int D,
+                                                         int* dev_status) {
+  __shared__ uint32_t s_idx[256];
+  __shared__ float s_val[256];
+  const int i = blockIdx.x;
+  const int j = (blockIdx.y * 256 + threadIdx.x) * 4;
+  const CsrRow row = csr_row(codes, i);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k0 = 0; k0 < row.len; k0 += 256) {
+    const int k = k0 + threadIdx.x;
+    uint32_t c = 0u;
+    float a = 0.f;
+    if (k < row.len) {
+      c = row.idx[k];
+      a = row.val[k];
+      const bool bad = (c >= (uint32_t)D) || (k > 0 && row.idx[k - 1] >= c);
+      if (bad) {
+        if (blockIdx.y == 0) atomicOr(dev_status, SFB_DEV_BAD_INDEX);
+        c = 0u;
+        a = 0.f;   // the offending entry is skipped
+      }
+    }
+    __syncthreads();
+    s_idx[threadIdx.x] = c;
+    s_val[threadIdx.x] = a;
+    __syncthreads();
+    const int n = min(256, row.len - k0);
+    if (j < ldt) {
+      for (int e = 0; e < n; ++e) {
+        const float4 w = *reinterpret_cast<const float4*>(Wt + (size_t)s_idx[e] * ldt + j);
+        const float av = s_val[e];
+        acc.x = fmaf(av, w.x, acc.x); acc.y = fmaf(av, w.y, acc.y);
+        acc.z = fmaf(av, w.z, acc.z); acc.w = fmaf(av, w.w, acc.w);
+      }
+    }
+  }
+  if (j < u.ld) {
+    const float* x = Xdata + (size_t)i * J;
+    float4 r;
+    r.x = (j < J) ? acc.x - x[j] : 0.f;
+    r.y = (j + 1 < J) ? acc.y - x[j + 1] : 0.f;
+    r.z = (j + 2 < J) ? acc.z - x[j + 2] : 0.f;
+    r.w = (j + 3 < J) ? acc.w - x[j + 3] : 0.f;
+    *reinterpret_cast<float4*>(u.row(i) + (size_t)j * 4) = r;
+  }
+}
+
+constexpr int SLAB_D = 8;        // atoms per block: one 32-byte sector of every row of W
+constexpr int SLAB_CHUNK = 256;  // samples searched per round (one per thread)
+
+// grid = (ceil(D / 8), ceil(J / JT)); dynamic shared memory: 8 * JT floats.
+__global__ void __launch_bounds__(256) sc_apply_kernel(float* __restrict__ W, CsrView codes, RowMap u, int K, int J,
+                                                       int D, int JT, float eta, const int* __restrict__ status_ro) {
+  extern __shared__ __align__(16) float Ws[];   // [SLAB_D][JT]
+  __shared__ int s_scan[256];
+  __shared__ int s_ent_i[SLAB_CHUNK * SLAB_D];
+  __shared__ int s_ent_d[SLAB_CHUNK * SLAB_D];
+  __shared__ float s_ent_a[SLAB_CHUNK * SLAB_D];
+  if (status_ro != nullptr && (*status_ro & SFB_DEV_BAD_HEADER)) return;
+  const int t = threadIdx.x;
+  const int d0 = blockIdx.x * SLAB_D, j0 = blockIdx.y * JT;
+  const int dn = min(SLAB_D, D - d0);
+  const int jn = min(JT, J - j0);
+  const bool vec_ok = ((D & 3) == 0) && (dn == SLAB_D);
+
+  for (int jj = t; jj < JT; jj += 256) {
+    float w[SLAB_D];
+#pragma unroll
+    for (int e = 0; e < SLAB_D; ++e) w[e] = 0.f;
+    if (jj < jn) {
+      const float* src = W + (size_t)(j0 + jj) * D + d0;
+      if (vec_ok) {
+        const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
+        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < SLAB_D; ++e)
+          if (e < dn) w[e] = src[e];
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < SLAB_D; ++e) Ws[e * JT + jj] = w[e];
+  }
+  __syncthreads();
+
+  for (int c0 = 0; c0 < K; c0 += SLAB_CHUNK) {
+    // (1) every thread searches one sample's sorted row for entries inside [d0, d0 + dn)
+    const int i = c0 + t;
+    int lo = 0, cnt = 0;
+    CsrRow row;
+    row.len = 0;
+    if (i < K) {
+      row = csr_row(codes, i);
+      int hi = row.len;
+      while (lo < hi) {   // lower bound of d0
+        const int mid = (lo + hi) >> 1;
+        if (row.idx[mid] < (uint32_t)d0) lo = mid + 1; else hi = mid;
+      }
+      while (lo + cnt < row.len && cnt < SLAB_D && row.idx[lo + cnt] < (uint32_t)(d0 + dn)) ++cnt;
+    }
+    // (2) block-wide exclusive scan of the counts (fixed order)
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if ((t & 31) >= o) incl += n;
+    }
+    if ((t & 31) == 31) s_scan[t >> 5] = incl;
+    __syncthreads();
+    if (t < 8) {
+      int v = s_scan[t];
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        const int n = __shfl_up_sync(0xffu, v, o);
+        if (t >= o) v += n;
+      }
+      s_scan[t] = v;
+    }
+    __syncthreads();
+    const int base = incl - cnt + ((t >> 5) > 0 ? s_scan[(t >> 5) - 1] : 0);
+    const int total = s_scan[7];
+    for (int e = 0; e < cnt; ++e) {
+      s_ent_i[base + e] = i;
+      s_ent_d[base + e] = (int)row.idx[lo + e] - d0;
+      s_ent_a[base + e] = row.val[lo + e];
+    }
+    __syncthreads();
+    // (3) apply the entries in (sample, atom) order; each thread owns fixed rows j of the slab
+    for (int e = 0; e < total; ++e) {
+      const float ca = -eta * s_ent_a[e];
+      const float* ur = reinterpret_cast<const float*>(u.row(s_ent_i[e])) + j0;
+      float* ws = Ws + s_ent_d[e] * JT;
+      for (int jj = t * 4; jj < jn; jj += 1024) {
+        if (jj + 3 < jn) {
+          const float4 uv = *reinterpret_cast<const float4*>(ur + jj);
+          float4 w = *reinterpret_cast<float4*>(ws + jj);
+          w.x = fmaf(ca, uv.x, w.x); w.y = fmaf(ca, uv.y, w.y); w.z = fmaf(ca, uv.z, w.z); w.w = fmaf(ca, uv.w, w.w);
+          *reinterpret_cast<float4*>(ws + jj) = w;
+        } else {
+          for (int b = 0; b < 4 && jj + b < jn; ++b) ws[jj + b] = fmaf(ca, ur[jj + b], ws[jj + b]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+
+  for (int jj = t; jj < jn; jj += 256) {
+    float* dst = W + (size_t)(j0 + jj) * D + d0;
+    if (vec_ok) {
+      *reinterpret_cast<float4*>(dst) = make_float4(Ws[jj], Ws[JT + jj], Ws[2 * JT + jj], Ws[3 * JT + jj]);
+      *reinterpret_cast<float4*>(dst + 4) = make_float4(Ws[4 * JT + jj], Ws[5 * JT + jj], Ws[6 * JT + jj], Ws[7 * JT + jj]);
+    } else {
+      for (int e = 0; e < dn; ++e) dst[e] = Ws[e * JT + jj];
+    }
+  }
+}
+
+}  // namespace
+
+// Workspace the forward needs: the atom-major copy, D rows of ldt = roundup(J, 4) floats.
+long long sc_forward_workspace_bytes(int J, int D) { return (long long)D * pad_to(J, 4) * 4; }
+
+int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView codes, const float* Xdata, RowMap u, int K,
+                         int J, int D, int* dev_status) {
+  const int ldt = (int)pad_to(J, 4);
+  dim3 tg((D + 31) / 32, (ldt + 31) / 32);
+  transpose_kernel<<<tg, 256, 0, s>>>(W, Wt, J, D, ldt);
+  dim3 grid(K, (ldt + 1023) / 1024);
+  sc_forward_kernel<<<grid, 256, 0, s>>>(Wt, ldt, codes, Xdata, u, K, J, D, dev_status);
+  return cudaGetLastError() == cudaSuccess ? 2 : SFB_ERR_CUDA;
+}
+
+int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
+                    const int* dev_status_ro, int* /*dev_status*/) {
+  const int JT = (int)pad_to(J < 4096 ? J : 4096, 4);
+  const size_t smem = (size_t)SLAB_D * JT * sizeof(float);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(sc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SLAB_D * 4096 * 4);
+    attr_done = true;
+  }
+  dim3 grid((D + SLAB_D - 1) / SLAB_D, (J + JT - 1) / JT);
+  sc_apply_kernel<<<grid, 256, smem, s>>>(W, codes, u, K, J, D, JT, eta, dev_status_ro);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+}  // namespace sfb

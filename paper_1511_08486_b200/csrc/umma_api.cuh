@@ -1,0 +1,23 @@
+// Tensor-core (tcgen05 / TMEM / TMA) side of the SF hot path: interface used by the C-ABI host code.
+#pragma once
+
+#include "common.cuh"
+
+namespace sfb {
+
+struct UmmaPlan;   // tensor maps and launch geometry for one descriptor
+
+// Builds the plan for a TF32 or BF16 descriptor.  z_ws: fp32 [K][ldz] product workspace;
+// w_shadow: bf16 copy of W (BF16 path) or nullptr.
+int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* w_shadow, UmmaPlan** out);
+void umma_plan_destroy(UmmaPlan* p);
+
+// z = W a on the tensor cores followed by the model epilogue; factors go through u / v row maps.
+int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
+                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status);
+
+// W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
+int umma_apply(UmmaPlan* p, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, const void* sf_buf, float eta, int K,
+               const int* dev_status);
+
+}  // namespace sfb

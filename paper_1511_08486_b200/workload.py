@@ -1,0 +1,83 @@
+"""Places one synthetic workload (see `sfbgen`) on the device and drives the C ABI with it.
+
+Only tensor allocation, host<->device copies and argument marshalling happen here.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def bf16_tensor(bits: np.ndarray, device) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> a torch.bfloat16 tensor holding exactly those bits."""
+    return torch.from_numpy(bits.view(np.int16).copy()).to(device).view(torch.bfloat16)
+
+
+class DeviceWorkload:
+    """Device copies of the inputs of configuration `cfg`, a context, and the SF buffer."""
+
+    def __init__(self, cfg: dict, inputs: dict, path: str | None = None, device="cuda:0", stream=None):
+        self.cfg, self.device = cfg, torch.device(device)
+        self.path = path or cfg["path"]
+        model = cfg["model"]
+        self.model = model
+        J, D, P, Bsz = cfg["J"], cfg["D"], cfg["P"], cfg["B"]
+        self.K = P * Bsz
+        self.pool = cfg["pool"]
+        sparse = model == "sc"
+        self.desc = B.make_desc(model, self.path, J, D, P, Bsz, v_sparse=int(sparse), margin=cfg.get("margin", 1.0),
+                                nnz_capacity=inputs.get("nnz_capacity", 0))
+        self.ctx = B.Context(self.desc, stream)
+        self.ldu, self.ldv = self.ctx.ldu, self.ctx.ldv
+        dev = self.device
+        self.W0 = torch.from_numpy(inputs["W"]).to(dev)
+        self.W = self.W0.clone()
+        bf16 = self.path == "bf16"
+        self.val_dtype = torch.bfloat16 if bf16 else torch.float32
+        self.batches = []
+        for b in range(self.pool):
+            t = {}
+            if model == "mlr":
+                t["X"] = bf16_tensor(inputs["X_bits"][b], dev) if bf16 else torch.from_numpy(inputs["X"][b]).to(dev)
+                t["labels"] = torch.from_numpy(inputs["labels"][b]).to(dev)
+                t["aux"] = B.make_aux(labels=t["labels"])
+            elif model == "dml":
+                t["X"] = torch.from_numpy(inputs["Xa"][b]).to(dev)
+                t["Xb"] = torch.from_numpy(inputs["Xb"][b]).to(dev)
+                t["similar"] = torch.from_numpy(inputs["similar"]).to(dev)
+                t["aux"] = B.make_aux(Xb=t["Xb"], similar=t["similar"])
+            else:
+                t["X"] = None
+                t["rowptr"] = torch.from_numpy(inputs["rowptr"][b].view(np.int32).copy()).to(dev)
+                t["idx"] = torch.from_numpy(inputs["idx"][b].view(np.int32).copy()).to(dev)
+                t["val"] = torch.from_numpy(inputs["val"][b]).to(dev)
+                t["Xdata"] = torch.from_numpy(inputs["Xdata"][b]).to(dev)
+                t["aux"] = B.make_aux(rowptr=t["rowptr"], idx=t["idx"], val=t["val"], Xdata=t["Xdata"])
+            self.batches.append(t)
+        self.sf_buf = torch.zeros(self.ctx.sf_buffer_bytes, dtype=torch.uint8, device=dev)
+        self.U = torch.zeros(self.K, self.ldu, dtype=self.val_dtype, device=dev)
+        self.V = None if sparse else torch.zeros(self.K, self.ldv, dtype=self.val_dtype, device=dev)
+
+    def reset(self):
+        self.W.copy_(self.W0)
+        self.ctx.invalidate()
+
+    def compute_factors(self, b: int = 0):
+        t = self.batches[b % self.pool]
+        self.ctx.compute_factors(self.W, t["X"], t["aux"], self.U, self.V)
+
+    def pack(self, b: int = 0, clock: int = 0):
+        t = self.batches[b % self.pool]
+        self.ctx.pack(self.U, self.V, t["aux"], self.sf_buf, clock)
+
+    def apply(self, eta: float, K: int | None = None):
+        self.ctx.apply(self.W, self.sf_buf, eta, K)
+
+    def step(self, t_idx: int, eta: float | None = None, K: int | None = None):
+        t = self.batches[t_idx % self.pool]
+        self.ctx.step(self.W, t["X"], t["aux"], self.sf_buf, self.cfg["eta"] if eta is None else eta, K, clock=t_idx)
+
+    def close(self):
+        self.ctx.destroy()

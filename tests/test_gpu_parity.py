@@ -1,0 +1,228 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same inputs.
+
+Tolerances (relative Frobenius error against the oracle): 1e-5 on the fp32 CUDA-core path,
+2e-3 on the TF32 path, 1e-2 on the bf16-in / fp32-accumulate path; SF buffer layout, indices and
+pure copies bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sfb_oracle as orc
+from sfbgen import get_config, make_inputs, scaled
+from tests.util import MODEL_ID, TOL, batch_of, dml_accept_gate, oracle_apply, oracle_factors, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def _workload(cfg, inputs, path):
+    from paper_1511_08486_b200.workload import DeviceWorkload
+    return DeviceWorkload(cfg, inputs, path=path)
+
+
+def _wire_dtype(path):
+    return orc.DTYPE_BF16 if path == "bf16" else orc.DTYPE_F32
+
+
+def _oracle_pack_of(cfg, path, U, V, batch, inputs, clock):
+    csr = (batch["rowptr"], batch["idx"], batch["val"]) if cfg["model"] == "sc" else None
+    return orc.pack(MODEL_ID[cfg["model"]], _wire_dtype(path), cfg["J"], cfg["D"], cfg["P"], cfg["B"], U, V, csr=csr,
+                    clock=clock, nnz_capacity=inputs.get("nnz_capacity", 0))
+
+
+def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, path)
+    tol = TOL[path]
+    J, D, K = cfg["J"], cfg["D"], cfg["K"]
+    eta = cfg["eta"] if eta is None else eta
+    W0 = inputs["W"]
+    batch = batch_of(inputs, cfg, 0)
+    try:
+        # ---- factors -----------------------------------------------------------------------------
+        U_or, V_or, extra = oracle_factors(cfg, W0, batch)
+        wl.compute_factors(0)
+        torch.cuda.synchronize()
+        U_gpu = to_f64(wl.U)[:, :J]
+        assert not to_f64(wl.U)[:, J:].any(), "pad columns of U must be zero"
+        U_ref = dml_accept_gate(cfg, U_gpu, U_or, extra, path) if cfg["model"] == "dml" else U_or
+        e_u = orc.rel_fro(U_gpu, U_ref)
+        assert e_u <= tol, f"E_U = {e_u:.3e} > {tol}"
+        if cfg["model"] != "sc":
+            V_gpu = to_f64(wl.V)
+            assert not V_gpu[:, D:].any(), "pad columns of V must be zero"
+            if check_v_exact:
+                assert np.array_equal(V_gpu[:, :D], V_or), "v is a pure copy (MLR) / one fp32 subtraction (DML)"
+        # ---- pack: the buffer is exactly the oracle's serialisation of the same (U, V) -----------
+        wl.pack(0, clock=5)
+        torch.cuda.synchronize()
+        buf = wl.sf_buf.cpu().numpy()
+        ref_buf = _oracle_pack_of(cfg, path, U_gpu, V_or, batch, inputs, 5)
+        assert buf.size == ref_buf.size
+        assert np.array_equal(buf, ref_buf), f"SF buffer differs at byte {np.nonzero(buf != ref_buf)[0][:4]}"
+        # ---- apply to zero: W = 0, eta = -1 gives U^T V ---------------------------------------------
+        wl.W.zero_()
+        wl.ctx.invalidate()
+        wl.apply(-1.0)
+        torch.cuda.synchronize()
+        dW_gpu = to_f64(wl.W)
+        if cfg["model"] == "sc":
+            dW_or = orc.apply_sparse(np.zeros((J, D)), U_gpu, batch["rowptr"], batch["idx"], batch["val"], -1.0)
+        else:
+            dW_or = orc.delta_w(U_gpu, V_or)
+        e_dw = orc.rel_fro(dW_gpu, dW_or)
+        assert e_dw <= tol, f"E_dW = {e_dw:.3e} > {tol}"
+        # partial apply: only the first worker's stream
+        if cfg["P"] > 1:
+            wl.W.zero_()
+            wl.ctx.invalidate()
+            wl.apply(-1.0, K=cfg["B"])
+            torch.cuda.synchronize()
+            Bn = cfg["B"]
+            if cfg["model"] == "sc":
+                rp = batch["rowptr"][:Bn + 1]
+                ref1 = orc.apply_sparse(np.zeros((J, D)), U_gpu[:Bn], rp, batch["idx"], batch["val"], -1.0)
+            else:
+                ref1 = orc.delta_w(U_gpu[:Bn], V_or[:Bn])
+            assert orc.rel_fro(to_f64(wl.W), ref1) <= tol
+        # ---- steps: W_T - W_0 against the oracle's trajectory ----------------------------------------
+        W_or = W0.astype(np.float64)
+        for t in range(steps):
+            bt = batch_of(inputs, cfg, t % cfg["pool"])
+            U_t, V_t, _ = oracle_factors(cfg, W_or, bt)
+            W_or = oracle_apply(cfg, W_or, U_t, V_t, bt, eta)
+        runs = []
+        for rep in range(2):
+            wl.reset()
+            for t in range(steps):
+                wl.step(t, eta=eta)
+            torch.cuda.synchronize()
+            runs.append((wl.W.cpu().numpy().copy(), wl.sf_buf.cpu().numpy().copy()))
+        assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1]), \
+            "two runs from the same state must be bit-identical"
+        W_gpu = runs[0][0].astype(np.float64)
+        moved = np.linalg.norm(W_or - W0)
+        e_step = np.linalg.norm((W_gpu - W0) - (W_or - W0)) / moved
+        # W is stored in fp32: its storage rounding (2^-24 per element, relative) is not the kernel's error
+        storage = steps * 2.0 ** -24 * np.linalg.norm(W0) / moved
+        assert e_step <= tol + storage, f"E_step = {e_step:.3e} > {tol} + {storage:.1e}"
+        # the buffer left by the last step is a valid serialisation with the step's clock
+        h, U_last, _ = orc.unpack(runs[0][1])
+        assert h["clock"] == steps - 1 and h["P"] == cfg["P"] and h["J"] == J
+        assert wl.ctx.status() == 0
+        return dict(e_u=e_u, e_dw=e_dw, e_step=e_step)
+    finally:
+        wl.close()
+
+
+# ------------------------------------------------------------------------------------- fp32 CUDA-core path
+def test_c0_mlr_tiny_f32():
+    cfg = get_config("C0")
+    check_config(cfg, "f32", eta=cfg["eta"], steps=1)
+    check_config(cfg, "f32", eta=20.0, steps=3)          # large step: the update dominates fp32 storage rounding
+
+
+@pytest.mark.parametrize("P,B", [(1, 32), (4, 8), (32, 1)])
+def test_c0_worker_split_invariance(P, B):
+    cfg = scaled("C0", P=P, B=B)
+    cfg["name"] = "C0"
+    check_config(cfg, "f32", eta=1.0, steps=1)
+
+
+def test_mlr_ragged_shapes_f32():
+    # J, D, K not multiples of any tile size; D not a multiple of 4 exercises the scalar edges
+    for J, D, P, B in ((37, 203, 3, 7), (130, 516, 2, 65), (257, 1000, 5, 13)):
+        check_config(scaled("C1", J=J, D=D, P=P, B=B, pool=2), "f32", eta=0.5, steps=2)
+
+
+def test_c1_mlr_large_scaled_f32():
+    check_config(scaled("C1", J=500, D=4000, P=8, B=32, pool=3), "f32", eta=1.0, steps=3)
+
+
+def test_c1_mlr_large_full_f32():
+    check_config(get_config("C1"), "f32", eta=1.0, steps=1)
+
+
+def test_c2_dml_scaled_f32():
+    check_config(scaled("C2", J=72, D=1001, P=3, B=20), "f32", eta=1e-4, steps=2)
+    check_config(scaled("C2", J=600, D=2000, P=8, B=32), "f32", eta=1e-4, steps=2)
+
+
+def test_c2_dml_full_f32():
+    check_config(get_config("C2"), "f32", eta=1e-5, steps=1)
+
+
+def test_c3_sc_scaled_f32():
+    check_config(scaled("C3", J=70, D=333, P=3, B=5, density=0.1), "f32", eta=1e-2, steps=2)
+    check_config(scaled("C3", J=512, D=2000, P=4, B=32), "f32", eta=1e-3, steps=2)
+
+
+def test_c3_sc_full_f32():
+    check_config(get_config("C3"), "f32", eta=1e-4, steps=1)
+
+
+def test_c3_unused_atoms_are_bit_identical():
+    cfg = scaled("C3", J=96, D=800, P=2, B=8, density=0.02)
+    inputs = make_inputs(cfg)
+    used = np.zeros(cfg["D"], bool)
+    used[inputs["idx"][0]] = True
+    assert (~used).any()
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.step(0, eta=0.1)
+        torch.cuda.synchronize()
+        W1 = wl.W.cpu().numpy()
+        assert np.array_equal(W1[:, ~used], inputs["W"][:, ~used])
+        assert not np.array_equal(W1[:, used], inputs["W"][:, used])
+    finally:
+        wl.close()
+
+
+# ------------------------------------------------------------------------------------- error behaviour
+def test_error_codes_and_device_status():
+    from paper_1511_08486_b200 import binding as B
+    cfg = get_config("C0")
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        with pytest.raises(B.SfbError) as e:
+            wl.apply(0.1, K=5)                               # not a whole number of worker streams
+        assert e.value.code == -1
+        with pytest.raises(B.SfbError):
+            wl.apply(0.1, K=cfg["K"] + cfg["B"])
+        # a label outside [0, J): status bit set, that sample's u written as zeros
+        wl.batches[0]["labels"][3] = 99
+        wl.compute_factors(0)
+        assert wl.ctx.status() == B.SFB_DEV_BAD_LABEL
+        U = to_f64(wl.U)
+        assert not U[3].any() and U[2].any()
+        assert wl.ctx.status() == 0                          # the word is cleared by the read
+        wl.batches[0]["labels"][3] = 1
+        # a buffer whose header does not match: apply leaves W untouched
+        wl.compute_factors(0)
+        wl.pack(0)
+        wl.sf_buf[20] = 11                                   # J field of the header
+        wl.apply(0.5)
+        assert wl.ctx.status() == B.SFB_DEV_BAD_HEADER
+        assert torch.equal(wl.W, wl.W0)
+    finally:
+        wl.close()
+    with pytest.raises(B.SfbError) as e:
+        B.Context(B.make_desc("sc", "f32", 8, 8, 2, 2, v_sparse=0))
+    assert e.value.code == -3
+    with pytest.raises(B.SfbError) as e:
+        B.Context(B.make_desc("mlr", "f32", 0, 8, 2, 2))
+    assert e.value.code == -2
+
+
+def test_sparse_bad_index_sets_status():
+    from paper_1511_08486_b200 import binding as B
+    cfg = scaled("C3", J=32, D=100, P=2, B=4, density=0.1)
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.batches[0]["idx"][0] = 1000
+        wl.compute_factors(0)
+        assert wl.ctx.status() & B.SFB_DEV_BAD_INDEX
+    finally:
+        wl.close()
