@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the SF hot path: `python bench.py --gpus N --steps K --warmup W [--impl reference]`.
+
+A step is one pass of the whole path (factor computation -> SF buffer -> rank-K apply, i.e. one
+`sfb_step`) over one synthetic minibatch of the named workload.  Prints ONE JSON line (rank 0).
+
+* `value`: SF-step samples/s with inputs resident in HBM, device-timed (CUDA events), max over ranks.
+* `e2e`: the same metric with the step's inputs copied from pinned host memory and a result read
+  back to the host inside the timed region, all through the C ABI.
+* `roofline`: the dominant kernel (the rank-K apply) against the measured peak for its bound.
+* `cpu_baseline`: the fp64 oracle, as it stands, on a bounded sample on the host cores.
+* `--impl reference`: times the oracle (the only reference implementation there is) instead.
+
+With N > 1 (torchrun) every rank runs an independent replica of the workload ("replicas only": the
+path has no exchange step on one node because the P workers are simulated inside one SF buffer).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "SF-step samples/s"
+UNIT = "samples/s"
+DATASHEET_BF16_TFLOPS = 2250.0
+FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 lanes x 2 flop x max SM clock
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self._stop, self._t = index, [], threading.Event(), None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                self.rows.append([c.strip() for c in out.strip().split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        self._t = threading.Thread(target=self._run, daemon=True)
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=6)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def algorithmic(cfg, path):
+    """Flops / bytes one apply launch must do (what the roofline fraction is computed from)."""
+    J, D, K = cfg["J"], cfg["D"], cfg["K"]
+    es = 2 if path == "bf16" else 4
+    if cfg["model"] == "sc":
+        return None
+    flops = 2.0 * J * D * K
+    bytes_ = 2.0 * J * D * 4 + K * (J + D) * es + (J * D * 2 if path == "bf16" else 0)
+    return dict(flops=flops, bytes=bytes_)
+
+
+def oracle_step_time(cfg, inputs, sample_workers: int):
+    """Seconds of one oracle step (factors + apply) on the first `sample_workers` workers' samples."""
+    from oracle import sfb_oracle as orc
+    from tests.util import MODEL_ID, batch_of
+    n = sample_workers * cfg["B"]
+    b = batch_of(inputs, cfg, 0)
+    if cfg["model"] == "sc":
+        rp = b["rowptr"][:n + 1]
+        b = dict(rowptr=rp, idx=b["idx"][:rp[-1]], val=b["val"][:rp[-1]], Xdata=b["Xdata"][:n])
+    else:
+        b = {k: (v[:n] if hasattr(v, "shape") and v.shape[0] == cfg["K"] else v) for k, v in b.items()}
+    t0 = time.perf_counter()
+    orc.step(MODEL_ID[cfg["model"]], inputs["W"], b, cfg["eta"], cfg.get("margin", 1.0))
+    return time.perf_counter() - t0, n
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def pick_sample_workers(cfg):
+    """Workers whose samples make up the oracle's bounded sample (~10-30 s of host work)."""
+    flops_per_worker = 4.0 * cfg["J"] * cfg["D"] * cfg["B"]           # forward + apply, fp64
+    budget = 1.5e12                                                    # ~15 s at ~100 GFLOP/s
+    return int(max(1, min(cfg["P"], budget // max(flops_per_worker, 1.0))))
+
+
+def run_reference(args, cfg, inputs):
+    """The oracle as the reference arm: each step is one oracle step on a bounded sample."""
+    sw = pick_sample_workers(cfg)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step_time(cfg, inputs, sw)
+    t, n = 0.0, 0
+    for _ in range(args.steps):
+        dt, n = oracle_step_time(cfg, inputs, sw)
+        t += dt
+    value = n * args.steps / t
+    cores = blas_threads()
+    sample = f"{sw} of {cfg['P']} workers' samples ({n} of {cfg['K']}) of minibatch 0 at full J x D, per step"
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, "f64-oracle")},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+
+
+def workload_name(cfg, path):
+    return (f"{cfg['name']} {cfg['model'].upper()} J={cfg['J']} D={cfg['D']} P={cfg['P']} B={cfg['B']} "
+            f"K={cfg['K']} path={path}")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C4")
+    ap.add_argument("--path", default=None, help="f32 | tf32 | bf16 (default: the configuration's own)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from sfbgen import get_config, make_inputs
+    cfg = get_config(args.config)
+    path = args.path or cfg["path"]
+
+    if args.impl == "reference":
+        if rank == 0:
+            inputs = make_inputs(cfg)
+            print(json.dumps(run_reference(args, cfg, inputs)), flush=True)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1511_08486_b200.build import build_library
+    from paper_1511_08486_b200.workload import DeviceWorkload
+
+    build_library()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    inputs = make_inputs(cfg)
+    wl = DeviceWorkload(cfg, inputs, path=path, device=dev)
+    K, eta = cfg["K"], cfg["eta"]
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # L2 flush buffer for workloads whose per-step footprint is below L2
+    step_bytes = 4.0 * cfg["J"] * cfg["D"] + wl.ctx.sf_buffer_bytes
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < (252 << 20) else None
+
+    def run_steps(n, t0=0):
+        for t in range(n):
+            if flush is not None:
+                flush.fill_(t & 1)
+            wl.step(t0 + t, eta=eta)
+
+    # ---- device-resident timing ----------------------------------------------------------------
+    wl.reset()
+    run_steps(max(args.warmup, 3))
+    barrier()
+    l0 = wl.ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        if flush is None:
+            ev0.record(stream)
+            run_steps(args.steps, t0=args.warmup)
+            ev1.record(stream)
+            barrier()
+            ms = ev0.elapsed_time(ev1)
+        else:   # time each step alone so the flush is outside the timed spans
+            ms = 0.0
+            for t in range(args.steps):
+                flush.fill_(t & 1)
+                ev0.record(stream)
+                wl.step(args.warmup + t, eta=eta)
+                ev1.record(stream)
+                torch.cuda.synchronize()
+                ms += ev0.elapsed_time(ev1)
+            barrier()
+    launches = wl.ctx.launch_count() - l0
+    status = wl.ctx.status()
+
+    # ---- per-stage timing (events recorded inside sfb_step, same workload) ------------------------
+    wl.ctx.profile(True)
+    nprof = min(args.steps, 128)
+    run_steps(nprof, t0=args.warmup)
+    f_ms, a_ms, n_rec = wl.ctx.stage_ms()
+    wl.ctx.profile(False)
+    f_ms, a_ms = f_ms / max(n_rec, 1), a_ms / max(n_rec, 1)
+
+    # ---- end to end: host buffers in, result out, inside the timed region ------------------------
+    host_batches = []
+    for t in wl.batches:
+        hb = {k: v.cpu().pin_memory() for k, v in t.items() if isinstance(v, torch.Tensor)}
+        host_batches.append(hb)
+    h2d = sum(v.numel() * v.element_size() for v in host_batches[0].values())
+    result_host = torch.empty(128, dtype=torch.uint8).pin_memory()
+    d2h = result_host.numel()
+
+    def e2e_step(t):
+        b = t % wl.pool
+        for k, hv in host_batches[b].items():
+            wl.batches[b][k].copy_(hv, non_blocking=True)
+        wl.step(t, eta=eta)
+        result_host.copy_(wl.sf_buf[:128], non_blocking=True)        # the committed header (clock, shapes)
+    for t in range(3):
+        e2e_step(t)
+    barrier()
+    ev0.record(stream)
+    for t in range(args.steps):
+        e2e_step(args.warmup + t)
+    ev1.record(stream)
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1)
+    clock_of_last = int(np.frombuffer(result_host.numpy().tobytes(), dtype=np.uint32)[7])
+
+    # ---- max over ranks ---------------------------------------------------------------------------
+    if world > 1:
+        tt = torch.tensor([ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(tt[0]), float(tt[1])
+
+    if rank == 0:
+        peaks = load_peaks()
+        alg = algorithmic(cfg, path)
+        value = world * K * args.steps / (ms * 1e-3)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": {"f32": "f32", "tf32": "tf32", "bf16": "bf16"}[path],
+            "data": "synthetic",
+            "config": {"workload": workload_name(cfg, path), "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                       "l2": "per-step footprint larger than L2" if flush is None else "L2 flushed between steps",
+                       "eta": eta, "pool": cfg["pool"]},
+            "e2e": {"value": world * K * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "last_clock_read_back": clock_of_last},
+            "gpu_launches": int(launches),
+            "device_status": status,
+            "stages_ms": {"factors": f_ms, "apply": a_ms, "steps_recorded": n_rec},
+            "clocks": clocks.summary(),
+        }
+        if alg is not None:
+            apply_tflops = alg["flops"] / (a_ms * 1e-3) / 1e12
+            fwd_tflops = alg["flops"] / (f_ms * 1e-3) / 1e12
+            if path == "f32":
+                out["roofline"] = {"bound": "alu", "achieved": apply_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
+                                   "frac": apply_tflops / FP32_FMA_TFLOPS, "traffic": None,
+                                   "kernel": "apply_f32_kernel", "peak_source": "148 SMs x 128 FMA lanes x 1.965 GHz"}
+            else:
+                scale = 1.0 if path == "bf16" else 0.5          # tf32 nominal rate is half of bf16
+                peak = peaks["bf16_sustained"] * scale
+                out["roofline"] = {"bound": "tensor", "achieved": apply_tflops, "peak": peak, "unit": "TFLOP/s",
+                                   "frac": apply_tflops / peak, "traffic": None, "kernel": "umma apply",
+                                   "peak_source": f"{peaks['source']} cuBLAS bf16 sustained" + ("" if path == "bf16" else " x 0.5 (tf32)"),
+                                   "frac_of_burst": apply_tflops / (peaks["bf16"] * scale),
+                                   "frac_of_datasheet": apply_tflops / (DATASHEET_BF16_TFLOPS * scale)}
+            out["apply_tflops"] = apply_tflops
+            out["forward_tflops"] = fwd_tflops
+        if not args.no_cpu_baseline:
+            sw = pick_sample_workers(cfg)
+            dt, n = oracle_step_time(cfg, inputs, sw)
+            out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                   "sample": f"one oracle step on {sw} of {cfg['P']} workers' samples ({n} of {K}) at full J x D, {dt:.1f} s"}
+        print(json.dumps(out), flush=True)
+    wl.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -147,6 +147,14 @@ int sfb_invalidate(sfb_ctx* ctx);
 /* Synchronises the stream, returns the sticky device status word in *device_status and clears it. */
 int sfb_status(sfb_ctx* ctx, int32_t* device_status);
 
+/* Measurement aid: while enabled, sfb_step records CUDA events on the context's stream before the
+ * factor stage, between the factor stage and the apply, and after the apply (at most the last 128
+ * steps are kept).  sfb_stage_ms synchronises the stream and returns the summed durations of the
+ * recorded steps and their count, then forgets them.  (No paper counterpart; Section 6.4 of the
+ * paper breaks iteration time down by stage in the same spirit.) */
+int sfb_profile(sfb_ctx* ctx, int enable);
+int sfb_stage_ms(sfb_ctx* ctx, float* factors_ms, float* apply_ms, int32_t* steps);
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t sfb_launch_count(const sfb_ctx* ctx);
 

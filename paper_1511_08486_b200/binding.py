@@ -22,6 +22,7 @@ PATHS = {"f32": SFB_PATH_F32, "tf32": SFB_PATH_TF32, "bf16": SFB_PATH_BF16}
 EXPORTS = (
     "sfb_create", "sfb_destroy", "sfb_sf_buffer_bytes", "sfb_ld", "sfb_compute_factors", "sfb_pack",
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
+    "sfb_profile", "sfb_stage_ms",
 )
 
 
@@ -77,6 +78,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_status.restype = C.c_int
     lib.sfb_launch_count.argtypes = [vp]
     lib.sfb_launch_count.restype = C.c_int64
+    lib.sfb_profile.argtypes = [vp, C.c_int]
+    lib.sfb_profile.restype = C.c_int
+    lib.sfb_stage_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.sfb_stage_ms.restype = C.c_int
     lib.sfb_strerror.argtypes = [C.c_int]
     lib.sfb_strerror.restype = C.c_char_p
     if path == LIB_PATH:
@@ -162,6 +167,14 @@ class Context:
         s = C.c_int32(0)
         self._chk(self._lib.sfb_status(self._h, C.byref(s)), "sfb_status")
         return s.value
+
+    def profile(self, enable: bool):
+        self._chk(self._lib.sfb_profile(self._h, int(enable)), "sfb_profile")
+
+    def stage_ms(self) -> tuple[float, float, int]:
+        f, a, n = C.c_float(0), C.c_float(0), C.c_int32(0)
+        self._chk(self._lib.sfb_stage_ms(self._h, C.byref(f), C.byref(a), C.byref(n)), "sfb_stage_ms")
+        return f.value, a.value, n.value
 
     def launch_count(self) -> int:
         return int(self._lib.sfb_launch_count(self._h))

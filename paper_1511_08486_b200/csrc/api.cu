@@ -22,6 +22,10 @@ struct sfb_ctx {
   const void* shadow_of;    // W pointer the shadow currently mirrors (nullptr = stale)
   UmmaPlan* umma;           // tensor-core plan (tensor maps), TF32 / BF16 paths
   int64_t launches;
+  bool profiling;
+  int prof_n;                       // steps recorded since the last read
+  cudaEvent_t prof_ev[128][3];      // start / after factors / after apply
+  bool prof_have_events;
 };
 
 namespace {
@@ -211,6 +215,9 @@ int sfb_destroy(sfb_ctx* c) {
   if (c == nullptr) return SFB_ERR_ARG;
   cudaStreamSynchronize(c->stream);
   if (c->umma) umma_plan_destroy(c->umma);
+  if (c->prof_have_events)
+    for (int i = 0; i < 128; ++i)
+      for (int e = 0; e < 3; ++e) cudaEventDestroy(c->prof_ev[i][e]);
   if (c->dev_status) cudaFree(c->dev_status);
   if (c->z_ws) cudaFree(c->z_ws);
   if (c->wt_ws) cudaFree(c->wt_ws);
@@ -226,6 +233,36 @@ int sfb_invalidate(sfb_ctx* c) {
 }
 
 int64_t sfb_launch_count(const sfb_ctx* c) { return c ? c->launches : 0; }
+
+int sfb_profile(sfb_ctx* c, int enable) {
+  if (c == nullptr) return SFB_ERR_ARG;
+  if (enable && !c->prof_have_events) {
+    for (int i = 0; i < 128; ++i)
+      for (int e = 0; e < 3; ++e)
+        if (cudaEventCreate(&c->prof_ev[i][e]) != cudaSuccess) return SFB_ERR_CUDA;
+    c->prof_have_events = true;
+  }
+  c->profiling = enable != 0;
+  c->prof_n = 0;
+  return SFB_OK;
+}
+
+int sfb_stage_ms(sfb_ctx* c, float* factors_ms, float* apply_ms, int32_t* steps) {
+  if (c == nullptr || factors_ms == nullptr || apply_ms == nullptr || steps == nullptr) return SFB_ERR_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  const int n = c->prof_n < 128 ? c->prof_n : 128;
+  float f = 0.f, a = 0.f;
+  for (int i = 0; i < n; ++i) {
+    float t0 = 0.f, t1 = 0.f;
+    if (cudaEventElapsedTime(&t0, c->prof_ev[i][0], c->prof_ev[i][1]) != cudaSuccess) return SFB_ERR_CUDA;
+    if (cudaEventElapsedTime(&t1, c->prof_ev[i][1], c->prof_ev[i][2]) != cudaSuccess) return SFB_ERR_CUDA;
+    f += t0;
+    a += t1;
+  }
+  *factors_ms = f; *apply_ms = a; *steps = n;
+  c->prof_n = 0;
+  return SFB_OK;
+}
 
 int sfb_status(sfb_ctx* c, int32_t* device_status) {
   if (c == nullptr || device_status == nullptr) return SFB_ERR_ARG;
@@ -304,6 +341,8 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   if (d.model != SFB_SC && (X == nullptr || !aligned(X, 16))) return SFB_ERR_ARG;
   CsrView codes;
   memset(&codes, 0, sizeof(codes));
+  const int slot = c->prof_n % 128;
+  if (c->profiling) cudaEventRecord(c->prof_ev[slot][0], c->stream);
   if (d.v_sparse) {
     ACC(launch_pack_csr(c->stream, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
                         c->dev_status));
@@ -312,7 +351,13 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes);
   if (r < 0) return r;
   ACC(launch_write_header(c->stream, sf_buf, d, c->l, clock, d.v_sparse ? aux->rowptr : nullptr));
-  return apply_from(c, W, sf_buf, eta, K, false);
+  if (c->profiling) cudaEventRecord(c->prof_ev[slot][1], c->stream);
+  r = apply_from(c, W, sf_buf, eta, K, false);
+  if (c->profiling) {
+    cudaEventRecord(c->prof_ev[slot][2], c->stream);
+    c->prof_n++;
+  }
+  return r;
 }
 
 }  // extern "C"
