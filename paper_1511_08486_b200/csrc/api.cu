@@ -190,7 +190,7 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
   bool ok = cudaMalloc(&c->dev_status, 256) == cudaSuccess;
   if (ok) ok = cudaMemsetAsync(c->dev_status, 0, 256, c->stream) == cudaSuccess;
   if (ok && desc->model == SFB_SC) ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
-  if (ok && desc->path != SFB_PATH_F32) {
+  if (ok && desc->path == SFB_PATH_BF16) {
     c->ldz = (int)pad_to(desc->J, 4);
     ok = cudaMalloc(&c->z_ws, (size_t)c->K * c->ldz * 4) == cudaSuccess;
   }

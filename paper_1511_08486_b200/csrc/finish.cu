@@ -199,6 +199,28 @@ __global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, 
   }
 }
 
+// v rows = Xa - Xb (one fp32 subtraction per element), pad columns zero; 4 values per thread.
+__global__ void __launch_bounds__(256) diff_rows_kernel(const float* __restrict__ Xa, const float* __restrict__ Xb, RowMap v,
+                                                        int K, int D) {
+  const int units = v.ld >> 2;
+  const long long total = (long long)K * units;
+  for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
+       g += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(g / units), c = (int)(g % units) * 4;
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c + 3 < D && (D & 3) == 0) {
+      const float4 a = *reinterpret_cast<const float4*>(Xa + (size_t)i * D + c);
+      const float4 b = *reinterpret_cast<const float4*>(Xb + (size_t)i * D + c);
+      r = make_float4(__fsub_rn(a.x, b.x), __fsub_rn(a.y, b.y), __fsub_rn(a.z, b.z), __fsub_rn(a.w, b.w));
+    } else {
+      float* e = reinterpret_cast<float*>(&r);
+      for (int q = 0; q < 4; ++q)
+        if (c + q < D) e[q] = __fsub_rn(Xa[(size_t)i * D + c + q], Xb[(size_t)i * D + c + q]);
+    }
+    *reinterpret_cast<float4*>(v.row(i) + (size_t)c * 4) = r;
+  }
+}
+
 __global__ void __launch_bounds__(256) cast_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wb,
                                                         long long n4) {
   for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n4; g += (long long)gridDim.x * blockDim.x) {
@@ -247,6 +269,13 @@ int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols) {
   if (total == 0) return 0;
   const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
   copy_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, K, cols);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D) {
+  const long long total = (long long)K * (v.ld >> 2);
+  const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
+  diff_rows_kernel<<<blocks, 256, 0, s>>>(Xa, Xb, v, K, D);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

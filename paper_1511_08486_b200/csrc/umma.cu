@@ -1,8 +1,451 @@
+// Tensor-core contractions of the SF hot path on sm_100a: tcgen05.mma with accumulators in tensor
+// memory (TMEM), operands brought to shared memory by TMA, one persistent CTA per SM.
+//
+//   forward:  Z[i][j] = sum_d A[i][d] * W[j][d]        (z_i = W a_i; Section 2, problem (P))
+//             both operands are contiguous along the reduction index d ("K-major").
+//   apply  :  W[j][d] -= eta * sum_i U[i][j] * V[i][d]   (W <- W - eta * sum_i u_i v_i^T; Section 3)
+//             the factors are stored one u_i / v_i per row, so both operands are contiguous along
+//             the output index ("MN-major"); tcgen05 reads them in that form directly from the SF
+//             buffer's worker streams, no transposed copy is made.
+//
+// Warp roles (192 threads): warp 0 issues TMA loads into a 4-stage shared-memory ring, warp 1 issues
+// the MMAs (one thread) into one of two TMEM accumulators, warps 2-5 drain the other accumulator
+// (tcgen05.ld) and run the epilogue, so the write-back of tile t overlaps the MMAs of tile t+1.
+// Every wait on an mbarrier is bounded; a wait that runs out sets SFB_DEV_TIMEOUT and the CTA leaves
+// through the common exit (TMEM freed) instead of hanging.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <cstring>
+
+#include "umma.cuh"
 #include "umma_api.cuh"
+
 namespace sfb {
-struct UmmaPlan { int dummy; };
-int umma_plan_create(const sfb_desc&, const Layout&, float*, int, __nv_bfloat16*, UmmaPlan**) { return SFB_ERR_UNSUPPORTED; }
-void umma_plan_destroy(UmmaPlan*) {}
-int umma_forward(UmmaPlan*, cudaStream_t, const void*, const __nv_bfloat16*, const void*, const sfb_aux*, RowMap, RowMap, RowMap, int*) { return SFB_ERR_UNSUPPORTED; }
-int umma_apply(UmmaPlan*, cudaStream_t, void*, __nv_bfloat16*, const void*, float, int, const int*) { return SFB_ERR_UNSUPPORTED; }
+
+// extra passes implemented in finish.cu
+int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D);
+
+namespace {
+
+constexpr int BM = 128;          // tile rows  = TMEM lanes
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * 128;   // 128 rows (K-major) or 128 output indices (MN-major) x 128 B... per 64/32 reduction steps
+constexpr int NUM_THREADS = 192;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+struct GemmParams {
+  int m_tiles, n_tiles, k_blocks;
+  int B, P;                 // rows per worker / workers, geometry of the 3-D operand maps
+  int m_bb, m_wp, m_tpw;    // forward: A rows per tile come as a box of m_bb rows x m_wp workers; tiles per worker
+  int k_bb, k_wp, k_bpw;    // apply: a reduction block is k_bb rows x k_wp workers; blocks per worker
+  int Mvalid, Nvalid;       // forward: (unused, N = J) ; apply: (J, D)
+  float* W;                 // apply: fp32 master, row stride ldw
+  __nv_bfloat16* shadow;    // apply: bf16 copy of the new W (or nullptr)
+  long long ldw;
+  float eta;
+  RowMap z;                 // forward: fp32 output rows
+  const int* status_ro;
+  int* status;
+};
+
+struct SharedCtl {
+  uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  volatile int abort;
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int* status) {
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && ctl->abort) return false;
+  }
+  ctl->abort = 1;
+  if (status != nullptr) atomicOr(status, SFB_DEV_TIMEOUT);
+  return false;
 }
+
+// ES: bytes per operand value (2 = bf16, 4 = tf32).  APPLY: MN-major operands and the W write-back
+// epilogue; otherwise K-major operands and the plain fp32 store of Z.  BN: tile columns.
+template <int ES, bool APPLY, int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+  constexpr int CH = 128 / ES;                 // values per 128-byte chunk
+  constexpr int BK = CH;                       // reduction steps per pipeline stage (64 bf16 / 32 tf32)
+  constexpr int UMMA_K = 32 / ES;              // reduction steps per instruction (16 bf16 / 8 tf32)
+  constexpr int B_STAGE_BYTES = BN * 128;
+  constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  constexpr uint32_t IDESC = ptx::instr_desc(ES == 2 ? 1u : 2u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM, BN);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles + STAGES * STAGE_BYTES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (p.status_ro != nullptr && (*p.status_ro & SFB_DEV_BAD_HEADER)) return;   // uniform over the grid
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(&ctl->full[s], 1);
+      ptx::mbar_init(&ctl->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(&ctl->tmem_full[b], 1);
+      ptx::mbar_init(&ctl->tmem_empty[b], 128);
+    }
+    ctl->abort = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmA);
+    ptx::prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&ctl->tmem_base, 2 * BN);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const int total_tiles = p.m_tiles * p.n_tiles;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    int s = 0;
+    uint32_t ph = 0;
+    int issued = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+      for (int kb = 0; kb < p.k_blocks; ++kb) {
+        ok = wait_or_abort(&ctl->empty[s], ph ^ 1u, ctl, p.status);
+        if (!ok) break;
+        if (lane == 0) {
+          uint8_t* a_dst = tiles + s * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_STAGE_BYTES;
+          ptx::mbar_expect_tx(&ctl->full[s], STAGE_BYTES);
+          if (!APPLY) {
+            const int k0 = kb * BK;
+            int slot0, p0;
+            if (p.B >= BM) { p0 = mt / p.m_tpw; slot0 = (mt % p.m_tpw) * BM; }
+            else { p0 = mt * p.m_wp; slot0 = 0; }
+            ptx::tma_load_3d(a_dst, &tmA, &ctl->full[s], k0, slot0, p0);
+            ptx::tma_load_3d(b_dst, &tmB, &ctl->full[s], k0, nt * BN, 0);
+          } else {
+            int row0, p0;
+            if (p.B >= BK) { p0 = kb / p.k_bpw; row0 = (kb % p.k_bpw) * BK; }
+            else { p0 = kb * p.k_wp; row0 = 0; }
+#pragma unroll
+            for (int c = 0; c < BM / CH; ++c)
+              ptx::tma_load_3d(a_dst + c * (BK * 128), &tmA, &ctl->full[s], mt * BM + c * CH, row0, p0);
+#pragma unroll
+            for (int c = 0; c < BN / CH; ++c)
+              ptx::tma_load_3d(b_dst + c * (BK * 128), &tmB, &ctl->full[s], nt * BN + c * CH, row0, p0);
+          }
+        }
+        __syncwarp();
+        ++issued;
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+      }
+    }
+    if (!ok || ctl->abort) {
+      // let copies already in flight land before the CTA goes away (bounded)
+      int n = issued < STAGES ? issued : STAGES;
+      for (int q = 0; q < n; ++q) {
+        int sq = s - 1 - q;
+        uint32_t pq = ph;
+        if (sq < 0) { sq += STAGES; pq ^= 1u; }
+        ptx::mbar_wait(&ctl->full[sq], pq, 1u << 16);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    int s = 0;
+    uint32_t ph = 0;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const int buf = it & 1;
+      const uint32_t acc_ph = (it >> 1) & 1u;
+      ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * BN;
+      for (int kb = 0; kb < p.k_blocks; ++kb) {
+        ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        if (lane == 0) {
+          const uint32_t a_addr = ptx::smem_u32(tiles + s * STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_STAGE_BYTES;
+          // K-major: 8-row groups 1024 B apart.  MN-major: 8-step groups 1024 B apart, chunks BK*128 B apart.
+          // MN-major fp32 (tf32) operands use the 32-byte-atom swizzle: groups of 4 steps, 512 B apart.
+          constexpr bool MN32 = APPLY && ES == 4;
+          const uint64_t a_desc = ptx::smem_desc(a_addr, APPLY ? BK * 128 : 16, MN32 ? 512 : 1024, MN32 ? 1 : 2);
+          const uint64_t b_desc = ptx::smem_desc(b_addr, APPLY ? BK * 128 : 16, MN32 ? 512 : 1024, MN32 ? 1 : 2);
+          // per instruction: K-major advances 32 B inside the swizzled row, MN-major UMMA_K rows of 128 B
+          constexpr uint32_t STEP = (APPLY ? UMMA_K * 128 : 32) >> 4;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+            if (ES == 2) ptx::mma_f16(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+            else ptx::mma_tf32(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+          }
+          ptx::mma_commit(&ctl->empty[s]);                     // stage reusable once these MMAs have read it
+          if (kb == p.k_blocks - 1) ptx::mma_commit(&ctl->tmem_full[buf]);   // accumulator complete
+        }
+        __syncwarp();
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 belong to this warp
+    const int r = quarter * 32 + lane;            // row of the tile this thread owns
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+      const int buf = it & 1;
+      const uint32_t acc_ph = (it >> 1) & 1u;
+      ok = wait_or_abort(&ctl->tmem_full[buf], acc_ph, ctl, p.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
+      float* row_ptr = nullptr;         // fp32 destination row of this thread (nullptr: nothing to store)
+      __nv_bfloat16* sh_ptr = nullptr;
+      int ncols;                        // valid columns of the row, counted from column 0 of the matrix
+      if (APPLY) {
+        const int j = mt * BM + r;
+        ncols = p.Nvalid;
+        if (j < p.Mvalid) {
+          row_ptr = p.W + (long long)j * p.ldw;
+          if (p.shadow != nullptr) sh_ptr = p.shadow + (long long)j * p.ldw;
+        }
+      } else {
+        int wp_, slot;
+        if (p.B >= BM) { wp_ = mt / p.m_tpw; slot = (mt % p.m_tpw) * BM + r; }
+        else { wp_ = mt * p.m_wp + r / p.m_bb; slot = r % p.m_bb; }
+        ncols = p.z.ld;
+        if (wp_ < p.P && slot < p.B) row_ptr = reinterpret_cast<float*>(p.z.row(wp_ * p.B + slot));
+      }
+#pragma unroll 1
+      for (int cc = 0; cc < BN / 32; ++cc) {
+        uint32_t v[32];
+        ptx::tmem_ld32(taddr + cc * 32, v);
+        ptx::tmem_ld_wait();
+        if (row_ptr != nullptr) {
+          const int c0 = nt * BN + cc * 32;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int c = c0 + q * 4;
+            if (c < ncols) {   // ncols is a multiple of 4 on these paths
+              float4 a = make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]),
+                                     __uint_as_float(v[q * 4 + 2]), __uint_as_float(v[q * 4 + 3]));
+              if (APPLY) {
+                float4 w = *reinterpret_cast<const float4*>(row_ptr + c);
+                w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
+                w.z = fmaf(-p.eta, a.z, w.z); w.w = fmaf(-p.eta, a.w, w.w);
+                *reinterpret_cast<float4*>(row_ptr + c) = w;
+                if (sh_ptr != nullptr) {
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+                  uint2 pk;
+                  pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                  pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                  *reinterpret_cast<uint2*>(sh_ptr + c) = pk;
+                }
+              } else {
+                *reinterpret_cast<float4*>(row_ptr + c) = a;
+              }
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&ctl->tmem_empty[buf]);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+// ------------------------------------------------------------------------------------------- host side
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (fn == nullptr) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+  }
+  return fn;
+}
+
+// 3-D map over factor-like rows: dim0 = cols values (contiguous), dim1 = rows per worker, dim2 = workers.
+bool encode_rows_map(CUtensorMap* m, int es, const void* base, long long cols, long long rows, long long workers,
+                     long long row_stride_bytes, long long worker_stride_bytes, int box0, int box1, int box2,
+                     bool atom32 = false) {
+  auto fn = get_encode();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)workers};
+  cuuint64_t strides[2] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)worker_stride_bytes};
+  cuuint32_t box[3] = {(cuuint32_t)box0, (cuuint32_t)box1, (cuuint32_t)box2};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const CUtensorMapDataType dt = es == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  const CUresult r = fn(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int pow2_at_least(int n) {
+  int p = 1;
+  while (p < n) p <<= 1;
+  return p;
+}
+
+template <int ES, bool APPLY, int BN>
+int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, int num_sms) {
+  constexpr int smem = STAGES * (A_STAGE_BYTES + BN * 128) + 1024 + (int)sizeof(SharedCtl);
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(umma_gemm_kernel<ES, APPLY, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess)
+      return SFB_ERR_CUDA;
+    attr_done = true;
+  }
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int grid = tiles < num_sms ? tiles : num_sms;
+  umma_gemm_kernel<ES, APPLY, BN><<<grid, NUM_THREADS, smem, s>>>(a, b, p);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+template <bool APPLY>
+int dispatch_gemm(cudaStream_t s, int es, int bn, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p,
+                  int num_sms) {
+  if (es == 2) return bn == 256 ? launch_gemm<2, APPLY, 256>(s, a, b, p, num_sms) : launch_gemm<2, APPLY, 128>(s, a, b, p, num_sms);
+  return bn == 256 ? launch_gemm<4, APPLY, 256>(s, a, b, p, num_sms) : launch_gemm<4, APPLY, 128>(s, a, b, p, num_sms);
+}
+
+}  // namespace
+
+struct UmmaPlan {
+  sfb_desc d;
+  Layout l;
+  float* z_ws;
+  int ldz;
+  int num_sms;
+  int es;
+};
+
+int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
+                     UmmaPlan** out) {
+  if (get_encode() == nullptr) return SFB_ERR_CUDA;
+  if (d.model == SFB_SC) return SFB_ERR_UNSUPPORTED;
+  UmmaPlan* p = new UmmaPlan();
+  p->d = d; p->l = l; p->z_ws = z_ws; p->ldz = ldz;
+  p->es = (d.path == SFB_PATH_BF16) ? 2 : 4;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev);
+  *out = p;
+  return SFB_OK;
+}
+
+void umma_plan_destroy(UmmaPlan* p) { delete p; }
+
+// Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
+static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status) {
+  const sfb_desc& d = pl->d;
+  const int es = pl->es, CH = 128 / es;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.B = d.B; p.P = d.P;
+  if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; p.m_tiles = d.P * p.m_tpw; }
+  else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; p.m_tiles = (d.P + p.m_wp - 1) / p.m_wp; }
+  const int bn = (d.J > 128 && (long long)p.m_tiles * ((d.J + 255) / 256) >= pl->num_sms) ? 256 : 128;
+  p.n_tiles = (d.J + bn - 1) / bn;
+  p.k_blocks = (d.D + CH - 1) / CH;
+  p.z = z;
+  p.status = dev_status;
+  CUtensorMap ta, tb;
+  if (!encode_rows_map(&ta, es, a.base, d.D, d.B, d.P, (long long)a.ld * es, a.worker_stride, CH, p.m_bb, p.m_wp))
+    return SFB_ERR_CUDA;
+  if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, CH, bn, 1))
+    return SFB_ERR_CUDA;
+  return dispatch_gemm<false>(s, es, bn, ta, tb, p, pl->num_sms);
+}
+
+int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
+                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status) {
+  const sfb_desc& d = pl->d;
+  const int K = d.P * d.B;
+  int launches = 0, r;
+  RowMap x_rows;
+  x_rows.base = const_cast<char*>(reinterpret_cast<const char*>(X));
+  x_rows.ld = d.D; x_rows.B = d.B; x_rows.es = pl->es;
+  x_rows.worker_stride = (long long)d.B * d.D * pl->es;
+  if (d.model == SFB_MLR) {
+    const bool bf16 = d.path == SFB_PATH_BF16;
+    RowMap zz = bf16 ? z : u;   // fp32 products: workspace when u is bf16, else u itself (finished in place)
+    if ((r = forward_gemm(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, zz, dev_status)) < 0) return r;
+    launches += r;
+    if ((r = launch_finish_mlr(s, zz, u, aux->labels, K, d.J, dev_status)) < 0) return r;
+    launches += r;
+    if (v.base != nullptr) {
+      if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
+      launches += r;
+    }
+    return launches;
+  }
+  // DML (TF32): the pair differences are the factor v and the GEMM operand
+  if (v.base == nullptr) return SFB_ERR_ARG;
+  if ((r = launch_diff_rows(s, reinterpret_cast<const float*>(X), reinterpret_cast<const float*>(aux->Xb), v, K, d.D)) < 0)
+    return r;
+  launches += r;
+  if ((r = forward_gemm(pl, s, W, v, u, dev_status)) < 0) return r;
+  launches += r;
+  if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
+  return launches + r;
+}
+
+int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, const void* sf_buf, float eta, int K,
+               const int* dev_status) {
+  const sfb_desc& d = pl->d;
+  const Layout& l = pl->l;
+  const int es = pl->es, CH = 128 / es, BK = CH;
+  const int workers = K / d.B;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.B = d.B; p.P = workers;
+  if (d.B >= BK) { p.k_bb = BK; p.k_wp = 1; p.k_bpw = (d.B + BK - 1) / BK; p.k_blocks = workers * p.k_bpw; }
+  else { p.k_bb = pow2_at_least(d.B); p.k_wp = BK / p.k_bb; p.k_bpw = 1; p.k_blocks = (workers + p.k_wp - 1) / p.k_wp; }
+  p.m_tiles = (d.J + BM - 1) / BM;
+  const int bn = ((long long)p.m_tiles * ((d.D + 255) / 256) >= pl->num_sms) ? 256 : 128;
+  p.n_tiles = (d.D + bn - 1) / bn;
+  p.Mvalid = d.J; p.Nvalid = d.D;
+  p.W = reinterpret_cast<float*>(W);
+  p.shadow = (d.path == SFB_PATH_BF16) ? w_shadow : nullptr;
+  p.ldw = d.D;
+  p.eta = eta;
+  p.status_ro = dev_status;
+  p.status = const_cast<int*>(dev_status);
+  const char* base = reinterpret_cast<const char*>(sf_buf) + l.streams_off;
+  CUtensorMap tu, tv;
+  // only the first `workers` streams are visible to the maps, so zero fill covers a ragged last block
+  if (!encode_rows_map(&tu, es, base, d.J, d.B, workers, (long long)l.ldu * es, l.stream_stride, CH, p.k_bb, p.k_wp,
+                       es == 4))
+    return SFB_ERR_CUDA;
+  if (!encode_rows_map(&tv, es, base + l.u_bytes, d.D, d.B, workers, (long long)l.ldv * es, l.stream_stride, CH, p.k_bb,
+                       p.k_wp, es == 4))
+    return SFB_ERR_CUDA;
+  return dispatch_gemm<true>(s, es, bn, tu, tv, p, pl->num_sms);
+}
+
+}  // namespace sfb

@@ -1,0 +1,67 @@
+"""GPU parity of the tensor-core (tcgen05 / TMEM / TMA) paths against the fp64 oracle.
+
+bf16-in / fp32-accumulate: relative Frobenius error <= 1e-2; TF32: <= 2e-3.  Sizes start at a single
+MMA tile and single pipeline stage (so a wrong descriptor or swizzle shows up in isolation), then
+span several tiles, ragged edges handled by TMA zero fill, worker streams shorter than one
+reduction block, and finally the full workload shapes.
+"""
+import numpy as np
+import pytest
+import torch
+
+from sfbgen import get_config, scaled
+from tests.test_gpu_parity import check_config
+
+pytestmark = pytest.mark.gpu
+
+
+def _cfg(name, path, **kw):
+    cfg = scaled(name, **kw)
+    cfg["path"] = path
+    return cfg
+
+
+# ------------------------------------------------------------------------------------------------ bf16
+def test_bf16_single_tile_single_stage():
+    # one 128 x 128 output tile, one 64-deep reduction block in the apply
+    check_config(_cfg("C4", "bf16", J=128, D=128, P=1, B=64, pool=1, labels="uniform"), "bf16", eta=0.5, steps=1)
+
+
+def test_bf16_multi_stage_multi_tile():
+    check_config(_cfg("C4", "bf16", J=256, D=512, P=2, B=128, pool=1, labels="uniform"), "bf16", eta=0.5, steps=2)
+    check_config(_cfg("C4", "bf16", J=640, D=1024, P=4, B=64, pool=2, labels="uniform"), "bf16", eta=0.5, steps=2)
+
+
+def test_bf16_ragged_and_short_streams():
+    # J, D not multiples of the tile; B below one reduction block (several workers share a block);
+    # B not a power of two (zero-filled slots); worker count not a multiple of the block's workers
+    for J, D, P, B in ((100, 200, 3, 10), (300, 264, 5, 8), (130, 72, 7, 3), (1000, 520, 2, 100), (77, 1032, 3, 130)):
+        check_config(_cfg("C4", "bf16", J=J, D=D, P=P, B=B, pool=1, labels="uniform"), "bf16", eta=0.5, steps=2)
+
+
+def test_bf16_c4_reduced():
+    check_config(_cfg("C4", "bf16", J=4096, D=8192, P=16, B=32, pool=2), "bf16", eta=1e-2, steps=3)
+
+
+def test_bf16_c4_full():
+    check_config(get_config("C4"), "bf16", eta=1e-3, steps=1)
+
+
+# ------------------------------------------------------------------------------------------------ tf32
+def test_tf32_single_tile_single_stage():
+    check_config(_cfg("C1", "tf32", J=128, D=128, P=1, B=32, pool=1), "tf32", eta=0.5, steps=1)
+
+
+def test_tf32_c0_and_ragged():
+    check_config(_cfg("C0", "tf32"), "tf32", eta=1.0, steps=1)
+    for J, D, P, B in ((100, 200, 3, 10), (300, 260, 5, 8), (257, 1000, 2, 100)):
+        check_config(_cfg("C1", "tf32", J=J, D=D, P=P, B=B, pool=1), "tf32", eta=0.5, steps=2)
+
+
+def test_tf32_c1_full():
+    check_config(_cfg("C1", "tf32"), "tf32", eta=1.0, steps=2)
+
+
+def test_tf32_dml():
+    check_config(_cfg("C2", "tf32", J=72, D=1000, P=3, B=20), "tf32", eta=1e-4, steps=2)
+    check_config(_cfg("C2", "tf32"), "tf32", eta=1e-5, steps=1)
