@@ -55,7 +55,33 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index, self.rows, self._stop, self._t = index, [], threading.Event(), None
 
+    def _run_nvml(self) -> bool:
+        """Fast sampling through NVML (read-only queries); returns False if NVML is unavailable."""
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            mx = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            bits = [(nv.nvmlClocksEventReasonHwSlowdown, "hw_slowdown"),
+                    (nv.nvmlClocksEventReasonHwThermalSlowdown, "hw_thermal_slowdown"),
+                    (nv.nvmlClocksEventReasonSwThermalSlowdown, "sw_thermal_slowdown"),
+                    (nv.nvmlClocksEventReasonSwPowerCap, "sw_power_cap")]
+        except Exception:
+            return False
+        while not self._stop.is_set():
+            try:
+                sm = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+                pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                rs = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                self.rows.append([str(sm), str(mx), str(pw)] + ["Active" if rs & b else "Not Active" for b, _ in bits])
+            except Exception:
+                pass
+            self._stop.wait(0.005)
+        return True
+
     def _run(self):
+        if self._run_nvml():
+            return
         while not self._stop.is_set():
             try:
                 out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
@@ -171,6 +197,8 @@ def main():
     ap.add_argument("--config", default="C4")
     ap.add_argument("--path", default=None, help="f32 | tf32 | bf16 (default: the configuration's own)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    for dim in ("J", "D", "P", "B"):
+        ap.add_argument(f"--{dim}", type=int, default=None, help=f"override {dim} (smaller cases for profiler captures)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -179,6 +207,10 @@ def main():
 
     from sfbgen import get_config, make_inputs
     cfg = get_config(args.config)
+    over = {k: getattr(args, k) for k in ("J", "D", "P", "B") if getattr(args, k) is not None}
+    if over:
+        from sfbgen import scaled
+        cfg = scaled(args.config, **over)
     path = args.path or cfg["path"]
 
     if args.impl == "reference":

@@ -11,7 +11,6 @@
 namespace sfb {
 namespace {
 
-constexpr int FIN_THREADS = 256;
 constexpr int ROW_CACHE_FLOATS = 48 * 1024;   // 192 KB of dynamic shared memory
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -58,7 +57,7 @@ __device__ __forceinline__ void store_u4(char* row, int j, float4 v, int es) {
 }
 
 // z rows are fp32 with ld a multiple of 4; values beyond J inside the last float4 are ignored.
-__global__ void __launch_bounds__(FIN_THREADS) finish_mlr_kernel(RowMap z, RowMap u, const int32_t* __restrict__ labels,
+__global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, const int32_t* __restrict__ labels,
                                                                  int K, int J, int cache_floats, int* dev_status) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
@@ -71,7 +70,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finish_mlr_kernel(RowMap z, RowMa
   const float kLog2e = 1.4426950408889634f;
 
   float m = -INFINITY;
-  for (int q = threadIdx.x; q < J4; q += FIN_THREADS) {
+  for (int q = threadIdx.x; q < J4; q += blockDim.x) {
     float4 t = *reinterpret_cast<const float4*>(zr + q * 4);
     const int j = q * 4;
     if (j + 1 >= J) t.y = -INFINITY;
@@ -84,7 +83,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finish_mlr_kernel(RowMap z, RowMa
 
   float s = 0.f;
   const float mb = m * kLog2e;
-  for (int q = threadIdx.x; q < J4; q += FIN_THREADS) {
+  for (int q = threadIdx.x; q < J4; q += blockDim.x) {
     const int j = q * 4;
     float4 t;
     if (cached) {
@@ -107,7 +106,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finish_mlr_kernel(RowMap z, RowMa
   const bool bad = (y < 0) || (y >= J);
   if (bad && threadIdx.x == 0) atomicOr(dev_status, SFB_DEV_BAD_LABEL);
   const int ld4 = u.ld >> 2;   // u.ld is a multiple of 4 (fp32) or 8 (bf16)
-  for (int q = threadIdx.x; q < ld4; q += FIN_THREADS) {
+  for (int q = threadIdx.x; q < ld4; q += blockDim.x) {
     const int j = q * 4;
     float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
     if (q < J4 && !bad) {
@@ -131,7 +130,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finish_mlr_kernel(RowMap z, RowMa
   }
 }
 
-__global__ void __launch_bounds__(FIN_THREADS) finish_dml_kernel(RowMap z, RowMap u, const uint8_t* __restrict__ similar,
+__global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, const uint8_t* __restrict__ similar,
                                                                  float margin, int K, int J, int cache_floats) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
@@ -143,7 +142,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finish_dml_kernel(RowMap z, RowMa
   const bool cached = (J4 * 4) <= cache_floats;
 
   float n = 0.f;
-  for (int q = threadIdx.x; q < J4; q += FIN_THREADS) {
+  for (int q = threadIdx.x; q < J4; q += blockDim.x) {
     float4 t = *reinterpret_cast<const float4*>(zr + q * 4);
     const int j = q * 4;
     if (j + 1 >= J) t.y = 0.f;
@@ -157,7 +156,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finish_dml_kernel(RowMap z, RowMa
   const float g = sim ? 1.f : ((n < margin) ? -1.f : 0.f);   // strict hinge: inactive at equality
 
   const int ld4 = u.ld >> 2;
-  for (int q = threadIdx.x; q < ld4; q += FIN_THREADS) {
+  for (int q = threadIdx.x; q < ld4; q += blockDim.x) {
     const int j = q * 4;
     float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
     if (q < J4 && g != 0.f) {
@@ -233,6 +232,9 @@ __global__ void __launch_bounds__(256) cast_bf16_kernel(const float* __restrict_
   }
 }
 
+// Long rows take a whole SM's worth of shared memory, so one block must supply all the memory parallelism.
+int fin_threads(int J) { return J >= 8192 ? 1024 : 256; }
+
 int fin_cache_floats(int J) {
   const int need = ((J + 3) / 4) * 4;
   return need <= ROW_CACHE_FLOATS ? need : 0;
@@ -248,7 +250,7 @@ int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels,
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     attr_done = true;
   }
-  finish_mlr_kernel<<<K, FIN_THREADS, (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status);
+  finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
@@ -260,7 +262,7 @@ int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     attr_done = true;
   }
-  finish_dml_kernel<<<K, FIN_THREADS, (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf);
+  finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

@@ -8,8 +8,8 @@
 //             the output index ("MN-major"); tcgen05 reads them in that form directly from the SF
 //             buffer's worker streams, no transposed copy is made.
 //
-// Warp roles (192 threads): warp 0 issues TMA loads into a 4-stage shared-memory ring, warp 1 issues
-// the MMAs (one thread) into one of two TMEM accumulators, warps 2-5 drain the other accumulator
+// Warp roles (320 threads): warp 0 issues TMA loads into a 4-stage shared-memory ring, warp 1 issues
+// the MMAs (one thread) into one of two TMEM accumulators, warps 2-9 drain the other accumulator
 // (tcgen05.ld) and run the epilogue, so the write-back of tile t overlaps the MMAs of tile t+1.
 // Every wait on an mbarrier is bounded; a wait that runs out sets SFB_DEV_TIMEOUT and the CTA leaves
 // through the common exit (TMEM freed) instead of hanging.
@@ -31,11 +31,13 @@ namespace {
 constexpr int BM = 128;          // tile rows  = TMEM lanes
 constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * 128;   // 128 rows (K-major) or 128 output indices (MN-major) x 128 B... per 64/32 reduction steps
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
+constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct GemmParams {
   int m_tiles, n_tiles, k_blocks;
+  int m_fastest;            // tile order: 1 = consecutive tiles share the B operand slab, 0 = share the A slab
   int B, P;                 // rows per worker / workers, geometry of the 3-D operand maps
   int m_bb, m_wp, m_tpw;    // forward: A rows per tile come as a box of m_bb rows x m_wp workers; tiles per worker
   int k_bb, k_wp, k_bpw;    // apply: a reduction block is k_bb rows x k_wp workers; blocks per worker
@@ -79,7 +81,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles + STAGES * STAGE_BYTES);
+  float* epi_stage = reinterpret_cast<float*>(tiles + STAGES * STAGE_BYTES);
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles + STAGES * STAGE_BYTES + EPI_STAGE_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (p.status_ro != nullptr && (*p.status_ro & SFB_DEV_BAD_HEADER)) return;   // uniform over the grid
@@ -91,7 +94,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->tmem_full[b], 1);
-      ptx::mbar_init(&ctl->tmem_empty[b], 128);
+      ptx::mbar_init(&ctl->tmem_empty[b], 256);
     }
     ctl->abort = 0;
     ptx::fence_barrier_init();
@@ -115,7 +118,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int issued = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+      const int mt = p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles;
+      const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
       for (int kb = 0; kb < p.k_blocks; ++kb) {
         ok = wait_or_abort(&ctl->empty[s], ph ^ 1u, ctl, p.status);
         if (!ok) break;
@@ -198,67 +202,86 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
-    const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int r = quarter * 32 + lane;            // row of the tile this thread owns
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // A warp may only read the TMEM lanes of its quarter (warp index mod 4).  Two warps share each
+    // quarter and split the tile's columns in halves.  Per 32 x 32 block: accumulators come out of
+    // TMEM one row per thread, go through an XOR-swizzled 4 KB shared-memory block, and are read back
+    // four rows x 128 bytes per warp instruction, so that every global access is a full 128-byte line.
+    const int e = warp - 2;
+    const int quarter = warp & 3;
+    const int half = e >> 2;
+    float* stage = epi_stage + e * 1024;
+    const int lrow = lane >> 3, lq = lane & 7;    // transposed assignment: row-in-group, 16-byte column
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+      const int mt = p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles;
+      const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
       ok = wait_or_abort(&ctl->tmem_full[buf], acc_ph, ctl, p.status);
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
-      float* row_ptr = nullptr;         // fp32 destination row of this thread (nullptr: nothing to store)
-      __nv_bfloat16* sh_ptr = nullptr;
-      int ncols;                        // valid columns of the row, counted from column 0 of the matrix
-      if (APPLY) {
-        const int j = mt * BM + r;
-        ncols = p.Nvalid;
-        if (j < p.Mvalid) {
-          row_ptr = p.W + (long long)j * p.ldw;
-          if (p.shadow != nullptr) sh_ptr = p.shadow + (long long)j * p.ldw;
-        }
-      } else {
-        int wp_, slot;
-        if (p.B >= BM) { wp_ = mt / p.m_tpw; slot = (mt % p.m_tpw) * BM + r; }
-        else { wp_ = mt * p.m_wp + r / p.m_bb; slot = r % p.m_bb; }
-        ncols = p.z.ld;
-        if (wp_ < p.P && slot < p.B) row_ptr = reinterpret_cast<float*>(p.z.row(wp_ * p.B + slot));
-      }
-#pragma unroll 1
-      for (int cc = 0; cc < BN / 32; ++cc) {
-        uint32_t v[32];
-        ptx::tmem_ld32(taddr + cc * 32, v);
-        ptx::tmem_ld_wait();
-        if (row_ptr != nullptr) {
-          const int c0 = nt * BN + cc * 32;
+      // destination rows of the 8 row groups this lane touches (row = quarter*32 + 4*g + lrow)
+      float* rowp[8];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const int c = c0 + q * 4;
-            if (c < ncols) {   // ncols is a multiple of 4 on these paths
-              float4 a = make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]),
-                                     __uint_as_float(v[q * 4 + 2]), __uint_as_float(v[q * 4 + 3]));
-              if (APPLY) {
-                float4 w = *reinterpret_cast<const float4*>(row_ptr + c);
-                w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
-                w.z = fmaf(-p.eta, a.z, w.z); w.w = fmaf(-p.eta, a.w, w.w);
-                *reinterpret_cast<float4*>(row_ptr + c) = w;
-                if (sh_ptr != nullptr) {
-                  __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
-                  uint2 pk;
-                  pk.x = *reinterpret_cast<uint32_t*>(&lo);
-                  pk.y = *reinterpret_cast<uint32_t*>(&hi);
-                  *reinterpret_cast<uint2*>(sh_ptr + c) = pk;
-                }
-              } else {
-                *reinterpret_cast<float4*>(row_ptr + c) = a;
+      for (int g = 0; g < 8; ++g) {
+        const int r = quarter * 32 + 4 * g + lrow;
+        rowp[g] = nullptr;
+        if (APPLY) {
+          const int j = mt * BM + r;
+          if (j < p.Mvalid) rowp[g] = p.W + (long long)j * p.ldw;
+        } else {
+          int wp_, slot;
+          if (p.B >= BM) { wp_ = mt / p.m_tpw; slot = (mt % p.m_tpw) * BM + r; }
+          else { wp_ = mt * p.m_wp + r / p.m_bb; slot = r % p.m_bb; }
+          if (wp_ < p.P && slot < p.B) rowp[g] = reinterpret_cast<float*>(p.z.row(wp_ * p.B + slot));
+        }
+      }
+      const int ncols = APPLY ? p.Nvalid : p.z.ld;   // multiples of 4 on these paths
+#pragma unroll 1
+      for (int cc = 0; cc < BN / 64; ++cc) {
+        const int col_in_tile = half * (BN / 2) + cc * 32;
+        const int c = nt * BN + col_in_tile + lq * 4;
+        float4 wv[8];
+        if (APPLY) {   // the old W does not depend on the MMAs: fetch it before touching the accumulator
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            wv[g] = (rowp[g] != nullptr && c < ncols) ? *reinterpret_cast<const float4*>(rowp[g] + c)
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        uint32_t v[32];
+        ptx::tmem_ld32(taddr + col_in_tile, v);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(stage + lane * 32 + ((q ^ (lane & 7)) << 2)) =
+              make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        __syncwarp();
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const int lr = 4 * g + lrow;
+          const float4 a = *reinterpret_cast<const float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2));
+          if (rowp[g] != nullptr && c < ncols) {
+            if (APPLY) {
+              float4 w = wv[g];
+              w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
+              w.z = fmaf(-p.eta, a.z, w.z); w.w = fmaf(-p.eta, a.w, w.w);
+              *reinterpret_cast<float4*>(rowp[g] + c) = w;
+              if (p.shadow != nullptr) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(p.shadow + (rowp[g] - p.W) + c) = pk;
               }
+            } else {
+              *reinterpret_cast<float4*>(rowp[g] + c) = a;
             }
           }
         }
+        __syncwarp();
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&ctl->tmem_empty[buf]);
@@ -312,7 +335,7 @@ int pow2_at_least(int n) {
 
 template <int ES, bool APPLY, int BN>
 int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, int num_sms) {
-  constexpr int smem = STAGES * (A_STAGE_BYTES + BN * 128) + 1024 + (int)sizeof(SharedCtl);
+  constexpr int smem = STAGES * (A_STAGE_BYTES + BN * 128) + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(umma_gemm_kernel<ES, APPLY, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
@@ -372,6 +395,8 @@ static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a,
   const int bn = (d.J > 128 && (long long)p.m_tiles * ((d.J + 255) / 256) >= pl->num_sms) ? 256 : 128;
   p.n_tiles = (d.J + bn - 1) / bn;
   p.k_blocks = (d.D + CH - 1) / CH;
+  // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
+  p.m_fastest = ((long long)d.J * d.D > (long long)d.P * d.B * d.D) ? 1 : 0;
   p.z = z;
   p.status = dev_status;
   CUtensorMap ta, tb;
@@ -430,6 +455,7 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
   const int bn = ((long long)p.m_tiles * ((d.D + 255) / 256) >= pl->num_sms) ? 256 : 128;
   p.n_tiles = (d.D + bn - 1) / bn;
   p.Mvalid = d.J; p.Nvalid = d.D;
+  p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
   p.W = reinterpret_cast<float*>(W);
   p.shadow = (d.path == SFB_PATH_BF16) ? w_shadow : nullptr;
   p.ldw = d.D;

@@ -101,11 +101,32 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
         assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1]), \
             "two runs from the same state must be bit-identical"
         W_gpu = runs[0][0].astype(np.float64)
-        moved = np.linalg.norm(W_or - W0)
-        e_step = np.linalg.norm((W_gpu - W0) - (W_or - W0)) / moved
-        # W is stored in fp32: its storage rounding (2^-24 per element, relative) is not the kernel's error
-        storage = steps * 2.0 ** -24 * np.linalg.norm(W0) / moved
-        assert e_step <= tol + storage, f"E_step = {e_step:.3e} > {tol} + {storage:.1e}"
+        if cfg["model"] == "dml":
+            # The hinge gate is discontinuous: a pair within the tie band may legitimately take either
+            # value, after which free-running trajectories differ.  So every step is checked on its own,
+            # started from the GPU's current L, with the GPU's gate accepted on in-band pairs only.
+            wl.reset()
+            e_step = 0.0
+            for t in range(steps):
+                bt = batch_of(inputs, cfg, t % cfg["pool"])
+                W_t = wl.W.cpu().numpy()
+                wl.step(t, eta=eta)
+                torch.cuda.synchronize()
+                _, U_wire, _ = orc.unpack(wl.sf_buf.cpu().numpy())
+                U_o, V_o, ex = oracle_factors(cfg, W_t, bt)
+                U_fix = dml_accept_gate(cfg, U_wire.astype(np.float64), U_o, ex, path)
+                ref_move = -eta * orc.delta_w(U_fix, V_o)
+                got_move = wl.W.cpu().numpy().astype(np.float64) - W_t.astype(np.float64)
+                storage = 2.0 ** -24 * np.linalg.norm(W_t) / np.linalg.norm(ref_move)
+                e_t = np.linalg.norm(got_move - ref_move) / np.linalg.norm(ref_move)
+                assert e_t <= tol + storage, f"step {t}: E_step = {e_t:.3e} > {tol} + {storage:.1e}"
+                e_step = max(e_step, e_t)
+        else:
+            moved = np.linalg.norm(W_or - W0)
+            e_step = np.linalg.norm((W_gpu - W0) - (W_or - W0)) / moved
+            # W is stored in fp32: its storage rounding (2^-24 per element, relative) is not the kernel's error
+            storage = steps * 2.0 ** -24 * np.linalg.norm(W0) / moved
+            assert e_step <= tol + storage, f"E_step = {e_step:.3e} > {tol} + {storage:.1e}"
         # the buffer left by the last step is a valid serialisation with the step's clock
         h, U_last, _ = orc.unpack(runs[0][1])
         assert h["clock"] == steps - 1 and h["P"] == cfg["P"] and h["J"] == J
