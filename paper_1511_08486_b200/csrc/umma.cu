@@ -37,6 +37,7 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct GemmParams {
   int m_tiles, n_tiles, k_blocks;
+  int a_policy, b_policy;   // L2 eviction policy of the operand loads (0 normal, 1 evict first, 2 evict last)
   int m_fastest;            // tile order: 1 = consecutive tiles share the B operand slab, 0 = share the A slab
   int B, P;                 // rows per worker / workers, geometry of the 3-D operand maps
   int m_bb, m_wp, m_tpw;    // forward: A rows per tile come as a box of m_bb rows x m_wp workers; tiles per worker
@@ -117,6 +118,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint32_t ph = 0;
     int issued = 0;
     bool ok = true;
+    const uint64_t pol_a = ptx::l2_policy(p.a_policy), pol_b = ptx::l2_policy(p.b_policy);
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int mt = p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles;
       const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
@@ -132,18 +134,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int slot0, p0;
             if (p.B >= BM) { p0 = mt / p.m_tpw; slot0 = (mt % p.m_tpw) * BM; }
             else { p0 = mt * p.m_wp; slot0 = 0; }
-            ptx::tma_load_3d(a_dst, &tmA, &ctl->full[s], k0, slot0, p0);
-            ptx::tma_load_3d(b_dst, &tmB, &ctl->full[s], k0, nt * BN, 0);
+            ptx::tma_load_3d_hint(a_dst, &tmA, &ctl->full[s], k0, slot0, p0, pol_a);
+            ptx::tma_load_3d_hint(b_dst, &tmB, &ctl->full[s], k0, nt * BN, 0, pol_b);
           } else {
             int row0, p0;
             if (p.B >= BK) { p0 = kb / p.k_bpw; row0 = (kb % p.k_bpw) * BK; }
             else { p0 = kb * p.k_wp; row0 = 0; }
 #pragma unroll
             for (int c = 0; c < BM / CH; ++c)
-              ptx::tma_load_3d(a_dst + c * (BK * 128), &tmA, &ctl->full[s], mt * BM + c * CH, row0, p0);
+              ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, &ctl->full[s], mt * BM + c * CH, row0, p0, pol_a);
 #pragma unroll
             for (int c = 0; c < BN / CH; ++c)
-              ptx::tma_load_3d(b_dst + c * (BK * 128), &tmB, &ctl->full[s], nt * BN + c * CH, row0, p0);
+              ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, &ctl->full[s], nt * BN + c * CH, row0, p0, pol_b);
           }
         }
         __syncwarp();
@@ -219,10 +221,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
-      ok = wait_or_abort(&ctl->tmem_full[buf], acc_ph, ctl, p.status);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
       // destination rows of the 8 row groups this lane touches (row = quarter*32 + 4*g + lrow)
       float* rowp[8];
 #pragma unroll
@@ -240,19 +238,42 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
       }
       const int ncols = APPLY ? p.Nvalid : p.z.ld;   // multiples of 4 on these paths
+      const int cbase = nt * BN + half * (BN / 2) + lq * 4;
+      // The old W does not depend on the MMAs: while this tile's accumulator is still being produced,
+      // pull the first block of W into registers and ask L2 for the rest of the tile.
+      float4 wv[8];
+#pragma unroll
+      for (int g = 0; g < 8; ++g) wv[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (APPLY) {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+          if (rowp[g] != nullptr && cbase < ncols) wv[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + cbase));
+        if (lq == 0) {   // one 128-byte line per (row, 32-column block)
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            for (int cc = 1; cc < BN / 64; ++cc)
+              if (rowp[g] != nullptr && cbase + cc * 32 < ncols)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp[g] + cbase + cc * 32));
+        }
+      }
+      ok = wait_or_abort(&ctl->tmem_full[buf], acc_ph, ctl, p.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
       for (int cc = 0; cc < BN / 64; ++cc) {
         const int col_in_tile = half * (BN / 2) + cc * 32;
-        const int c = nt * BN + col_in_tile + lq * 4;
-        float4 wv[8];
-        if (APPLY) {   // the old W does not depend on the MMAs: fetch it before touching the accumulator
-#pragma unroll
-          for (int g = 0; g < 8; ++g)
-            wv[g] = (rowp[g] != nullptr && c < ncols) ? *reinterpret_cast<const float4*>(rowp[g] + c)
-                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+        const int c = cbase + cc * 32;
         uint32_t v[32];
         ptx::tmem_ld32(taddr + col_in_tile, v);
+        float4 wn[8];   // next block of W, in flight while this block is combined and stored
+#pragma unroll
+        for (int g = 0; g < 8; ++g) wn[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (APPLY && cc + 1 < BN / 64) {
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
+        }
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int q = 0; q < 8; ++q)
@@ -268,19 +289,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               float4 w = wv[g];
               w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
               w.z = fmaf(-p.eta, a.z, w.z); w.w = fmaf(-p.eta, a.w, w.w);
-              *reinterpret_cast<float4*>(rowp[g] + c) = w;
+              __stcs(reinterpret_cast<float4*>(rowp[g] + c), w);   // streamed: keep L2 for the factors
               if (p.shadow != nullptr) {
                 __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
                 uint2 pk;
                 pk.x = *reinterpret_cast<uint32_t*>(&lo);
                 pk.y = *reinterpret_cast<uint32_t*>(&hi);
-                *reinterpret_cast<uint2*>(p.shadow + (rowp[g] - p.W) + c) = pk;
+                __stcs(reinterpret_cast<uint2*>(p.shadow + (rowp[g] - p.W) + c), pk);
               }
             } else {
-              *reinterpret_cast<float4*>(rowp[g] + c) = a;
+              __stcs(reinterpret_cast<float4*>(rowp[g] + c), a);
             }
           }
         }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) wv[g] = wn[g];
         __syncwarp();
       }
       ptx::tc_fence_before();
@@ -397,6 +420,8 @@ static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a,
   p.k_blocks = (d.D + CH - 1) / CH;
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
   p.m_fastest = ((long long)d.J * d.D > (long long)d.P * d.B * d.D) ? 1 : 0;
+  p.a_policy = p.m_fastest ? 2 : 0;   // the operand whose slab changes every tile is re-read all along: keep it
+  p.b_policy = p.m_fastest ? 0 : 2;
   p.z = z;
   p.status = dev_status;
   CUtensorMap ta, tb;
@@ -456,6 +481,8 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
   p.n_tiles = (d.D + bn - 1) / bn;
   p.Mvalid = d.J; p.Nvalid = d.D;
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
+  p.a_policy = p.m_fastest ? 2 : 0;
+  p.b_policy = p.m_fastest ? 0 : 2;
   p.W = reinterpret_cast<float*>(W);
   p.shadow = (d.path == SFB_PATH_BF16) ? w_shadow : nullptr;
   p.ldw = d.D;
