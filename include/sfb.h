@@ -71,7 +71,8 @@ enum {
   SFB_ERR_SHAPE = -2,       /* non-positive or unsupported sizes */
   SFB_ERR_UNSUPPORTED = -3, /* model/path combination not provided, or not an sm_100 device */
   SFB_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed */
-  SFB_ERR_ALLOC = -5        /* workspace allocation failed */
+  SFB_ERR_ALLOC = -5,       /* workspace allocation failed */
+  SFB_ERR_SCRATCH = -6      /* problem larger than the fixed scratch of sfb_sc_factors_noalloc */
 };
 
 /* bits of the device status word */
@@ -159,6 +160,31 @@ int sfb_stage_ms(sfb_ctx* ctx, float* factors_ms, float* apply_ms, int32_t* step
 int64_t sfb_launch_count(const sfb_ctx* ctx);
 
 const char* sfb_strerror(int code);
+
+/* Sparse-coding factors u_i = W a_i - x_i for callers that must not allocate device memory: code
+ * that runs while its stream is being captured into a CUDA graph, latency-bound loops that cannot
+ * afford the allocator's implicit synchronisation, and processes whose device memory was handed
+ * out once, with a fixed budget, by an outer framework.  (The paper has no counterpart: this is a
+ * packaging variant of sfb_compute_factors for SFB_SC, same kernels, same results.)
+ *
+ * It takes no context.  Its scratch, the atom-major copy of W, is a fixed 16 MiB device array
+ * built into the library (every GPU that loads the library carries it until the process exits),
+ * so D * roundup(J, 4) may be at most sfb_noalloc_max_scratch_floats() = 4 Mi values; larger
+ * problems return SFB_ERR_SCRATCH and launch nothing.  The call itself never allocates or frees.
+ *
+ * W [J][D] fp32; rowptr [K+1], idx, val: CSR codes (fp32 values, strictly ascending indices);
+ * Xdata [K][J] fp32; U out [K][ldu] fp32 with ldu >= J a multiple of 4 (pad columns written as
+ * zeros).  dev_status: optional device int that receives the SFB_DEV_* bits (cleared by the call);
+ * NULL keeps them in the library's own word.  All pointers are device pointers of the caller.
+ *
+ * The first call on each device looks up the address of the built-in array; make that first call
+ * outside any stream capture.  All calls share the array and it keeps the last call's contents:
+ * everything a call depends on is rewritten by that call, but two calls that overlap on the GPU
+ * (different streams, or concurrent host threads) race on it, so keep them on one stream. */
+int sfb_sc_factors_noalloc(const void* W, int32_t J, int32_t D, int32_t K, const uint32_t* rowptr,
+                           const uint32_t* idx, const void* val, const void* Xdata, void* U, int32_t ldu,
+                           int32_t* dev_status, void* cuda_stream);
+int64_t sfb_noalloc_max_scratch_floats(void);
 
 #ifdef __cplusplus
 }

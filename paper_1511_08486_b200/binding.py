@@ -22,7 +22,7 @@ PATHS = {"f32": SFB_PATH_F32, "tf32": SFB_PATH_TF32, "bf16": SFB_PATH_BF16}
 EXPORTS = (
     "sfb_create", "sfb_destroy", "sfb_sf_buffer_bytes", "sfb_ld", "sfb_compute_factors", "sfb_pack",
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
-    "sfb_profile", "sfb_stage_ms",
+    "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
 )
 
 
@@ -82,6 +82,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_profile.restype = C.c_int
     lib.sfb_stage_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.sfb_stage_ms.restype = C.c_int
+    lib.sfb_sc_factors_noalloc.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, C.c_int32, vp, vp]
+    lib.sfb_sc_factors_noalloc.restype = C.c_int
+    lib.sfb_noalloc_max_scratch_floats.argtypes = []
+    lib.sfb_noalloc_max_scratch_floats.restype = C.c_int64
     lib.sfb_strerror.argtypes = [C.c_int]
     lib.sfb_strerror.restype = C.c_char_p
     if path == LIB_PATH:
@@ -121,6 +125,25 @@ def sfb_ld(desc: sfb_desc) -> tuple[int, int]:
     if r != SFB_OK:
         raise SfbError(r, "sfb_ld")
     return ldu.value, ldv.value
+
+
+def sfb_sc_factors_noalloc(W, J, D, K, rowptr, idx, val, Xdata, U, ldu, dev_status=None, stream=None) -> None:
+    """Sparse-coding factors without any device allocation (see include/sfb.h); raises SfbError on a negative code.
+
+    For callers that cannot allocate: no context is created, the scratch is a fixed array inside the
+    library.  Calls share that array, so keep them on one stream.
+    """
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    r = load_library().sfb_sc_factors_noalloc(_ptr(W), J, D, K, _ptr(rowptr), _ptr(idx), _ptr(val), _ptr(Xdata),
+                                              _ptr(U), ldu, _ptr(dev_status), C.c_void_p(stream))
+    if r != SFB_OK:
+        raise SfbError(r, "sfb_sc_factors_noalloc")
+
+
+def sfb_noalloc_max_scratch_floats() -> int:
+    return int(load_library().sfb_noalloc_max_scratch_floats())
 
 
 class Context:

@@ -153,6 +153,7 @@ const char* sfb_strerror(int code) {
     case SFB_ERR_UNSUPPORTED: return "model/path combination not provided, or not an sm_100 device";
     case SFB_ERR_CUDA: return "a CUDA call failed";
     case SFB_ERR_ALLOC: return "workspace allocation failed";
+    case SFB_ERR_SCRATCH: return "problem exceeds the fixed scratch array of the no-allocation entry point";
     default: return "unknown error";
   }
 }
