@@ -16,6 +16,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "umma.cuh"
@@ -28,19 +29,20 @@ int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v,
 
 namespace {
 
-constexpr int BM = 128;          // tile rows  = TMEM lanes
-constexpr int STAGES = 4;
-constexpr int A_STAGE_BYTES = BM * 128;   // 128 rows (K-major) or 128 output indices (MN-major) x 128 B... per 64/32 reduction steps
+constexpr int BM = 128;          // rows per CTA tile = TMEM lanes
+constexpr int A_STAGE_BYTES = BM * 128;   // A operand of one pipeline stage: 128 rows (or output indices) x 128 bytes
 constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
+constexpr int RING_BYTES = 192 * 1024;   // shared memory given to the operand ring
+constexpr int MAX_STAGES = 8;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct GemmParams {
-  int m_tiles, n_tiles, k_blocks;
+  int m_tiles, n_tiles, k_blocks;   // m_tiles counts tiles of 128*CG rows
   int a_policy, b_policy;   // L2 eviction policy of the operand loads (0 normal, 1 evict first, 2 evict last)
   int m_fastest;            // tile order: 1 = consecutive tiles share the B operand slab, 0 = share the A slab
   int B, P;                 // rows per worker / workers, geometry of the 3-D operand maps
-  int m_bb, m_wp, m_tpw;    // forward: A rows per tile come as a box of m_bb rows x m_wp workers; tiles per worker
+  int m_bb, m_wp, m_tpw;    // forward: 128 A rows come as a box of m_bb rows x m_wp workers; 128-row units per worker
   int k_bb, k_wp, k_bpw;    // apply: a reduction block is k_bb rows x k_wp workers; blocks per worker
   int Mvalid, Nvalid;       // forward: (unused, N = J) ; apply: (J, D)
   float* W;                 // apply: fp32 master, row stride ldw
@@ -53,7 +55,7 @@ struct GemmParams {
 };
 
 struct SharedCtl {
-  uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -70,15 +72,24 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sh
 
 // ES: bytes per operand value (2 = bf16, 4 = tf32).  APPLY: MN-major operands and the W write-back
 // epilogue; otherwise K-major operands and the plain fp32 store of Z.  BN: tile columns.
-template <int ES, bool APPLY, int BN>
+// CG: CTAs per MMA.  With CG = 2 the kernel runs as clusters of two CTAs working on a 256 x BN tile:
+// each CTA loads its own 128 rows of A and its own half of B's columns, the even CTA issues
+// tcgen05.mma.cta_group::2 (M = 256) for the pair, each CTA drains its own 128 accumulator rows.
+// Signals of the pair: TMA bytes of both CTAs are credited to the even CTA's "full" barrier;
+// "stage free" and "accumulator ready" are committed (tcgen05.commit) once to the even CTA's barrier
+// and once to the odd CTA's; both CTAs' epilogues arrive on the even CTA's "accumulator drained"
+// barrier.
+template <int ES, bool APPLY, int BN, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr int CH = 128 / ES;                 // values per 128-byte chunk
   constexpr int BK = CH;                       // reduction steps per pipeline stage (64 bf16 / 32 tf32)
   constexpr int UMMA_K = 32 / ES;              // reduction steps per instruction (16 bf16 / 8 tf32)
-  constexpr int B_STAGE_BYTES = BN * 128;
+  constexpr int BNC = BN / CG;                 // B columns this CTA loads
+  constexpr int B_STAGE_BYTES = BNC * 128;
   constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-  constexpr uint32_t IDESC = ptx::instr_desc(ES == 2 ? 1u : 2u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM, BN);
+  constexpr int STAGES = (RING_BYTES / STAGE_BYTES) < MAX_STAGES ? (RING_BYTES / STAGE_BYTES) : MAX_STAGES;
+  constexpr uint32_t IDESC = ptx::instr_desc(ES == 2 ? 1u : 2u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM * CG, BN);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -88,6 +99,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (p.status_ro != nullptr && (*p.status_ro & SFB_DEV_BAD_HEADER)) return;   // uniform over the grid
 
+  const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;   // 0 = the CTA that issues the MMAs
+  const int cluster_id = blockIdx.x / CG, num_clusters = gridDim.x / CG;
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&ctl->full[s], 1);
@@ -95,7 +109,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->tmem_full[b], 1);
-      ptx::mbar_init(&ctl->tmem_empty[b], 256);
+      ptx::mbar_init(&ctl->tmem_empty[b], 8 * CG);   // one arrival per epilogue warp of every CTA of the pair
     }
     ctl->abort = 0;
     ptx::fence_barrier_init();
@@ -103,49 +117,64 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::prefetch_tmap(&tmB);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&ctl->tmem_base, 2 * BN);
-    ptx::tmem_relinquish();
+    ptx::tmem_alloc<CG>(&ctl->tmem_base, 2 * BN);
+    ptx::tmem_relinquish<CG>();
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync();   // the peer's barriers exist before anything is signalled remotely
   ptx::tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   const int total_tiles = p.m_tiles * p.n_tiles;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (every CTA)
     int s = 0;
     uint32_t ph = 0;
     int issued = 0;
     bool ok = true;
     const uint64_t pol_a = ptx::l2_policy(p.a_policy), pol_b = ptx::l2_policy(p.b_policy);
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int mt = p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles;
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
+      const int mt = (p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles) * CG + (int)rank;   // 128-row unit
       const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
+      const int ncol0 = nt * BN + (int)rank * BNC;                                           // first B column loaded here
       for (int kb = 0; kb < p.k_blocks; ++kb) {
         ok = wait_or_abort(&ctl->empty[s], ph ^ 1u, ctl, p.status);
         if (!ok) break;
         if (lane == 0) {
           uint8_t* a_dst = tiles + s * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_STAGE_BYTES;
-          ptx::mbar_expect_tx(&ctl->full[s], STAGE_BYTES);
+          uint32_t full_addr = ptx::smem_u32(&ctl->full[s]);
+          if (CG == 2) {
+            full_addr = ptx::map_to_cta(full_addr, 0);
+          }
+          if (rank == 0) ptx::mbar_expect_tx(&ctl->full[s], CG * STAGE_BYTES);
           if (!APPLY) {
             const int k0 = kb * BK;
             int slot0, p0;
             if (p.B >= BM) { p0 = mt / p.m_tpw; slot0 = (mt % p.m_tpw) * BM; }
             else { p0 = mt * p.m_wp; slot0 = 0; }
-            ptx::tma_load_3d_hint(a_dst, &tmA, &ctl->full[s], k0, slot0, p0, pol_a);
-            ptx::tma_load_3d_hint(b_dst, &tmB, &ctl->full[s], k0, nt * BN, 0, pol_b);
+            if (CG == 1) {
+              ptx::tma_load_3d_hint(a_dst, &tmA, &ctl->full[s], k0, slot0, p0, pol_a);
+              ptx::tma_load_3d_hint(b_dst, &tmB, &ctl->full[s], k0, ncol0, 0, pol_b);
+            } else {
+              ptx::tma_load_3d_hint_pair(a_dst, &tmA, full_addr, k0, slot0, p0, pol_a);
+              ptx::tma_load_3d_hint_pair(b_dst, &tmB, full_addr, k0, ncol0, 0, pol_b);
+            }
           } else {
             int row0, p0;
             if (p.B >= BK) { p0 = kb / p.k_bpw; row0 = (kb % p.k_bpw) * BK; }
             else { p0 = kb * p.k_wp; row0 = 0; }
 #pragma unroll
-            for (int c = 0; c < BM / CH; ++c)
-              ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, &ctl->full[s], mt * BM + c * CH, row0, p0, pol_a);
+            for (int c = 0; c < BM / CH; ++c) {
+              if (CG == 1) ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, &ctl->full[s], mt * BM + c * CH, row0, p0, pol_a);
+              else ptx::tma_load_3d_hint_pair(a_dst + c * (BK * 128), &tmA, full_addr, mt * BM + c * CH, row0, p0, pol_a);
+            }
 #pragma unroll
-            for (int c = 0; c < BN / CH; ++c)
-              ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, &ctl->full[s], nt * BN + c * CH, row0, p0, pol_b);
+            for (int c = 0; c < BNC / CH; ++c) {
+              if (CG == 1) ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, &ctl->full[s], ncol0 + c * CH, row0, p0, pol_b);
+              else ptx::tma_load_3d_hint_pair(b_dst + c * (BK * 128), &tmB, full_addr, ncol0 + c * CH, row0, p0, pol_b);
+            }
           }
         }
         __syncwarp();
@@ -153,7 +182,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
-    if (!ok || ctl->abort) {
+    if ((!ok || ctl->abort) && rank == 0) {
       // let copies already in flight land before the CTA goes away (bounded)
       int n = issued < STAGES ? issued : STAGES;
       for (int q = 0; q < n; ++q) {
@@ -164,12 +193,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ MMA issuer (even CTA only)
     int s = 0;
     uint32_t ph = 0;
     int it = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+    bool ok = (rank == 0);
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++it) {
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
       ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
@@ -193,18 +222,22 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-            if (ES == 2) ptx::mma_f16(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
-            else ptx::mma_tf32(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+            if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+            else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
           }
-          ptx::mma_commit(&ctl->empty[s]);                     // stage reusable once these MMAs have read it
-          if (kb == p.k_blocks - 1) ptx::mma_commit(&ctl->tmem_full[buf]);   // accumulator complete
+          ptx::mma_commit<CG>(&ctl->empty[s]);                     // stage reusable once these MMAs have read it
+          if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->empty[s]), 1));
+          if (kb == p.k_blocks - 1) {                              // accumulator complete, in both CTAs
+            ptx::mma_commit<CG>(&ctl->tmem_full[buf]);
+            if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_full[buf]), 1));
+          }
         }
         __syncwarp();
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // ------------------------------------------------------------------ epilogue (warps 2..9, every CTA)
     // A warp may only read the TMEM lanes of its quarter (warp index mod 4).  Two warps share each
     // quarter and split the tile's columns in halves.  Per 32 x 32 block: accumulators come out of
     // TMEM one row per thread, go through an XOR-swizzled 4 KB shared-memory block, and are read back
@@ -216,8 +249,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int lrow = lane >> 3, lq = lane & 7;    // transposed assignment: row-in-group, 16-byte column
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles;
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++it) {
+      const int mt = (p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles) * CG + (int)rank;
       const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
@@ -307,15 +340,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         __syncwarp();
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&ctl->tmem_empty[buf]);
+      __syncwarp();
+      if (lane == 0) {   // this warp's part of the accumulator is drained
+        if (CG == 1 || rank == 0) ptx::mbar_arrive(&ctl->tmem_empty[buf]);
+        else ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[buf]), 0));
+      }
     }
   }
 
   ptx::tc_fence_before();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync();   // nobody leaves while its pair may still signal it or read its tiles
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 2 * BN);
+    ptx::tmem_dealloc<CG>(tmem_base, 2 * BN);
   }
 }
 
@@ -356,27 +394,65 @@ int pow2_at_least(int n) {
   return p;
 }
 
-template <int ES, bool APPLY, int BN>
+template <int ES, bool APPLY, int BN, int CG>
 int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, int num_sms) {
-  constexpr int smem = STAGES * (A_STAGE_BYTES + BN * 128) + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
+  constexpr int stage_bytes = A_STAGE_BYTES + (BN / CG) * 128;
+  constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
+  constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
+  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG>;
   static bool attr_done = false;
+  static int max_clusters = 0;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(umma_gemm_kernel<ES, APPLY, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return SFB_ERR_CUDA;
+    if (CG == 2) {   // how many CTA pairs the device can hold at once
+      cudaLaunchConfig_t q;
+      memset(&q, 0, sizeof(q));
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+      q.gridDim = dim3(num_sms & ~1, 1, 1);
+      q.blockDim = dim3(NUM_THREADS, 1, 1);
+      q.dynamicSmemBytes = smem;
+      q.attrs = qa; q.numAttrs = 1;
+      if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &q) != cudaSuccess || max_clusters < 1) {
+        cudaGetLastError();
+        max_clusters = num_sms / 2;
+      }
+    }
     attr_done = true;
   }
   const int tiles = p.m_tiles * p.n_tiles;
-  const int grid = tiles < num_sms ? tiles : num_sms;
-  umma_gemm_kernel<ES, APPLY, BN><<<grid, NUM_THREADS, smem, s>>>(a, b, p);
+  if (CG == 1) {
+    const int grid = tiles < num_sms ? tiles : num_sms;
+    kernel<<<grid, NUM_THREADS, smem, s>>>(a, b, p);
+  } else {
+    const int clusters = tiles < max_clusters ? tiles : max_clusters;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(2 * clusters, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, a, b, p) != cudaSuccess) return SFB_ERR_CUDA;
+  }
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
+// cg = 2 (CTA pairs, 256-row tiles) only comes with 256-column tiles.
 template <bool APPLY>
-int dispatch_gemm(cudaStream_t s, int es, int bn, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p,
-                  int num_sms) {
-  if (es == 2) return bn == 256 ? launch_gemm<2, APPLY, 256>(s, a, b, p, num_sms) : launch_gemm<2, APPLY, 128>(s, a, b, p, num_sms);
-  return bn == 256 ? launch_gemm<4, APPLY, 256>(s, a, b, p, num_sms) : launch_gemm<4, APPLY, 128>(s, a, b, p, num_sms);
+int dispatch_gemm(cudaStream_t s, int es, int bn, int cg, const CUtensorMap& a, const CUtensorMap& b,
+                  const GemmParams& p, int num_sms) {
+  if (es == 2) {
+    if (bn == 256) return cg == 2 ? launch_gemm<2, APPLY, 256, 2>(s, a, b, p, num_sms) : launch_gemm<2, APPLY, 256, 1>(s, a, b, p, num_sms);
+    return launch_gemm<2, APPLY, 128, 1>(s, a, b, p, num_sms);
+  }
+  if (bn == 256) return cg == 2 ? launch_gemm<4, APPLY, 256, 2>(s, a, b, p, num_sms) : launch_gemm<4, APPLY, 256, 1>(s, a, b, p, num_sms);
+  return launch_gemm<4, APPLY, 128, 1>(s, a, b, p, num_sms);
 }
 
 }  // namespace
@@ -388,6 +464,7 @@ struct UmmaPlan {
   int ldz;
   int num_sms;
   int es;
+  bool pair_ok;   // CTA-pair kernels allowed (off with SFB_NO_CTA_PAIRS=1, for A/B measurements)
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -400,6 +477,8 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev);
+  const char* no_pairs = getenv("SFB_NO_CTA_PAIRS");
+  p->pair_ok = !(no_pairs != nullptr && no_pairs[0] == '1');
   *out = p;
   return SFB_OK;
 }
@@ -416,6 +495,10 @@ static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a,
   if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; p.m_tiles = d.P * p.m_tpw; }
   else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; p.m_tiles = (d.P + p.m_wp - 1) / p.m_wp; }
   const int bn = (d.J > 128 && (long long)p.m_tiles * ((d.J + 255) / 256) >= pl->num_sms) ? 256 : 128;
+  // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
+  const int cg = (bn == 256 && pl->pair_ok && (long long)((p.m_tiles + 1) / 2) * ((d.J + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
+  const int m_units = p.m_tiles;
+  p.m_tiles = (m_units + cg - 1) / cg;
   p.n_tiles = (d.J + bn - 1) / bn;
   p.k_blocks = (d.D + CH - 1) / CH;
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
@@ -427,9 +510,9 @@ static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a,
   CUtensorMap ta, tb;
   if (!encode_rows_map(&ta, es, a.base, d.D, d.B, d.P, (long long)a.ld * es, a.worker_stride, CH, p.m_bb, p.m_wp))
     return SFB_ERR_CUDA;
-  if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, CH, bn, 1))
+  if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, CH, bn / cg, 1))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<false>(s, es, bn, ta, tb, p, pl->num_sms);
+  return dispatch_gemm<false>(s, es, bn, cg, ta, tb, p, pl->num_sms);
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
@@ -476,8 +559,10 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
   p.B = d.B; p.P = workers;
   if (d.B >= BK) { p.k_bb = BK; p.k_wp = 1; p.k_bpw = (d.B + BK - 1) / BK; p.k_blocks = workers * p.k_bpw; }
   else { p.k_bb = pow2_at_least(d.B); p.k_wp = BK / p.k_bb; p.k_bpw = 1; p.k_blocks = (workers + p.k_wp - 1) / p.k_wp; }
-  p.m_tiles = (d.J + BM - 1) / BM;
-  const int bn = ((long long)p.m_tiles * ((d.D + 255) / 256) >= pl->num_sms) ? 256 : 128;
+  const int m_units = (d.J + BM - 1) / BM;
+  const int bn = ((long long)m_units * ((d.D + 255) / 256) >= pl->num_sms) ? 256 : 128;
+  const int cg = (bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((d.D + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
+  p.m_tiles = (m_units + cg - 1) / cg;
   p.n_tiles = (d.D + bn - 1) / bn;
   p.Mvalid = d.J; p.Nvalid = d.D;
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
@@ -498,7 +583,7 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
   if (!encode_rows_map(&tv, es, base + l.u_bytes, d.D, d.B, workers, (long long)l.ldv * es, l.stream_stride, CH, p.k_bb,
                        p.k_wp, es == 4))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<true>(s, es, bn, tu, tv, p, pl->num_sms);
+  return dispatch_gemm<true>(s, es, bn, cg, tu, tv, p, pl->num_sms);
 }
 
 }  // namespace sfb
