@@ -16,6 +16,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -30,7 +31,6 @@ int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v,
 namespace {
 
 constexpr int BM = 128;          // rows per CTA tile = TMEM lanes
-constexpr int A_STAGE_BYTES = BM * 128;   // A operand of one pipeline stage: 128 rows (or output indices) x 128 bytes
 constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
 constexpr int RING_BYTES = 192 * 1024;   // shared memory given to the operand ring
@@ -38,13 +38,13 @@ constexpr int MAX_STAGES = 8;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct GemmParams {
-  int m_tiles, n_tiles, k_blocks;   // m_tiles counts tiles of 128*CG rows
+  int m_tiles, n_tiles, k_blocks;   // m_tiles counts tiles of 128*CG rows; k_blocks counts blocks of BK reduction steps
   int a_policy, b_policy;   // L2 eviction policy of the operand loads (0 normal, 1 evict first, 2 evict last)
   int m_fastest;            // tile order: 1 = consecutive tiles share the B operand slab, 0 = share the A slab
-  int B, P;                 // rows per worker / workers, geometry of the 3-D operand maps
+  int B, P;                 // rows per worker / workers, geometry of the operand maps
   int m_bb, m_wp, m_tpw;    // forward: 128 A rows come as a box of m_bb rows x m_wp workers; 128-row units per worker
   int k_bb, k_wp, k_bpw;    // apply: a reduction block is k_bb rows x k_wp workers; blocks per worker
-  int Mvalid, Nvalid;       // forward: (unused, N = J) ; apply: (J, D)
+  int Mvalid, Nvalid;       // apply: (J, D)
   float* W;                 // apply: fp32 master, row stride ldw
   __nv_bfloat16* shadow;    // apply: bf16 copy of the new W (or nullptr)
   long long ldw;
@@ -70,26 +70,34 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sh
   return false;
 }
 
-// ES: bytes per operand value (2 = bf16, 4 = tf32).  APPLY: MN-major operands and the W write-back
-// epilogue; otherwise K-major operands and the plain fp32 store of Z.  BN: tile columns.
-// CG: CTAs per MMA.  With CG = 2 the kernel runs as clusters of two CTAs working on a 256 x BN tile:
-// each CTA loads its own 128 rows of A and its own half of B's columns, the even CTA issues
-// tcgen05.mma.cta_group::2 (M = 256) for the pair, each CTA drains its own 128 accumulator rows.
-// Signals of the pair: TMA bytes of both CTAs are credited to the even CTA's "full" barrier;
-// "stage free" and "accumulator ready" are committed (tcgen05.commit) once to the even CTA's barrier
-// and once to the odd CTA's; both CTAs' epilogues arrive on the even CTA's "accumulator drained"
-// barrier.
-template <int ES, bool APPLY, int BN, int CG>
+// Template parameters of the GEMM kernel:
+//   ES     bytes per operand value (2 = bf16, 4 = tf32); CH = 128 / ES values make one 128-byte chunk.
+//   APPLY  MN-major operands (factor rows) and the W write-back epilogue; otherwise K-major operands
+//          (sample rows / W rows) and a plain fp32 store of Z.
+//   BN     tile columns.
+//   CG     CTAs per MMA.  With CG = 2 the kernel runs as clusters of two CTAs on a 256 x BN tile: each
+//          CTA loads its own 128 rows of A and its own half of B's columns, the even CTA issues
+//          tcgen05.mma.cta_group::2 (M = 256) for the pair, each CTA drains its own 128 accumulator
+//          rows.  TMA bytes of both CTAs are credited to the even CTA's "full" barrier; "stage free"
+//          and "accumulator ready" are committed (tcgen05.commit) once to the even CTA's barrier and
+//          once to the odd CTA's; both epilogues arrive on the even CTA's "accumulator drained" barrier.
+//   KA     128-byte atoms of the reduction index per pipeline stage (BK = KA * CH reduction steps).
+//   FOLD   operands come through 4-D tensor maps whose extra dimension walks the 128-byte chunks, so
+//          one TMA instruction fills a whole operand stage (needs J, D multiples of CH); otherwise
+//          one 3-D TMA per chunk, with zero fill on every ragged edge.
+template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr int CH = 128 / ES;                 // values per 128-byte chunk
-  constexpr int BK = CH;                       // reduction steps per pipeline stage (64 bf16 / 32 tf32)
+  constexpr int BK = CH * KA;                  // reduction steps per pipeline stage
   constexpr int UMMA_K = 32 / ES;              // reduction steps per instruction (16 bf16 / 8 tf32)
   constexpr int BNC = BN / CG;                 // B columns this CTA loads
-  constexpr int B_STAGE_BYTES = BNC * 128;
+  constexpr int A_STAGE_BYTES = BM * 128 * KA;
+  constexpr int B_STAGE_BYTES = BNC * 128 * KA;
   constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
   constexpr int STAGES = (RING_BYTES / STAGE_BYTES) < MAX_STAGES ? (RING_BYTES / STAGE_BYTES) : MAX_STAGES;
   constexpr uint32_t IDESC = ptx::instr_desc(ES == 2 ? 1u : 2u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM * CG, BN);
+  static_assert(STAGES >= 2, "ring too shallow");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -98,6 +106,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (p.status_ro != nullptr && (*p.status_ro & SFB_DEV_BAD_HEADER)) return;   // uniform over the grid
+#ifdef SFB_EXP_CLOCKS
+  long long exp_c0 = clock64();
+  unsigned long long exp_t0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(exp_t0));
+#endif
 
   const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;   // 0 = the CTA that issues the MMAs
   const int cluster_id = blockIdx.x / CG, num_clusters = gridDim.x / CG;
@@ -134,47 +147,86 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int issued = 0;
     bool ok = true;
     const uint64_t pol_a = ptx::l2_policy(p.a_policy), pol_b = ptx::l2_policy(p.b_policy);
+#ifdef SFB_EXP_CLOCKS
+    long long exp_wait_empty = 0;
+#endif
     for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
       const int mt = (p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles) * CG + (int)rank;   // 128-row unit
       const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
       const int ncol0 = nt * BN + (int)rank * BNC;                                           // first B column loaded here
+      int slot0 = 0, mp0 = 0;          // forward: first slot / worker of this CTA's 128 sample rows
+      if (!APPLY) {
+        if (p.B >= BM) { mp0 = mt / p.m_tpw; slot0 = (mt % p.m_tpw) * BM; }
+        else { mp0 = mt * p.m_wp; }
+      }
+      int row0 = 0, kp0 = 0;           // apply: first row / worker of the current reduction block
       for (int kb = 0; kb < p.k_blocks; ++kb) {
+#ifdef SFB_EXP_CLOCKS
+        long long w0 = clock64();
+#endif
         ok = wait_or_abort(&ctl->empty[s], ph ^ 1u, ctl, p.status);
+#ifdef SFB_EXP_CLOCKS
+        exp_wait_empty += clock64() - w0;
+#endif
         if (!ok) break;
         if (lane == 0) {
           uint8_t* a_dst = tiles + s * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_STAGE_BYTES;
-          uint32_t full_addr = ptx::smem_u32(&ctl->full[s]);
-          if (CG == 2) {
-            full_addr = ptx::map_to_cta(full_addr, 0);
-          }
-          if (rank == 0) ptx::mbar_expect_tx(&ctl->full[s], CG * STAGE_BYTES);
+          uint64_t* bar = &ctl->full[s];
+          uint32_t full_addr = ptx::smem_u32(bar);
+          if (CG == 2) full_addr = ptx::map_to_cta(full_addr, 0);
+          if (rank == 0) ptx::mbar_expect_tx(bar, CG * STAGE_BYTES);
           if (!APPLY) {
-            const int k0 = kb * BK;
-            int slot0, p0;
-            if (p.B >= BM) { p0 = mt / p.m_tpw; slot0 = (mt % p.m_tpw) * BM; }
-            else { p0 = mt * p.m_wp; slot0 = 0; }
-            if (CG == 1) {
-              ptx::tma_load_3d_hint(a_dst, &tmA, &ctl->full[s], k0, slot0, p0, pol_a);
-              ptx::tma_load_3d_hint(b_dst, &tmB, &ctl->full[s], k0, ncol0, 0, pol_b);
+            if (FOLD) {   // dims (value-in-atom, row, worker, atom): one box = KA atoms of 128 rows
+              if (CG == 1) {
+                ptx::tma_load_4d_hint(a_dst, &tmA, bar, 0, slot0, mp0, kb * KA, pol_a);
+                ptx::tma_load_4d_hint(b_dst, &tmB, bar, 0, ncol0, 0, kb * KA, pol_b);
+              } else {
+                ptx::tma_load_4d_hint_pair(a_dst, &tmA, full_addr, 0, slot0, mp0, kb * KA, pol_a);
+                ptx::tma_load_4d_hint_pair(b_dst, &tmB, full_addr, 0, ncol0, 0, kb * KA, pol_b);
+              }
             } else {
-              ptx::tma_load_3d_hint_pair(a_dst, &tmA, full_addr, k0, slot0, p0, pol_a);
-              ptx::tma_load_3d_hint_pair(b_dst, &tmB, full_addr, k0, ncol0, 0, pol_b);
+#pragma unroll
+              for (int a = 0; a < KA; ++a) {
+                const int k0 = (kb * KA + a) * CH;
+                if (CG == 1) {
+                  ptx::tma_load_3d_hint(a_dst + a * (BM * 128), &tmA, bar, k0, slot0, mp0, pol_a);
+                  ptx::tma_load_3d_hint(b_dst + a * (BNC * 128), &tmB, bar, k0, ncol0, 0, pol_b);
+                } else {
+                  ptx::tma_load_3d_hint_pair(a_dst + a * (BM * 128), &tmA, full_addr, k0, slot0, mp0, pol_a);
+                  ptx::tma_load_3d_hint_pair(b_dst + a * (BNC * 128), &tmB, full_addr, k0, ncol0, 0, pol_b);
+                }
+              }
             }
           } else {
-            int row0, p0;
-            if (p.B >= BK) { p0 = kb / p.k_bpw; row0 = (kb % p.k_bpw) * BK; }
-            else { p0 = kb * p.k_wp; row0 = 0; }
+            if (FOLD) {   // dims (value-in-chunk, row, worker, chunk): one box = all chunks x BK rows
+              if (CG == 1) {
+                ptx::tma_load_4d_hint(a_dst, &tmA, bar, 0, row0, kp0, (mt * BM) / CH, pol_a);
+                ptx::tma_load_4d_hint(b_dst, &tmB, bar, 0, row0, kp0, ncol0 / CH, pol_b);
+              } else {
+                ptx::tma_load_4d_hint_pair(a_dst, &tmA, full_addr, 0, row0, kp0, (mt * BM) / CH, pol_a);
+                ptx::tma_load_4d_hint_pair(b_dst, &tmB, full_addr, 0, row0, kp0, ncol0 / CH, pol_b);
+              }
+            } else {
 #pragma unroll
-            for (int c = 0; c < BM / CH; ++c) {
-              if (CG == 1) ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, &ctl->full[s], mt * BM + c * CH, row0, p0, pol_a);
-              else ptx::tma_load_3d_hint_pair(a_dst + c * (BK * 128), &tmA, full_addr, mt * BM + c * CH, row0, p0, pol_a);
-            }
+              for (int c = 0; c < BM / CH; ++c) {
+                if (CG == 1) ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, bar, mt * BM + c * CH, row0, kp0, pol_a);
+                else ptx::tma_load_3d_hint_pair(a_dst + c * (BK * 128), &tmA, full_addr, mt * BM + c * CH, row0, kp0, pol_a);
+              }
 #pragma unroll
-            for (int c = 0; c < BNC / CH; ++c) {
-              if (CG == 1) ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, &ctl->full[s], ncol0 + c * CH, row0, p0, pol_b);
-              else ptx::tma_load_3d_hint_pair(b_dst + c * (BK * 128), &tmB, full_addr, ncol0 + c * CH, row0, p0, pol_b);
+              for (int c = 0; c < BNC / CH; ++c) {
+                if (CG == 1) ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, bar, ncol0 + c * CH, row0, kp0, pol_b);
+                else ptx::tma_load_3d_hint_pair(b_dst + c * (BK * 128), &tmB, full_addr, ncol0 + c * CH, row0, kp0, pol_b);
+              }
             }
+          }
+        }
+        if (APPLY) {   // next reduction block: next BK rows of this worker, or the next group of workers
+          if (p.B >= BK) {
+            row0 += BK;
+            if (row0 >= p.B) { row0 = 0; ++kp0; }
+          } else {
+            kp0 += p.k_wp;
           }
         }
         __syncwarp();
@@ -182,6 +234,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
+#ifdef SFB_EXP_CLOCKS
+    if (blockIdx.x == 0 && lane == 0) printf("EXPW apply=%d producer_wait_empty=%lld\n", (int)APPLY, exp_wait_empty);
+#endif
     if ((!ok || ctl->abort) && rank == 0) {
       // let copies already in flight land before the CTA goes away (bounded)
       int n = issued < STAGES ? issued : STAGES;
@@ -198,32 +253,64 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint32_t ph = 0;
     int it = 0;
     bool ok = (rank == 0);
+#ifdef SFB_EXP_CLOCKS
+    long long exp_wait_full = 0, exp_wait_tmem = 0;
+#endif
     for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++it) {
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
+#ifdef SFB_EXP_CLOCKS
+      long long w1 = clock64();
+#endif
       ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
+#ifdef SFB_EXP_CLOCKS
+      exp_wait_tmem += clock64() - w1;
+#endif
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * BN;
       for (int kb = 0; kb < p.k_blocks; ++kb) {
+#ifdef SFB_EXP_CLOCKS
+        long long w2 = clock64();
+#endif
         ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
+#ifdef SFB_EXP_CLOCKS
+        exp_wait_full += clock64() - w2;
+#endif
         if (!ok) break;
+#ifndef SFB_EXP_NO_KLOOP_FENCE
         ptx::tc_fence_after();
+#endif
         if (lane == 0) {
           const uint32_t a_addr = ptx::smem_u32(tiles + s * STAGE_BYTES);
           const uint32_t b_addr = a_addr + A_STAGE_BYTES;
-          // K-major: 8-row groups 1024 B apart.  MN-major: 8-step groups 1024 B apart, chunks BK*128 B apart.
-          // MN-major fp32 (tf32) operands use the 32-byte-atom swizzle: groups of 4 steps, 512 B apart.
-          constexpr bool MN32 = APPLY && ES == 4;
-          const uint64_t a_desc = ptx::smem_desc(a_addr, APPLY ? BK * 128 : 16, MN32 ? 512 : 1024, MN32 ? 1 : 2);
-          const uint64_t b_desc = ptx::smem_desc(b_addr, APPLY ? BK * 128 : 16, MN32 ? 512 : 1024, MN32 ? 1 : 2);
-          // per instruction: K-major advances 32 B inside the swizzled row, MN-major UMMA_K rows of 128 B
-          constexpr uint32_t STEP = (APPLY ? UMMA_K * 128 : 32) >> 4;
+          if (!APPLY) {
+            // K-major: a stage is KA atoms, each [rows][128 B] with 8-row groups 1024 B apart; inside an
+            // atom the instruction's 32 bytes of reduction index advance the start address.
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-            if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
-            else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+            for (int a = 0; a < KA; ++a) {
+              const uint64_t a_desc = ptx::smem_desc(a_addr + a * (BM * 128), 16, 1024, 2);
+              const uint64_t b_desc = ptx::smem_desc(b_addr + a * (BNC * 128), 16, 1024, 2);
+#pragma unroll
+              for (int k = 0; k < CH / UMMA_K; ++k) {
+                const uint32_t acc = (kb > 0 || a > 0 || k > 0) ? 1u : 0u;
+                if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
+                else ptx::mma_tf32<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
+              }
+            }
+          } else {
+            // MN-major: a stage is chunks of [BK reduction steps][128 B], BK*128 B apart; groups of 8
+            // steps are 1024 B apart (32-bit values: 32-byte-atom swizzle, groups of 4 steps, 512 B).
+            constexpr bool MN32 = ES == 4;
+            const uint64_t a_desc = ptx::smem_desc(a_addr, BK * 128, MN32 ? 512 : 1024, MN32 ? 1 : 2);
+            const uint64_t b_desc = ptx::smem_desc(b_addr, BK * 128, MN32 ? 512 : 1024, MN32 ? 1 : 2);
+            constexpr uint32_t STEP = (UMMA_K * 128) >> 4;
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+              if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+              else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+            }
           }
           ptx::mma_commit<CG>(&ctl->empty[s]);                     // stage reusable once these MMAs have read it
           if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->empty[s]), 1));
@@ -236,6 +323,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
+#ifdef SFB_EXP_CLOCKS
+    if (blockIdx.x == 0 && lane == 0)
+      printf("EXPW apply=%d mma_wait_full=%lld mma_wait_tmem_empty=%lld\n", (int)APPLY, exp_wait_full, exp_wait_tmem);
+#endif
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9, every CTA)
     // A warp may only read the TMEM lanes of its quarter (warp index mod 4).  Two warps share each
@@ -277,7 +368,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       float4 wv[8];
 #pragma unroll
       for (int g = 0; g < 8; ++g) wv[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+#ifdef SFB_EXP_SKIP_EPILOGUE_LOADS
+      if (APPLY && p.eta == 123.456f) {
+#else
       if (APPLY) {
+#endif
 #pragma unroll
         for (int g = 0; g < 8; ++g)
           if (rowp[g] != nullptr && cbase < ncols) wv[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + cbase));
@@ -302,7 +397,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float4 wn[8];   // next block of W, in flight while this block is combined and stored
 #pragma unroll
         for (int g = 0; g < 8; ++g) wn[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+#ifdef SFB_EXP_SKIP_EPILOGUE_LOADS
+        if (APPLY && cc + 1 < BN / 64 && p.eta == 123.456f) {
+#else
         if (APPLY && cc + 1 < BN / 64) {
+#endif
 #pragma unroll
           for (int g = 0; g < 8; ++g)
             if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
@@ -317,7 +416,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int g = 0; g < 8; ++g) {
           const int lr = 4 * g + lrow;
           const float4 a = *reinterpret_cast<const float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2));
+#ifdef SFB_EXP_SKIP_EPILOGUE_STORES
+          if (a.x == 123.456f && rowp[g] != nullptr && c < ncols) {
+#else
           if (rowp[g] != nullptr && c < ncols) {
+#endif
             if (APPLY) {
               float4 w = wv[g];
               w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
@@ -348,6 +451,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   }
 
+#ifdef SFB_EXP_CLOCKS
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    unsigned long long exp_t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(exp_t1));
+    printf("EXPCLK apply=%d cycles=%lld ns=%llu MHz=%.0f\n", (int)APPLY, clock64() - exp_c0, exp_t1 - exp_t0,
+           1e3 * (double)(clock64() - exp_c0) / (double)(exp_t1 - exp_t0));
+  }
+#endif
   ptx::tc_fence_before();
   __syncthreads();
   if (CG == 2) ptx::cluster_sync();   // nobody leaves while its pair may still signal it or read its tiles
@@ -370,21 +481,34 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
   return fn;
 }
 
-// 3-D map over factor-like rows: dim0 = cols values (contiguous), dim1 = rows per worker, dim2 = workers.
+// Tensor map over factor-like rows (row r of worker w at base + w * worker_stride + r * row_stride).
+//   fold == false: 3-D (value, row, worker); box = {CH values, box_rows, box_workers}.
+//   fold == true : 4-D (value within a 128-byte chunk, row, worker, chunk) with the chunk dimension
+//                  striding 128 bytes along the row; box = {CH, box_rows, box_workers, box_chunks}.
+//                  `cols` must be a multiple of CH (a chunk never straddles the end of a row).
 bool encode_rows_map(CUtensorMap* m, int es, const void* base, long long cols, long long rows, long long workers,
-                     long long row_stride_bytes, long long worker_stride_bytes, int box0, int box1, int box2,
-                     bool atom32 = false) {
+                     long long row_stride_bytes, long long worker_stride_bytes, int box_rows, int box_workers,
+                     bool fold, int box_chunks, bool atom32) {
   auto fn = get_encode();
   if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)workers};
-  cuuint64_t strides[2] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)worker_stride_bytes};
-  cuuint32_t box[3] = {(cuuint32_t)box0, (cuuint32_t)box1, (cuuint32_t)box2};
-  cuuint32_t estr[3] = {1, 1, 1};
+  const int CH = 128 / es;
   const CUtensorMapDataType dt = es == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-  const CUresult r = fn(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const CUtensorMapSwizzle sw = atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r;
+  if (!fold) {
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)workers};
+    cuuint64_t strides[2] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)worker_stride_bytes};
+    cuuint32_t box[3] = {(cuuint32_t)CH, (cuuint32_t)box_rows, (cuuint32_t)box_workers};
+    r = fn(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[4] = {(cuuint64_t)CH, (cuuint64_t)rows, (cuuint64_t)workers, (cuuint64_t)(cols / CH)};
+    cuuint64_t strides[3] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)worker_stride_bytes, 128};
+    cuuint32_t box[4] = {(cuuint32_t)CH, (cuuint32_t)box_rows, (cuuint32_t)box_workers, (cuuint32_t)box_chunks};
+    r = fn(m, dt, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   return r == CUDA_SUCCESS;
 }
 
@@ -394,12 +518,12 @@ int pow2_at_least(int n) {
   return p;
 }
 
-template <int ES, bool APPLY, int BN, int CG>
+template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD>
 int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, int num_sms) {
-  constexpr int stage_bytes = A_STAGE_BYTES + (BN / CG) * 128;
+  constexpr int stage_bytes = (BM + BN / CG) * 128 * KA;
   constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
   constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
-  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG>;
+  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD>;
   static bool attr_done = false;
   static int max_clusters = 0;
   if (!attr_done) {
@@ -443,16 +567,29 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
-// cg = 2 (CTA pairs, 256-row tiles) only comes with 256-column tiles.
-template <bool APPLY>
-int dispatch_gemm(cudaStream_t s, int es, int bn, int cg, const CUtensorMap& a, const CUtensorMap& b,
-                  const GemmParams& p, int num_sms) {
-  if (es == 2) {
-    if (bn == 256) return cg == 2 ? launch_gemm<2, APPLY, 256, 2>(s, a, b, p, num_sms) : launch_gemm<2, APPLY, 256, 1>(s, a, b, p, num_sms);
-    return launch_gemm<2, APPLY, 128, 1>(s, a, b, p, num_sms);
+// Kernel variants: "big" = CTA pairs on 256 x 256 tiles; with J, D multiples of the chunk it also folds
+// the operand loads (one TMA per operand per stage) and doubles the reduction depth of a stage.
+struct Variant {
+  int bn, cg, ka;
+  bool fold;
+};
+
+template <int ES, bool APPLY>
+int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p,
+                int num_sms) {
+  if (v.cg == 2) {
+    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true>(s, a, b, p, num_sms);
+    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true>(s, a, b, p, num_sms);
+    return launch_gemm<ES, APPLY, 256, 2, 1, false>(s, a, b, p, num_sms);
   }
-  if (bn == 256) return cg == 2 ? launch_gemm<4, APPLY, 256, 2>(s, a, b, p, num_sms) : launch_gemm<4, APPLY, 256, 1>(s, a, b, p, num_sms);
-  return launch_gemm<4, APPLY, 128, 1>(s, a, b, p, num_sms);
+  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false>(s, a, b, p, num_sms);
+  return launch_gemm<ES, APPLY, 128, 1, 1, false>(s, a, b, p, num_sms);
+}
+
+template <bool APPLY>
+int dispatch_gemm(cudaStream_t s, int es, const Variant& v, const CUtensorMap& a, const CUtensorMap& b,
+                  const GemmParams& p, int num_sms) {
+  return es == 2 ? dispatch_es<2, APPLY>(s, v, a, b, p, num_sms) : dispatch_es<4, APPLY>(s, v, a, b, p, num_sms);
 }
 
 }  // namespace
@@ -465,6 +602,8 @@ struct UmmaPlan {
   int num_sms;
   int es;
   bool pair_ok;   // CTA-pair kernels allowed (off with SFB_NO_CTA_PAIRS=1, for A/B measurements)
+  bool fold_ok;   // folded operand loads allowed (off with SFB_NO_FOLD=1)
+  int fold_ka;    // 128-byte atoms of the reduction index per stage in the folded kernels (SFB_FOLD_KA, default 2)
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -479,11 +618,26 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev);
   const char* no_pairs = getenv("SFB_NO_CTA_PAIRS");
   p->pair_ok = !(no_pairs != nullptr && no_pairs[0] == '1');
+  const char* no_fold = getenv("SFB_NO_FOLD");
+  p->fold_ok = !(no_fold != nullptr && no_fold[0] == '1');
+  const char* ka = getenv("SFB_FOLD_KA");
+  p->fold_ka = (ka != nullptr && ka[0] == '1') ? 1 : 2;
   *out = p;
   return SFB_OK;
 }
 
 void umma_plan_destroy(UmmaPlan* p) { delete p; }
+
+// Tile shape and kernel variant for an M x N output (M counted in 128-row units).
+static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_chunk_aligned) {
+  Variant v;
+  v.bn = (N > 128 && (long long)m_units * ((N + 255) / 256) >= pl->num_sms) ? 256 : 128;
+  // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
+  v.cg = (v.bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
+  v.fold = v.cg == 2 && pl->fold_ok && dims_chunk_aligned;
+  v.ka = v.fold ? pl->fold_ka : 1;
+  return v;
+}
 
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
 static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status) {
@@ -492,15 +646,14 @@ static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a,
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.B = d.B; p.P = d.P;
-  if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; p.m_tiles = d.P * p.m_tpw; }
-  else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; p.m_tiles = (d.P + p.m_wp - 1) / p.m_wp; }
-  const int bn = (d.J > 128 && (long long)p.m_tiles * ((d.J + 255) / 256) >= pl->num_sms) ? 256 : 128;
-  // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
-  const int cg = (bn == 256 && pl->pair_ok && (long long)((p.m_tiles + 1) / 2) * ((d.J + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
-  const int m_units = p.m_tiles;
-  p.m_tiles = (m_units + cg - 1) / cg;
-  p.n_tiles = (d.J + bn - 1) / bn;
-  p.k_blocks = (d.D + CH - 1) / CH;
+  int m_units;
+  if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; m_units = d.P * p.m_tpw; }
+  else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; m_units = (d.P + p.m_wp - 1) / p.m_wp; }
+  // folding walks the reduction index (D) in 128-byte atoms: rows must be whole atoms long
+  const Variant v = pick_variant(pl, m_units, d.J, (d.D % CH) == 0 && (a.ld % CH) == 0);
+  p.m_tiles = (m_units + v.cg - 1) / v.cg;
+  p.n_tiles = (d.J + v.bn - 1) / v.bn;
+  p.k_blocks = (d.D + CH * v.ka - 1) / (CH * v.ka);
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
   p.m_fastest = ((long long)d.J * d.D > (long long)d.P * d.B * d.D) ? 1 : 0;
   p.a_policy = p.m_fastest ? 2 : 0;   // the operand whose slab changes every tile is re-read all along: keep it
@@ -508,11 +661,13 @@ static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a,
   p.z = z;
   p.status = dev_status;
   CUtensorMap ta, tb;
-  if (!encode_rows_map(&ta, es, a.base, d.D, d.B, d.P, (long long)a.ld * es, a.worker_stride, CH, p.m_bb, p.m_wp))
+  if (!encode_rows_map(&ta, es, a.base, d.D, d.B, d.P, (long long)a.ld * es, a.worker_stride, p.m_bb, p.m_wp, v.fold,
+                       v.ka, false))
     return SFB_ERR_CUDA;
-  if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, CH, bn / cg, 1))
+  if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, v.bn / v.cg, 1,
+                       v.fold, v.ka, false))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<false>(s, es, bn, cg, ta, tb, p, pl->num_sms);
+  return dispatch_gemm<false>(s, es, v, ta, tb, p, pl->num_sms);
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
@@ -552,18 +707,19 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
                const int* dev_status) {
   const sfb_desc& d = pl->d;
   const Layout& l = pl->l;
-  const int es = pl->es, CH = 128 / es, BK = CH;
+  const int es = pl->es, CH = 128 / es;
   const int workers = K / d.B;
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.B = d.B; p.P = workers;
+  const int m_units = (d.J + BM - 1) / BM;
+  // folding walks the output indices (J for u, D for v) in 128-byte chunks
+  const Variant v = pick_variant(pl, m_units, d.D, (d.J % CH) == 0 && (d.D % CH) == 0);
+  const int BK = CH * v.ka;
   if (d.B >= BK) { p.k_bb = BK; p.k_wp = 1; p.k_bpw = (d.B + BK - 1) / BK; p.k_blocks = workers * p.k_bpw; }
   else { p.k_bb = pow2_at_least(d.B); p.k_wp = BK / p.k_bb; p.k_bpw = 1; p.k_blocks = (workers + p.k_wp - 1) / p.k_wp; }
-  const int m_units = (d.J + BM - 1) / BM;
-  const int bn = ((long long)m_units * ((d.D + 255) / 256) >= pl->num_sms) ? 256 : 128;
-  const int cg = (bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((d.D + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
-  p.m_tiles = (m_units + cg - 1) / cg;
-  p.n_tiles = (d.D + bn - 1) / bn;
+  p.m_tiles = (m_units + v.cg - 1) / v.cg;
+  p.n_tiles = (d.D + v.bn - 1) / v.bn;
   p.Mvalid = d.J; p.Nvalid = d.D;
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
   p.a_policy = p.m_fastest ? 2 : 0;
@@ -577,13 +733,13 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
   const char* base = reinterpret_cast<const char*>(sf_buf) + l.streams_off;
   CUtensorMap tu, tv;
   // only the first `workers` streams are visible to the maps, so zero fill covers a ragged last block
-  if (!encode_rows_map(&tu, es, base, d.J, d.B, workers, (long long)l.ldu * es, l.stream_stride, CH, p.k_bb, p.k_wp,
-                       es == 4))
+  if (!encode_rows_map(&tu, es, base, d.J, d.B, workers, (long long)l.ldu * es, l.stream_stride, p.k_bb, p.k_wp, v.fold,
+                       BM / CH, es == 4))
     return SFB_ERR_CUDA;
-  if (!encode_rows_map(&tv, es, base + l.u_bytes, d.D, d.B, workers, (long long)l.ldv * es, l.stream_stride, CH, p.k_bb,
-                       p.k_wp, es == 4))
+  if (!encode_rows_map(&tv, es, base + l.u_bytes, d.D, d.B, workers, (long long)l.ldv * es, l.stream_stride, p.k_bb,
+                       p.k_wp, v.fold, (v.bn / v.cg) / CH, es == 4))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<true>(s, es, bn, cg, tu, tv, p, pl->num_sms);
+  return dispatch_gemm<true>(s, es, v, tu, tv, p, pl->num_sms);
 }
 
 }  // namespace sfb

@@ -78,6 +78,23 @@ __device__ __forceinline__ void tma_load_3d_hint(void* dst, const CUtensorMap* m
         "l"(policy) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d_hint(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1, int c2,
+                                                 int c3, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
+        "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_hint_pair(void* dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int c0,
+                                                      int c1, int c2, int c3, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2),
+        "r"(c3), "l"(policy) : "memory");
+}
+
 // The pair form: both CTAs of the pair run it, the bytes are credited to a barrier of the even CTA
 // (`bar_cluster_addr` is that barrier's address in the cluster's shared window).
 __device__ __forceinline__ void tma_load_3d_hint_pair(void* dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int c0,
