@@ -5,9 +5,10 @@
 //
 // W is J x D row-major, so an atom (column d) is strided in memory.  The forward therefore works on
 // an atom-major copy W^T (one coalesced J-vector per nonzero), rebuilt from W by a tiled transpose.
-// The apply gives every thread block a slab of 8 consecutive atoms (32-byte sectors of every row of
-// W) held in shared memory; the block walks all samples in order, finds each sample's nonzeros
-// inside its slab by binary search in the sorted CSR row, and applies them in (sample, atom) order.
+// The apply gives every thread block a slab of 16 consecutive atoms (64 bytes of each of 1024 rows of
+// W) held in shared memory; the block walks all samples in order, finds each sample's
+// nonzeros inside its slab by binary search in the sorted CSR row, and applies them in (sample, atom)
+// order.
 // No floating-point atomics: every element of W is owned by one block and updated in a fixed order,
 // so the result is bit-reproducible; atoms no code uses are written back unchanged.
 #include "common.cuh"
@@ -108,33 +109,44 @@ __global__ void __launch_bounds__(256) sc_forward_kernel(const float* __restrict
   }
 }
 
-constexpr int SLAB_D = 8;        // atoms per block: one 32-byte sector of every row of W
-constexpr int SLAB_CHUNK = 256;  // samples searched per round (one per thread)
+constexpr int SLAB_D = 16;         // atoms per block: two 32-byte sectors of every row of W
+constexpr int SLAB_T = 256;        // threads per block
+constexpr int SLAB_J = 4 * SLAB_T; // rows of W per block: four consecutive rows per thread
+constexpr int SLAB_CAP = 1024;     // entries applied per pass (more are handled by further passes)
+constexpr int SLAB_BATCH = 8;      // entries whose u values are fetched together
 
-// grid = (ceil(D / 8), ceil(J / JT)); dynamic shared memory: 8 * JT floats.
-__global__ void __launch_bounds__(256) sc_apply_kernel(float* __restrict__ W, CsrView codes, RowMap u, int K, int J,
-                                                       int D, int JT, float eta, const int* __restrict__ status_ro) {
-  extern __shared__ __align__(16) float Ws[];   // [SLAB_D][JT]
-  __shared__ int s_scan[256];
-  __shared__ int s_ent_i[SLAB_CHUNK * SLAB_D];
-  __shared__ int s_ent_d[SLAB_CHUNK * SLAB_D];
-  __shared__ float s_ent_a[SLAB_CHUNK * SLAB_D];
+// grid = (ceil(D / 16), ceil(J / 1024)); the block owns the 16-atom x 1024-row slab of W in shared memory.
+// Per round of 256 samples: every thread finds the entries of one sample's sorted CSR row that fall
+// inside the slab (binary search + short scan), a block-wide scan orders them by (sample, atom), and
+// the entries are applied in that order: thread t adds -eta * a * u_i[j] to its own four rows j of
+// the slab, with the u values of 8 entries fetched ahead as independent 16-byte loads.
+// A thread owns its rows for the whole kernel, so there is no race and the summation order is fixed.
+__global__ void __launch_bounds__(SLAB_T) sc_apply_kernel(float* __restrict__ W, CsrView codes, RowMap u, int K, int J,
+                                                          int D, float eta, const int* __restrict__ status_ro) {
+  extern __shared__ __align__(16) float Ws[];   // 64 KB: Ws[atom * SLAB_J + row]
+  __shared__ int s_key[SLAB_CAP];               // sample * 16 + atom-in-slab
+  __shared__ float s_val[SLAB_CAP];             // -eta * code value
+  __shared__ int s_warp[SLAB_T / 32];
   if (status_ro != nullptr && (*status_ro & SFB_DEV_BAD_HEADER)) return;
   const int t = threadIdx.x;
-  const int d0 = blockIdx.x * SLAB_D, j0 = blockIdx.y * JT;
+  const int d0 = blockIdx.x * SLAB_D, j0 = blockIdx.y * SLAB_J;
   const int dn = min(SLAB_D, D - d0);
-  const int jn = min(JT, J - j0);
+  const int jn = min(SLAB_J, J - j0);
   const bool vec_ok = ((D & 3) == 0) && (dn == SLAB_D);
 
-  for (int jj = t; jj < JT; jj += 256) {
+  // slab in: thread handles whole rows (16 atoms = 64 bytes), transposed into Ws[atom][row]
+  for (int jj = t; jj < SLAB_J; jj += SLAB_T) {
     float w[SLAB_D];
 #pragma unroll
     for (int e = 0; e < SLAB_D; ++e) w[e] = 0.f;
     if (jj < jn) {
       const float* src = W + (size_t)(j0 + jj) * D + d0;
       if (vec_ok) {
-        const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
-        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+#pragma unroll
+        for (int q = 0; q < SLAB_D / 4; ++q) {
+          const float4 v = *reinterpret_cast<const float4*>(src + 4 * q);
+          w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+        }
       } else {
 #pragma unroll
         for (int e = 0; e < SLAB_D; ++e)
@@ -142,12 +154,14 @@ __global__ void __launch_bounds__(256) sc_apply_kernel(float* __restrict__ W, Cs
       }
     }
 #pragma unroll
-    for (int e = 0; e < SLAB_D; ++e) Ws[e * JT + jj] = w[e];
+    for (int e = 0; e < SLAB_D; ++e) Ws[e * SLAB_J + jj] = w[e];
   }
   __syncthreads();
 
-  for (int c0 = 0; c0 < K; c0 += SLAB_CHUNK) {
-    // (1) every thread searches one sample's sorted row for entries inside [d0, d0 + dn)
+  const int jt = 4 * t;                      // this thread's first row inside the slab
+  const bool row_ok = jt < jn;               // J is padded to 4 in U rows, so a float4 never leaves the row
+  for (int c0 = 0; c0 < K; c0 += SLAB_T) {
+    // (1) this thread's sample: entries of its sorted row inside [d0, d0 + dn)
     const int i = c0 + t;
     int lo = 0, cnt = 0;
     CsrRow row;
@@ -168,52 +182,72 @@ __global__ void __launch_bounds__(256) sc_apply_kernel(float* __restrict__ W, Cs
       const int n = __shfl_up_sync(0xffffffffu, incl, o);
       if ((t & 31) >= o) incl += n;
     }
-    if ((t & 31) == 31) s_scan[t >> 5] = incl;
+    if ((t & 31) == 31) s_warp[t >> 5] = incl;
     __syncthreads();
-    if (t < 8) {
-      int v = s_scan[t];
+    if (t < 32) {
+      int v = (t < SLAB_T / 32) ? s_warp[t] : 0;
 #pragma unroll
-      for (int o = 1; o < 8; o <<= 1) {
-        const int n = __shfl_up_sync(0xffu, v, o);
+      for (int o = 1; o < SLAB_T / 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, v, o);
         if (t >= o) v += n;
       }
-      s_scan[t] = v;
+      if (t < SLAB_T / 32) s_warp[t] = v;
     }
     __syncthreads();
-    const int base = incl - cnt + ((t >> 5) > 0 ? s_scan[(t >> 5) - 1] : 0);
-    const int total = s_scan[7];
-    for (int e = 0; e < cnt; ++e) {
-      s_ent_i[base + e] = i;
-      s_ent_d[base + e] = (int)row.idx[lo + e] - d0;
-      s_ent_a[base + e] = row.val[lo + e];
-    }
+    const int base = incl - cnt + ((t >> 5) > 0 ? s_warp[(t >> 5) - 1] : 0);
+    const int total = s_warp[SLAB_T / 32 - 1];
     __syncthreads();
-    // (3) apply the entries in (sample, atom) order; each thread owns fixed rows j of the slab
-    for (int e = 0; e < total; ++e) {
-      const float ca = -eta * s_ent_a[e];
-      const float* ur = reinterpret_cast<const float*>(u.row(s_ent_i[e])) + j0;
-      float* ws = Ws + s_ent_d[e] * JT;
-      for (int jj = t * 4; jj < jn; jj += 1024) {
-        if (jj + 3 < jn) {
-          const float4 uv = *reinterpret_cast<const float4*>(ur + jj);
-          float4 w = *reinterpret_cast<float4*>(ws + jj);
-          w.x = fmaf(ca, uv.x, w.x); w.y = fmaf(ca, uv.y, w.y); w.z = fmaf(ca, uv.z, w.z); w.w = fmaf(ca, uv.w, w.w);
-          *reinterpret_cast<float4*>(ws + jj) = w;
-        } else {
-          for (int b = 0; b < 4 && jj + b < jn; ++b) ws[jj + b] = fmaf(ca, ur[jj + b], ws[jj + b]);
+    // (3) apply, SLAB_CAP entries per pass, in (sample, atom) order
+    for (int win = 0; win < total; win += SLAB_CAP) {
+      for (int e = 0; e < cnt; ++e) {
+        const int pos = base + e - win;
+        if (pos >= 0 && pos < SLAB_CAP) {
+          s_key[pos] = i * SLAB_D + ((int)row.idx[lo + e] - d0);
+          s_val[pos] = -eta * row.val[lo + e];
         }
       }
+      __syncthreads();
+      const int n = min(SLAB_CAP, total - win);
+      if (row_ok) {
+        const char* ucol = u.base + (size_t)(j0 + jt) * 4;   // this thread's four columns of U
+        for (int e0 = 0; e0 < n; e0 += SLAB_BATCH) {
+          float4 uv[SLAB_BATCH];
+#pragma unroll
+          for (int q = 0; q < SLAB_BATCH; ++q) {   // independent loads first; repeats of one sample hit L1
+            uv[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (e0 + q < n) {
+              const int smp = s_key[e0 + q] / SLAB_D;
+              uv[q] = __ldg(reinterpret_cast<const float4*>(ucol + (long long)(smp / u.B) * u.worker_stride +
+                                                            (long long)(smp % u.B) * u.ld * 4));
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < SLAB_BATCH; ++q) {
+            if (e0 + q < n) {
+              const float ca = s_val[e0 + q];
+              float4* ws = reinterpret_cast<float4*>(Ws + (s_key[e0 + q] % SLAB_D) * SLAB_J + jt);
+              float4 w = *ws;
+              w.x = fmaf(ca, uv[q].x, w.x); w.y = fmaf(ca, uv[q].y, w.y);
+              w.z = fmaf(ca, uv[q].z, w.z); w.w = fmaf(ca, uv[q].w, w.w);
+              *ws = w;
+            }
+          }
+        }
+      }
+      __syncthreads();
     }
-    __syncthreads();
   }
 
-  for (int jj = t; jj < jn; jj += 256) {
+  for (int jj = t; jj < jn; jj += SLAB_T) {
     float* dst = W + (size_t)(j0 + jj) * D + d0;
     if (vec_ok) {
-      *reinterpret_cast<float4*>(dst) = make_float4(Ws[jj], Ws[JT + jj], Ws[2 * JT + jj], Ws[3 * JT + jj]);
-      *reinterpret_cast<float4*>(dst + 4) = make_float4(Ws[4 * JT + jj], Ws[5 * JT + jj], Ws[6 * JT + jj], Ws[7 * JT + jj]);
+#pragma unroll
+      for (int q = 0; q < SLAB_D / 4; ++q)
+        *reinterpret_cast<float4*>(dst + 4 * q) =
+            make_float4(Ws[(4 * q) * SLAB_J + jj], Ws[(4 * q + 1) * SLAB_J + jj], Ws[(4 * q + 2) * SLAB_J + jj],
+                        Ws[(4 * q + 3) * SLAB_J + jj]);
     } else {
-      for (int e = 0; e < dn; ++e) dst[e] = Ws[e * JT + jj];
+      for (int e = 0; e < dn; ++e) dst[e] = Ws[e * SLAB_J + jj];
     }
   }
 }
@@ -235,15 +269,14 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
 
 int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                     const int* dev_status_ro, int* /*dev_status*/) {
-  const int JT = (int)pad_to(J < 4096 ? J : 4096, 4);
-  const size_t smem = (size_t)SLAB_D * JT * sizeof(float);
   static bool attr_done = false;
   if (!attr_done) {
-    cudaFuncSetAttribute(sc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SLAB_D * 4096 * 4);
+    cudaFuncSetAttribute(sc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SLAB_D * SLAB_J * 4);
+    cudaFuncSetAttribute(sc_apply_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     attr_done = true;
   }
-  dim3 grid((D + SLAB_D - 1) / SLAB_D, (J + JT - 1) / JT);
-  sc_apply_kernel<<<grid, 256, smem, s>>>(W, codes, u, K, J, D, JT, eta, dev_status_ro);
+  dim3 grid((D + SLAB_D - 1) / SLAB_D, (J + SLAB_J - 1) / SLAB_J);
+  sc_apply_kernel<<<grid, SLAB_T, SLAB_D * SLAB_J * 4, s>>>(W, codes, u, K, J, D, eta, dev_status_ro);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
