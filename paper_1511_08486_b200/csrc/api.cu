@@ -17,7 +17,8 @@ struct sfb_ctx {
   int* dev_status;          // sticky device status word
   float* z_ws;              // fp32 products z = W a, [K][ldz], when u is stored in another type (bf16 path)
   int ldz;
-  float* wt_ws;             // SC: atom-major copy of W for the forward
+  float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
+  float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
   __nv_bfloat16* w_shadow;  // bf16 path: bf16 copy of W, refreshed by the apply
   const void* shadow_of;    // W pointer the shadow currently mirrors (nullptr = stale)
   UmmaPlan* umma;           // tensor-core plan (tensor maps), TF32 / BF16 paths
@@ -40,7 +41,7 @@ int check_desc(const sfb_desc* d) {
   if ((long long)d->P * d->B > (1 << 24)) return SFB_ERR_SHAPE;
   if (d->model == SFB_SC) {
     if (!d->v_sparse) return SFB_ERR_UNSUPPORTED;          // dictionary updates take CSR codes
-    if (d->path != SFB_PATH_F32) return SFB_ERR_UNSUPPORTED;
+    if (d->path == SFB_PATH_BF16) return SFB_ERR_UNSUPPORTED;   // fp32 sparse path, or dense tf32 on tensor cores
     if (d->nnz_capacity == 0 || d->nnz_capacity % (32ull * d->P) != 0) return SFB_ERR_SHAPE;
     if (d->nnz_capacity / d->P > (1ull << 30)) return SFB_ERR_SHAPE;
   } else if (d->v_sparse) {
@@ -73,6 +74,7 @@ RowMap stream_v(const sfb_ctx* c, const void* sf_buf) {
   m.ld = c->l.ldv;
   return m;
 }
+RowMap dense_codes(const sfb_ctx* c) { return caller_rows(c->a_dense, c->l.ldv, c->d.B, 4); }
 RowMap z_rows(const sfb_ctx* c) { return caller_rows(c->z_ws, c->ldz, c->d.B, 4); }
 
 CsrView global_codes(const sfb_aux* a, int B) {
@@ -120,9 +122,16 @@ int ensure_shadow(sfb_ctx* c, const void* W) {
 int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, RowMap u, RowMap v, CsrView codes) {
   const sfb_desc& d = c->d;
   const float* Wf = reinterpret_cast<const float*>(W);
-  if (d.model == SFB_SC) {
+  if (d.model == SFB_SC && d.path == SFB_PATH_F32) {
     ACC(launch_sc_forward_ws(c->stream, Wf, c->wt_ws, codes, reinterpret_cast<const float*>(aux->Xdata), u, c->K, d.J,
                              d.D, c->dev_status));
+    return SFB_OK;
+  }
+  if (d.model == SFB_SC) {   // dense alternative: the codes as dense tf32 rows through the tensor-core GEMM
+    const RowMap a = dense_codes(c);
+    ACC(launch_densify_codes(c->stream, codes, a, c->K, d.D, c->dev_status));
+    ACC(umma_forward_rows(c->umma, c->stream, W, a, u, c->dev_status));
+    ACC(launch_finish_sc(c->stream, u, reinterpret_cast<const float*>(aux->Xdata), c->K, d.J));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {
@@ -190,7 +199,10 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
   c->K = desc->P * desc->B;
   bool ok = cudaMalloc(&c->dev_status, 256) == cudaSuccess;
   if (ok) ok = cudaMemsetAsync(c->dev_status, 0, 256, c->stream) == cudaSuccess;
-  if (ok && desc->model == SFB_SC) ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
+  if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_F32)
+    ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
+  if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_TF32)
+    ok = cudaMalloc(&c->a_dense, (size_t)c->K * c->l.ldv * 4) == cudaSuccess;
   if (ok && desc->path == SFB_PATH_BF16) {
     c->ldz = (int)pad_to(desc->J, 4);
     ok = cudaMalloc(&c->z_ws, (size_t)c->K * c->ldz * 4) == cudaSuccess;
@@ -222,6 +234,7 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->dev_status) cudaFree(c->dev_status);
   if (c->z_ws) cudaFree(c->z_ws);
   if (c->wt_ws) cudaFree(c->wt_ws);
+  if (c->a_dense) cudaFree(c->a_dense);
   if (c->w_shadow) cudaFree(c->w_shadow);
   delete c;
   return SFB_OK;
@@ -310,14 +323,18 @@ int sfb_pack(sfb_ctx* c, const void* U, const void* V, const sfb_aux* aux, void*
 static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check) {
   const sfb_desc& d = c->d;
   if (check) ACC(launch_check_header(c->stream, sf_buf, d, c->l, c->dev_status));
-  if (d.v_sparse) {
+  if (d.v_sparse && d.path == SFB_PATH_F32) {
     ACC(launch_sc_apply(c->stream, reinterpret_cast<float*>(W), stream_codes(c, sf_buf), stream_u(c, sf_buf), K, d.J,
                         d.D, eta, c->dev_status, c->dev_status));
+  } else if (d.v_sparse) {
+    // dense alternative: rebuild the dense code rows from the buffer's CSR streams unless this step just made them
+    if (check) ACC(launch_densify_codes(c->stream, stream_codes(c, sf_buf), dense_codes(c), K, d.D, c->dev_status));
+    ACC(umma_apply(c->umma, c->stream, W, nullptr, stream_u(c, sf_buf), dense_codes(c), eta, K, c->dev_status));
   } else if (d.path == SFB_PATH_F32) {
     ACC(launch_apply_f32(c->stream, reinterpret_cast<float*>(W), stream_u(c, sf_buf), stream_v(c, sf_buf), K, d.J, d.D,
                          eta, c->dev_status));
   } else {
-    ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, sf_buf, eta, K, c->dev_status));
+    ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status));
     if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
   }
   return SFB_OK;

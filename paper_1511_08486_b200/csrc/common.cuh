@@ -106,6 +106,12 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
 int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                     const int* dev_status_ro, int* dev_status);
 
+// Dense fp32 rows a_i of the CSR codes (zeros elsewhere), for the tensor-core sparse-coding path.
+int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status);
+
+// SC epilogue on dense products: u = z - x in place (u rows hold z), pad columns zero.
+int launch_finish_sc(cudaStream_t s, RowMap u, const float* Xdata, int K, int J);
+
 // W (fp32) -> bf16 shadow, round to nearest even.
 int launch_cast_bf16(cudaStream_t s, const float* W, __nv_bfloat16* Wb, long long n);
 

@@ -109,6 +109,37 @@ __global__ void __launch_bounds__(256) sc_forward_kernel(const float* __restrict
   }
 }
 
+// One block per sample: zero the dense row, then scatter the sample's nonzeros into it.
+__global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, int K, int D, int* dev_status) {
+  const int i = blockIdx.x;
+  float* dst = reinterpret_cast<float*>(a.row(i));
+  for (int q = threadIdx.x; q < (a.ld >> 2); q += 256) reinterpret_cast<float4*>(dst)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncthreads();
+  const CsrRow row = csr_row(codes, i);
+  for (int k = threadIdx.x; k < row.len; k += 256) {
+    const uint32_t c = row.idx[k];
+    if (c >= (uint32_t)D || (k > 0 && row.idx[k - 1] >= c)) atomicOr(dev_status, SFB_DEV_BAD_INDEX);   // entry skipped
+    else dst[c] = row.val[k];
+  }
+}
+
+__global__ void __launch_bounds__(256) finish_sc_kernel(RowMap u, const float* __restrict__ Xdata, int K, int J) {
+  const int units = u.ld >> 2;
+  const long long total = (long long)K * units;
+  for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
+       g += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(g / units), j = (int)(g % units) * 4;
+    float4* p = reinterpret_cast<float4*>(u.row(i) + (size_t)j * 4);
+    float4 z = *p;
+    const float* x = Xdata + (size_t)i * J;
+    z.x = (j < J) ? z.x - x[j] : 0.f;
+    z.y = (j + 1 < J) ? z.y - x[j + 1] : 0.f;
+    z.z = (j + 2 < J) ? z.z - x[j + 2] : 0.f;
+    z.w = (j + 3 < J) ? z.w - x[j + 3] : 0.f;
+    *p = z;
+  }
+}
+
 constexpr int SLAB_D = 16;         // atoms per block: two 32-byte sectors of every row of W
 constexpr int SLAB_T = 256;        // threads per block
 constexpr int SLAB_J = 4 * SLAB_T; // rows of W per block: four consecutive rows per thread
@@ -265,6 +296,18 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
   dim3 grid(K, (ldt + 1023) / 1024);
   sc_forward_kernel<<<grid, 256, 0, s>>>(Wt, ldt, codes, Xdata, u, K, J, D, dev_status);
   return cudaGetLastError() == cudaSuccess ? 2 : SFB_ERR_CUDA;
+}
+
+int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status) {
+  densify_kernel<<<K, 256, 0, s>>>(codes, a, K, D, dev_status);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_finish_sc(cudaStream_t s, RowMap u, const float* Xdata, int K, int J) {
+  const long long total = (long long)K * (u.ld >> 2);
+  const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
+  finish_sc_kernel<<<blocks, 256, 0, s>>>(u, Xdata, K, J);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
 int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,

@@ -609,7 +609,6 @@ struct UmmaPlan {
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
                      UmmaPlan** out) {
   if (get_encode() == nullptr) return SFB_ERR_CUDA;
-  if (d.model == SFB_SC) return SFB_ERR_UNSUPPORTED;
   UmmaPlan* p = new UmmaPlan();
   p->d = d; p->l = l; p->z_ws = z_ws; p->ldz = ldz;
   p->es = (d.path == SFB_PATH_BF16) ? 2 : 4;
@@ -640,7 +639,7 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
 }
 
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
-static int forward_gemm(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status) {
+int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   GemmParams p;
@@ -682,7 +681,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   if (d.model == SFB_MLR) {
     const bool bf16 = d.path == SFB_PATH_BF16;
     RowMap zz = bf16 ? z : u;   // fp32 products: workspace when u is bf16, else u itself (finished in place)
-    if ((r = forward_gemm(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, zz, dev_status)) < 0) return r;
+    if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, zz, dev_status)) < 0) return r;
     launches += r;
     if ((r = launch_finish_mlr(s, zz, u, aux->labels, K, d.J, dev_status)) < 0) return r;
     launches += r;
@@ -697,16 +696,15 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   if ((r = launch_diff_rows(s, reinterpret_cast<const float*>(X), reinterpret_cast<const float*>(aux->Xb), v, K, d.D)) < 0)
     return r;
   launches += r;
-  if ((r = forward_gemm(pl, s, W, v, u, dev_status)) < 0) return r;
+  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status)) < 0) return r;
   launches += r;
   if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
   return launches + r;
 }
 
-int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, const void* sf_buf, float eta, int K,
-               const int* dev_status) {
+int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
+               int K, const int* dev_status) {
   const sfb_desc& d = pl->d;
-  const Layout& l = pl->l;
   const int es = pl->es, CH = 128 / es;
   const int workers = K / d.B;
   GemmParams p;
@@ -730,13 +728,12 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, c
   p.eta = eta;
   p.status_ro = dev_status;
   p.status = const_cast<int*>(dev_status);
-  const char* base = reinterpret_cast<const char*>(sf_buf) + l.streams_off;
   CUtensorMap tu, tv;
   // only the first `workers` streams are visible to the maps, so zero fill covers a ragged last block
-  if (!encode_rows_map(&tu, es, base, d.J, d.B, workers, (long long)l.ldu * es, l.stream_stride, p.k_bb, p.k_wp, v.fold,
-                       BM / CH, es == 4))
+  if (!encode_rows_map(&tu, es, u_rows.base, d.J, d.B, workers, (long long)u_rows.ld * es, u_rows.worker_stride, p.k_bb,
+                       p.k_wp, v.fold, BM / CH, es == 4))
     return SFB_ERR_CUDA;
-  if (!encode_rows_map(&tv, es, base + l.u_bytes, d.D, d.B, workers, (long long)l.ldv * es, l.stream_stride, p.k_bb,
+  if (!encode_rows_map(&tv, es, v_rows.base, d.D, d.B, workers, (long long)v_rows.ld * es, v_rows.worker_stride, p.k_bb,
                        p.k_wp, v.fold, (v.bn / v.cg) / CH, es == 4))
     return SFB_ERR_CUDA;
   return dispatch_gemm<true>(s, es, v, tu, tv, p, pl->num_sms);

@@ -16,8 +16,12 @@ void umma_plan_destroy(UmmaPlan* p);
 int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
                  const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status);
 
+// Z rows (fp32) = A rows (the path's value type) times Wop^T on the tensor cores; no epilogue beyond the store.
+int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status);
+
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
-int umma_apply(UmmaPlan* p, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, const void* sf_buf, float eta, int K,
-               const int* dev_status);
+// u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).
+int umma_apply(UmmaPlan* p, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
+               int K, const int* dev_status);
 
 }  // namespace sfb

@@ -65,3 +65,10 @@ def test_tf32_c1_full():
 def test_tf32_dml():
     check_config(_cfg("C2", "tf32", J=72, D=1000, P=3, B=20), "tf32", eta=1e-4, steps=2)
     check_config(_cfg("C2", "tf32"), "tf32", eta=1e-5, steps=1)
+
+
+def test_tf32_sparse_coding_dense_alternative():
+    # the codes as dense tf32 rows through the tensor-core GEMMs; the wire buffer keeps them CSR
+    check_config(_cfg("C3", "tf32", J=70, D=332, P=3, B=5, density=0.1), "tf32", eta=1e-2, steps=2)
+    check_config(_cfg("C3", "tf32", J=512, D=2000, P=4, B=32), "tf32", eta=1e-3, steps=2)
+    check_config(_cfg("C3", "tf32"), "tf32", eta=1e-4, steps=1)
