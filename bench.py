@@ -118,15 +118,25 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
-def algorithmic(cfg, path):
-    """Flops / bytes one apply launch must do (what the roofline fraction is computed from)."""
+def algorithmic(cfg, path, inputs=None):
+    """Flops / bytes one apply launch must do (what the roofline fraction is computed from).
+
+    Dense apply: 2*J*D*K flop; bytes = W read + W write (+ bf16 shadow) + the K (u, v) pairs.
+    Sparse-v scatter apply (SC, fp32 path): 2*J*nnz flop; bytes = W read + W write + U + CSR codes.
+    """
     J, D, K = cfg["J"], cfg["D"], cfg["K"]
     es = 2 if path == "bf16" else 4
-    if cfg["model"] == "sc":
-        return None
+    if cfg["model"] == "sc" and path == "f32":
+        nnz = int(inputs["rowptr"][0][-1]) if inputs is not None else int(cfg["density"] * K * D)
+        return dict(flops=2.0 * J * nnz, bytes=2.0 * J * D * 4 + K * J * 4 + nnz * 8.0, sparse=True)
     flops = 2.0 * J * D * K
     bytes_ = 2.0 * J * D * 4 + K * (J + D) * es + (J * D * 2 if path == "bf16" else 0)
-    return dict(flops=flops, bytes=bytes_)
+    return dict(flops=flops, bytes=bytes_, sparse=False)
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one apply launch, from the ncu captures summarised
+# under profiles/ (captured at J = 8192 and scaled by J where the full launch is too large to capture).
+NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 6.0e9}
 
 
 def oracle_step_time(cfg, inputs, sample_workers: int):
@@ -181,6 +191,22 @@ def run_reference(args, cfg, inputs):
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
+
+
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of `values` over all ranks (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_throughput(units_per_rank_step, steps, ms, world):
+    """Units all ranks processed divided by the (max over ranks) time: replicas => weak scaling."""
+    return world * units_per_rank_step * steps / (ms * 1e-3)
 
 
 def workload_name(cfg, path):
@@ -311,15 +337,12 @@ def main():
     clock_of_last = int(np.frombuffer(result_host.numpy().tobytes(), dtype=np.uint32)[7])
 
     # ---- max over ranks ---------------------------------------------------------------------------
-    if world > 1:
-        tt = torch.tensor([ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(tt[0]), float(tt[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], device=dev)
 
     if rank == 0:
         peaks = load_peaks()
-        alg = algorithmic(cfg, path)
-        value = world * K * args.steps / (ms * 1e-3)
+        alg = algorithmic(cfg, path, inputs)
+        value = whole_job_throughput(K, args.steps, ms, world)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -328,7 +351,7 @@ def main():
             "config": {"workload": workload_name(cfg, path), "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "per-step footprint larger than L2" if flush is None else "L2 flushed between steps",
                        "eta": eta, "pool": cfg["pool"]},
-            "e2e": {"value": world * K * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": whole_job_throughput(K, args.steps, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "last_clock_read_back": clock_of_last},
             "gpu_launches": int(launches),
             "device_status": status,
@@ -338,7 +361,13 @@ def main():
         if alg is not None:
             apply_tflops = alg["flops"] / (a_ms * 1e-3) / 1e12
             fwd_tflops = alg["flops"] / (f_ms * 1e-3) / 1e12
-            if path == "f32":
+            traffic = NCU_APPLY_TRAFFIC_BYTES.get((args.config, path)) if not over else None
+            if alg["sparse"]:
+                gbs = alg["bytes"] / (a_ms * 1e-3) / 1e9
+                out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm_gbs"], "traffic": traffic, "kernel": "sc_apply_kernel",
+                                   "peak_source": f"{peaks['source']} HBM copy bandwidth"}
+            elif path == "f32":
                 out["roofline"] = {"bound": "alu", "achieved": apply_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
                                    "frac": apply_tflops / FP32_FMA_TFLOPS, "traffic": None,
                                    "kernel": "apply_f32_kernel", "peak_source": "148 SMs x 128 FMA lanes x 1.965 GHz"}
@@ -346,7 +375,7 @@ def main():
                 scale = 1.0 if path == "bf16" else 0.5          # tf32 nominal rate is half of bf16
                 peak = peaks["bf16_sustained"] * scale
                 out["roofline"] = {"bound": "tensor", "achieved": apply_tflops, "peak": peak, "unit": "TFLOP/s",
-                                   "frac": apply_tflops / peak, "traffic": None, "kernel": "umma apply",
+                                   "frac": apply_tflops / peak, "traffic": traffic, "kernel": "umma_gemm_kernel (apply)",
                                    "peak_source": f"{peaks['source']} cuBLAS bf16 sustained" + ("" if path == "bf16" else " x 0.5 (tf32)"),
                                    "frac_of_burst": apply_tflops / (peaks["bf16"] * scale),
                                    "frac_of_datasheet": apply_tflops / (DATASHEET_BF16_TFLOPS * scale)}

@@ -203,10 +203,6 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
   if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_TF32)
     ok = cudaMalloc(&c->a_dense, (size_t)c->K * c->l.ldv * 4) == cudaSuccess;
-  if (ok && desc->path == SFB_PATH_BF16) {
-    c->ldz = (int)pad_to(desc->J, 4);
-    ok = cudaMalloc(&c->z_ws, (size_t)c->K * c->ldz * 4) == cudaSuccess;
-  }
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();

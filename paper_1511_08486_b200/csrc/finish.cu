@@ -170,6 +170,71 @@ __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, co
   }
 }
 
+// Second half of the fused multiclass-logistic epilogue.  The forward GEMM left e[j] = exp(z[j] - m_p)
+// in the u row (p = the half tile that holds class j) and (m_p, s_p = sum of those exps) per part.
+// Here: m = max_p m_p, s = sum_p s_p exp(m_p - m), u[j] = e[j] * exp(m_p - m) / s - [j == label], in place.
+template <int ES>
+__global__ void __launch_bounds__(256) finish_mlr_fused_kernel(RowMap u, const float2* __restrict__ stats, int n_parts,
+                                                               int part_cols, const int32_t* __restrict__ labels, int K,
+                                                               int J, int* dev_status) {
+  extern __shared__ float scale[];   // [n_parts]
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  if (i >= K) return;
+  const float kLog2e = 1.4426950408889634f;
+  const float2* st = stats + (size_t)i * n_parts;
+  float m = -INFINITY;
+  for (int q = threadIdx.x; q < n_parts; q += 256) m = fmaxf(m, st[q].x);
+  m = block_max(m, red);
+  float ssum = 0.f;
+  for (int q = threadIdx.x; q < n_parts; q += 256) {
+    const float2 ps = st[q];
+    const float f = (ps.x == -INFINITY) ? 0.f : exp2f((ps.x - m) * kLog2e);
+    scale[q] = f;
+    ssum += ps.y * f;
+  }
+  ssum = block_sum(ssum, red);   // also orders the writes of scale[] before the reads below
+  const float inv = 1.0f / ssum;
+  const int y = labels[i];
+  const bool bad = (y < 0) || (y >= J);
+  if (bad && threadIdx.x == 0) atomicOr(dev_status, SFB_DEV_BAD_LABEL);
+  char* ur = u.row(i);
+  constexpr int PER = 16 / ES;          // values per 16-byte unit (part_cols is a multiple of it)
+  const int units = u.ld / PER;
+  for (int q = threadIdx.x; q < units; q += 256) {
+    const int j = q * PER;
+    uint4 raw = *reinterpret_cast<const uint4*>(ur + (size_t)q * 16);
+    float vals[PER];
+    if (ES == 4) {
+      const float* f = reinterpret_cast<const float*>(&raw);
+#pragma unroll
+      for (int e = 0; e < PER; ++e) vals[e] = f[e];
+    } else {
+      const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&raw);
+#pragma unroll
+      for (int e = 0; e < PER; ++e) vals[e] = __bfloat162float(h[e]);
+    }
+    const float f = (j < J && !bad) ? scale[j / part_cols] * inv : 0.f;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      float r = vals[e] * f;
+      if (j + e == y) r -= 1.f;
+      if (j + e >= J || bad) r = 0.f;
+      vals[e] = r;
+    }
+    if (ES == 4) {
+      float* f4 = reinterpret_cast<float*>(&raw);
+#pragma unroll
+      for (int e = 0; e < PER; ++e) f4[e] = vals[e];
+    } else {
+      __nv_bfloat16* h = reinterpret_cast<__nv_bfloat16*>(&raw);
+#pragma unroll
+      for (int e = 0; e < PER; ++e) h[e] = __float2bfloat16_rn(vals[e]);
+    }
+    *reinterpret_cast<uint4*>(ur + (size_t)q * 16) = raw;
+  }
+}
+
 // 16-byte-vectorised row copy; rows are whole numbers of 16-byte units on both sides.
 __global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, int K, int cols) {
   const int units_dst = dst.ld * dst.es / 16;
@@ -263,6 +328,15 @@ int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar
     attr_done = true;
   }
   finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_finish_mlr_fused(cudaStream_t s, RowMap u, const float2* stats, int n_parts, int part_cols,
+                            const int32_t* labels, int K, int J, int* dev_status) {
+  const size_t smem = (size_t)n_parts * sizeof(float);
+  if (smem > 48 * 1024) return SFB_ERR_SHAPE;
+  if (u.es == 4) finish_mlr_fused_kernel<4><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status);
+  else finish_mlr_fused_kernel<2><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

@@ -27,6 +27,8 @@ namespace sfb {
 
 // extra passes implemented in finish.cu
 int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D);
+int launch_finish_mlr_fused(cudaStream_t s, RowMap u, const float2* stats, int n_parts, int part_cols,
+                            const int32_t* labels, int K, int J, int* dev_status);
 
 namespace {
 
@@ -49,7 +51,9 @@ struct GemmParams {
   __nv_bfloat16* shadow;    // apply: bf16 copy of the new W (or nullptr)
   long long ldw;
   float eta;
-  RowMap z;                 // forward: fp32 output rows
+  RowMap z;                 // forward: output rows (fp32 products, or exps in the factor's storage type)
+  float2* stats;            // forward, EPI 1: (max, sum of exps) per (sample, half tile), [K][n_parts]
+  int n_parts;
   const int* status_ro;
   int* status;
 };
@@ -82,10 +86,14 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sh
 //          and "accumulator ready" are committed (tcgen05.commit) once to the even CTA's barrier and
 //          once to the odd CTA's; both epilogues arrive on the even CTA's "accumulator drained" barrier.
 //   KA     128-byte atoms of the reduction index per pipeline stage (BK = KA * CH reduction steps).
+//   EPI    forward epilogue: 0 = store the products z; 1 = multiclass-logistic epilogue: store
+//          exp(z - m) with m the row maximum over this warp's half tile, in the factor's storage
+//          type, plus (m, sum of exps) per (sample, half tile) for the finishing pass that
+//          rescales to the softmax and subtracts the one-hot label (Section 2.1: u = softmax - onehot).
 //   FOLD   operands come through 4-D tensor maps whose extra dimension walks the 128-byte chunks, so
 //          one TMA instruction fills a whole operand stage (needs J, D multiples of CH); otherwise
 //          one 3-D TMA per chunk, with zero fill on every ragged edge.
-template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD>
+template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr int CH = 128 / ES;                 // values per 128-byte chunk
@@ -388,6 +396,66 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
+      if (!APPLY && EPI == 1) {
+        // ---- multiclass-logistic epilogue: thread = sample row while the values sit in registers
+        const float kLog2e = 1.4426950408889634f;
+        const int ccol0 = nt * BN + half * (BN / 2);     // first class of this warp's half tile
+        float m = -INFINITY;
+#pragma unroll 1
+        for (int cc = 0; cc < BN / 64; ++cc) {
+          uint32_t v[32];
+          ptx::tmem_ld32(taddr + half * (BN / 2) + cc * 32, v);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 32; ++q)
+            if (ccol0 + cc * 32 + q < p.Nvalid) m = fmaxf(m, __uint_as_float(v[q]));
+        }
+        const float mb = (m == -INFINITY) ? 0.f : m * kLog2e;   // half tile entirely beyond the last class
+        float ssum = 0.f;
+#pragma unroll 1
+        for (int cc = 0; cc < BN / 64; ++cc) {
+          const int c = cbase + cc * 32;
+          uint32_t v[32];
+          ptx::tmem_ld32(taddr + half * (BN / 2) + cc * 32, v);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 32; ++q) {
+            const float ex = (ccol0 + cc * 32 + q < p.Nvalid) ? exp2f(fmaf(__uint_as_float(v[q]), kLog2e, -mb)) : 0.f;
+            ssum += ex;
+            v[q] = __float_as_uint(ex);
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<uint4*>(stage + lane * 32 + ((q ^ (lane & 7)) << 2)) =
+                make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+          __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const int lr = 4 * g + lrow;
+            const float4 a = *reinterpret_cast<const float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2));
+            if (rowp[g] != nullptr && c < ncols) {
+              if (p.z.es == 4) {
+                __stcs(reinterpret_cast<float4*>(rowp[g] + c), a);
+              } else {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                __stcs(reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(rowp[g]) + c), pk);
+              }
+            }
+          }
+          __syncwarp();
+        }
+        {   // (max, sum) of this thread's own row
+          const int r = quarter * 32 + lane;
+          int wp_, slot;
+          if (p.B >= BM) { wp_ = mt / p.m_tpw; slot = (mt % p.m_tpw) * BM + r; }
+          else { wp_ = mt * p.m_wp + r / p.m_bb; slot = r % p.m_bb; }
+          if (wp_ < p.P && slot < p.B)
+            p.stats[(long long)(wp_ * p.B + slot) * p.n_parts + nt * 2 + half] = make_float2(m, ssum);
+        }
+      } else
 #pragma unroll 1
       for (int cc = 0; cc < BN / 64; ++cc) {
         const int col_in_tile = half * (BN / 2) + cc * 32;
@@ -518,12 +586,12 @@ int pow2_at_least(int n) {
   return p;
 }
 
-template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD>
+template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI>
 int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, int num_sms) {
   constexpr int stage_bytes = (BM + BN / CG) * 128 * KA;
   constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
   constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
-  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD>;
+  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD, EPI>;
   static bool attr_done = false;
   static int max_clusters = 0;
   if (!attr_done) {
@@ -574,22 +642,22 @@ struct Variant {
   bool fold;
 };
 
-template <int ES, bool APPLY>
+template <int ES, bool APPLY, int EPI>
 int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p,
                 int num_sms) {
   if (v.cg == 2) {
-    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true>(s, a, b, p, num_sms);
-    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true>(s, a, b, p, num_sms);
-    return launch_gemm<ES, APPLY, 256, 2, 1, false>(s, a, b, p, num_sms);
+    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, p, num_sms);
+    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, p, num_sms);
+    return launch_gemm<ES, APPLY, 256, 2, 1, false, EPI>(s, a, b, p, num_sms);
   }
-  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false>(s, a, b, p, num_sms);
-  return launch_gemm<ES, APPLY, 128, 1, 1, false>(s, a, b, p, num_sms);
+  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false, EPI>(s, a, b, p, num_sms);
+  return launch_gemm<ES, APPLY, 128, 1, 1, false, EPI>(s, a, b, p, num_sms);
 }
 
-template <bool APPLY>
+template <bool APPLY, int EPI>
 int dispatch_gemm(cudaStream_t s, int es, const Variant& v, const CUtensorMap& a, const CUtensorMap& b,
                   const GemmParams& p, int num_sms) {
-  return es == 2 ? dispatch_es<2, APPLY>(s, v, a, b, p, num_sms) : dispatch_es<4, APPLY>(s, v, a, b, p, num_sms);
+  return es == 2 ? dispatch_es<2, APPLY, EPI>(s, v, a, b, p, num_sms) : dispatch_es<4, APPLY, EPI>(s, v, a, b, p, num_sms);
 }
 
 }  // namespace
@@ -604,6 +672,7 @@ struct UmmaPlan {
   bool pair_ok;   // CTA-pair kernels allowed (off with SFB_NO_CTA_PAIRS=1, for A/B measurements)
   bool fold_ok;   // folded operand loads allowed (off with SFB_NO_FOLD=1)
   int fold_ka;    // 128-byte atoms of the reduction index per stage in the folded kernels (SFB_FOLD_KA, default 2)
+  float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -621,11 +690,23 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   p->fold_ok = !(no_fold != nullptr && no_fold[0] == '1');
   const char* ka = getenv("SFB_FOLD_KA");
   p->fold_ka = (ka != nullptr && ka[0] == '1') ? 1 : 2;
+  p->stats = nullptr;
+  if (d.model == SFB_MLR) {
+    const size_t parts = 2 * (size_t)((d.J + 127) / 128);
+    if (cudaMalloc(&p->stats, (size_t)d.P * d.B * parts * sizeof(float2)) != cudaSuccess) {
+      cudaGetLastError();
+      delete p;
+      return SFB_ERR_ALLOC;
+    }
+  }
   *out = p;
   return SFB_OK;
 }
 
-void umma_plan_destroy(UmmaPlan* p) { delete p; }
+void umma_plan_destroy(UmmaPlan* p) {
+  if (p->stats) cudaFree(p->stats);
+  delete p;
+}
 
 // Tile shape and kernel variant for an M x N output (M counted in 128-row units).
 static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_chunk_aligned) {
@@ -639,7 +720,8 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
 }
 
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
-int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status) {
+int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
+                      float2* stats, int* n_parts_out, int* part_cols_out) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   GemmParams p;
@@ -659,6 +741,11 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.b_policy = p.m_fastest ? 0 : 2;
   p.z = z;
   p.status = dev_status;
+  p.Nvalid = d.J;
+  p.stats = stats;
+  p.n_parts = 2 * p.n_tiles;
+  if (n_parts_out != nullptr) *n_parts_out = p.n_parts;
+  if (part_cols_out != nullptr) *part_cols_out = v.bn / 2;
   CUtensorMap ta, tb;
   if (!encode_rows_map(&ta, es, a.base, d.D, d.B, d.P, (long long)a.ld * es, a.worker_stride, p.m_bb, p.m_wp, v.fold,
                        v.ka, false))
@@ -666,7 +753,8 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, v.bn / v.cg, 1,
                        v.fold, v.ka, false))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<false>(s, es, v, ta, tb, p, pl->num_sms);
+  return stats != nullptr ? dispatch_gemm<false, 1>(s, es, v, ta, tb, p, pl->num_sms)
+                          : dispatch_gemm<false, 0>(s, es, v, ta, tb, p, pl->num_sms);
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
@@ -681,9 +769,15 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   if (d.model == SFB_MLR) {
     const bool bf16 = d.path == SFB_PATH_BF16;
     RowMap zz = bf16 ? z : u;   // fp32 products: workspace when u is bf16, else u itself (finished in place)
-    if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, zz, dev_status)) < 0) return r;
+    // the GEMM epilogue leaves exp(z - local max) in u and (max, sum) per half tile; the finishing
+    // pass rescales to the softmax and subtracts the one-hot label, in place
+    int n_parts = 0, part_cols = 0;
+    (void)zz;
+    if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
+                               &part_cols)) < 0)
+      return r;
     launches += r;
-    if ((r = launch_finish_mlr(s, zz, u, aux->labels, K, d.J, dev_status)) < 0) return r;
+    if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status)) < 0) return r;
     launches += r;
     if (v.base != nullptr) {
       if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
@@ -696,7 +790,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   if ((r = launch_diff_rows(s, reinterpret_cast<const float*>(X), reinterpret_cast<const float*>(aux->Xb), v, K, d.D)) < 0)
     return r;
   launches += r;
-  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status)) < 0) return r;
+  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr)) < 0) return r;
   launches += r;
   if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
   return launches + r;
@@ -736,7 +830,7 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   if (!encode_rows_map(&tv, es, v_rows.base, d.D, d.B, workers, (long long)v_rows.ld * es, v_rows.worker_stride, p.k_bb,
                        p.k_wp, v.fold, (v.bn / v.cg) / CH, es == 4))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<true>(s, es, v, tu, tv, p, pl->num_sms);
+  return dispatch_gemm<true, 0>(s, es, v, tu, tv, p, pl->num_sms);
 }
 
 }  // namespace sfb
