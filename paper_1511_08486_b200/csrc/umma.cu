@@ -43,6 +43,7 @@ struct GemmParams {
   int m_tiles, n_tiles, k_blocks;   // m_tiles counts tiles of 128*CG rows; k_blocks counts blocks of BK reduction steps
   int a_policy, b_policy;   // L2 eviction policy of the operand loads (0 normal, 1 evict first, 2 evict last)
   int m_fastest;            // tile order: 1 = consecutive tiles share the B operand slab, 0 = share the A slab
+  int group;                // tiles of the fast dimension walked before the slow one advances (0 = all)
   int B, P;                 // rows per worker / workers, geometry of the operand maps
   int m_bb, m_wp, m_tpw;    // forward: 128 A rows come as a box of m_bb rows x m_wp workers; 128-row units per worker
   int k_bb, k_wp, k_bpw;    // apply: a reduction block is k_bb rows x k_wp workers; blocks per worker
@@ -72,6 +73,28 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sh
   ctl->abort = 1;
   if (status != nullptr) atomicOr(status, SFB_DEV_TIMEOUT);
   return false;
+}
+
+// Tile order.  m_fastest = 0: consecutive tiles walk `group` column tiles, then the next row tile,
+// and only after all row tiles the next group of columns; so one wave of CTAs touches few B slabs
+// (they stay in L2 across waves) while the A slabs stream.  m_fastest = 1: the same with rows and
+// columns exchanged.  group = 0 means one group spanning the whole dimension.
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& mt, int& nt) {
+  if (!p.m_fastest) {
+    const int g = p.group > 0 ? p.group : p.n_tiles;
+    const int per = p.m_tiles * g;
+    const int sc = tile / per, r = tile - sc * per;
+    const int ge = min(g, p.n_tiles - sc * g);
+    mt = r / ge;
+    nt = sc * g + (r - mt * ge);
+  } else {
+    const int g = p.group > 0 ? p.group : p.m_tiles;
+    const int per = p.n_tiles * g;
+    const int sc = tile / per, r = tile - sc * per;
+    const int ge = min(g, p.m_tiles - sc * g);
+    nt = r / ge;
+    mt = sc * g + (r - nt * ge);
+  }
 }
 
 // Template parameters of the GEMM kernel:
@@ -159,9 +182,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     long long exp_wait_empty = 0;
 #endif
     for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
-      const int mt = (p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles) * CG + (int)rank;   // 128-row unit
-      const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
-      const int ncol0 = nt * BN + (int)rank * BNC;                                           // first B column loaded here
+      int mt, nt;
+      tile_coords(p, tile, mt, nt);
+      mt = mt * CG + (int)rank;                           // 128-row unit of this CTA
+      const int ncol0 = nt * BN + (int)rank * BNC;       // first B column loaded here
       int slot0 = 0, mp0 = 0;          // forward: first slot / worker of this CTA's 128 sample rows
       if (!APPLY) {
         if (p.B >= BM) { mp0 = mt / p.m_tpw; slot0 = (mt % p.m_tpw) * BM; }
@@ -349,8 +373,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int it = 0;
     bool ok = true;
     for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++it) {
-      const int mt = (p.m_fastest ? tile % p.m_tiles : tile / p.n_tiles) * CG + (int)rank;
-      const int nt = p.m_fastest ? tile / p.m_tiles : tile % p.n_tiles;
+      int mt, nt;
+      tile_coords(p, tile, mt, nt);
+      mt = mt * CG + (int)rank;
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
       // destination rows of the 8 row groups this lane touches (row = quarter*32 + 4*g + lrow)
@@ -673,6 +698,7 @@ struct UmmaPlan {
   bool fold_ok;   // folded operand loads allowed (off with SFB_NO_FOLD=1)
   int fold_ka;    // 128-byte atoms of the reduction index per stage in the folded kernels (SFB_FOLD_KA, default 2)
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
+  int fwd_group, apply_group;   // tile-order group widths (SFB_FWD_GROUP / SFB_APPLY_GROUP override the defaults)
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -690,6 +716,10 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   p->fold_ok = !(no_fold != nullptr && no_fold[0] == '1');
   const char* ka = getenv("SFB_FOLD_KA");
   p->fold_ka = (ka != nullptr && ka[0] == '1') ? 1 : 2;
+  const char* fg = getenv("SFB_FWD_GROUP");
+  const char* ag = getenv("SFB_APPLY_GROUP");
+  p->fwd_group = fg != nullptr ? atoi(fg) : 8;
+  p->apply_group = ag != nullptr ? atoi(ag) : 8;
   p->stats = nullptr;
   if (d.model == SFB_MLR) {
     const size_t parts = 2 * (size_t)((d.J + 127) / 128);
@@ -739,6 +769,7 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.m_fastest = ((long long)d.J * d.D > (long long)d.P * d.B * d.D) ? 1 : 0;
   p.a_policy = p.m_fastest ? 2 : 0;   // the operand whose slab changes every tile is re-read all along: keep it
   p.b_policy = p.m_fastest ? 0 : 2;
+  p.group = pl->fwd_group;
   p.z = z;
   p.status = dev_status;
   p.Nvalid = d.J;
@@ -816,6 +847,7 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
   p.a_policy = p.m_fastest ? 2 : 0;
   p.b_policy = p.m_fastest ? 0 : 2;
+  p.group = pl->apply_group;
   p.W = reinterpret_cast<float*>(W);
   p.shadow = (d.path == SFB_PATH_BF16) ? w_shadow : nullptr;
   p.ldw = d.D;
