@@ -136,7 +136,7 @@ def algorithmic(cfg, path, inputs=None):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one apply launch, from the ncu captures summarised
 # under profiles/ (captured at J = 8192 and scaled by J where the full launch is too large to capture).
-NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 6.0e9}
+NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 4.03e9}
 
 
 def oracle_step_time(cfg, inputs, sample_workers: int):
