@@ -161,6 +161,17 @@ int64_t sfb_launch_count(const sfb_ctx* ctx);
 
 const char* sfb_strerror(int code);
 
+/* Halton-sequence broadcast (Section 4.3): the Q workers that worker p (zero-based) of P would
+ * send its factor stream to, (p + floor(P f)) mod P for f = 1/2, 1/4, 3/4, 1/8, 3/8, ... in that
+ * order, written to peers[0..Q).  Host-only; peers is a HOST array.  SFB_ERR_ARG on bad arguments. */
+int sfb_halton_peers(int32_t P, int32_t Q, int32_t p, int32_t* peers);
+
+/* Stale-synchronous rule (Section 4.1): 1 if worker p, having computed t_p batches and received
+ * tau[q] batches from each of the P workers, may start its next batch (no q with
+ * t_p - tau[q] > staleness), else 0.  staleness 0 = BSP, negative = unbounded (ASP).  Host-only;
+ * tau is a HOST array.  Negative return = SFB_ERR_*. */
+int sfb_ssp_may_proceed(int64_t t_p, const int64_t* tau, int32_t P, int64_t staleness);
+
 /* Sparse-coding factors u_i = W a_i - x_i for callers that must not allocate device memory: code
  * that runs while its stream is being captured into a CUDA graph, latency-bound loops that cannot
  * afford the allocator's implicit synchronisation, and processes whose device memory was handed

@@ -23,6 +23,7 @@ EXPORTS = (
     "sfb_create", "sfb_destroy", "sfb_sf_buffer_bytes", "sfb_ld", "sfb_compute_factors", "sfb_pack",
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
     "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
+    "sfb_halton_peers", "sfb_ssp_may_proceed",
 )
 
 
@@ -86,6 +87,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_sc_factors_noalloc.restype = C.c_int
     lib.sfb_noalloc_max_scratch_floats.argtypes = []
     lib.sfb_noalloc_max_scratch_floats.restype = C.c_int64
+    lib.sfb_halton_peers.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32)]
+    lib.sfb_halton_peers.restype = C.c_int
+    lib.sfb_ssp_may_proceed.argtypes = [C.c_int64, C.POINTER(C.c_int64), C.c_int32, C.c_int64]
+    lib.sfb_ssp_may_proceed.restype = C.c_int
     lib.sfb_strerror.argtypes = [C.c_int]
     lib.sfb_strerror.restype = C.c_char_p
     if path == LIB_PATH:
@@ -140,6 +145,22 @@ def sfb_sc_factors_noalloc(W, J, D, K, rowptr, idx, val, Xdata, U, ldu, dev_stat
                                               _ptr(U), ldu, _ptr(dev_status), C.c_void_p(stream))
     if r != SFB_OK:
         raise SfbError(r, "sfb_sc_factors_noalloc")
+
+
+def sfb_halton_peers(P: int, Q: int, p: int) -> list[int]:
+    out = (C.c_int32 * max(Q, 1))()
+    r = load_library().sfb_halton_peers(P, Q, p, out)
+    if r != SFB_OK:
+        raise SfbError(r, "sfb_halton_peers")
+    return [int(out[i]) for i in range(Q)]
+
+
+def sfb_ssp_may_proceed(t_p: int, tau, staleness: int) -> bool:
+    arr = (C.c_int64 * len(tau))(*[int(t) for t in tau])
+    r = load_library().sfb_ssp_may_proceed(int(t_p), arr, len(tau), int(staleness))
+    if r < 0:
+        raise SfbError(r, "sfb_ssp_may_proceed")
+    return bool(r)
 
 
 def sfb_noalloc_max_scratch_floats() -> int:
