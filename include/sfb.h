@@ -142,6 +142,13 @@ int sfb_apply(sfb_ctx* ctx, void* W, const void* sf_buf, float eta, int32_t K);
 int sfb_step(sfb_ctx* ctx, void* W, const void* X, const sfb_aux* aux, void* sf_buf, float eta, int32_t K,
              uint32_t clock);
 
+/* Proximal operator applied after the update (Section 2.1: prox_{eta h}; Section 3: "finally each
+ * worker applies the proximal operator").  SFB_SC: h is the indicator of ||W_k||_2 <= 1 for every
+ * column (atom) k, so each column whose norm exceeds 1 is divided by its norm and the others are
+ * left bit-identical (Figure 3, function prox).  SFB_MLR / SFB_DML: h = 0, nothing to do (returns
+ * SFB_OK without launching).  W [J][D] fp32 in place. */
+int sfb_prox(sfb_ctx* ctx, void* W);
+
 /* Tells the context that W was changed by someone else, so a cached bf16 shadow is stale. */
 int sfb_invalidate(sfb_ctx* ctx);
 

@@ -160,6 +160,16 @@ def apply_sparse(W, U, rowptr, idx, val, eta):
     return Wn
 
 
+def prox_unit_columns(W):
+    """Proximal operator of the sparse-coding constraint ||W_k||_2 <= 1 (Section 2, SC; Figure 3 `prox`):
+    every column whose norm exceeds 1 is divided by its norm, the others are left alone."""
+    Wn = _f64(W).copy()
+    n = np.sqrt((Wn * Wn).sum(axis=0))
+    big = n > 1.0
+    Wn[:, big] /= n[big]
+    return Wn
+
+
 # --------------------------------------------------------------------------------------
 # One step = factors from W_t and minibatch t, then apply (BSP: one W serves all workers)
 # --------------------------------------------------------------------------------------

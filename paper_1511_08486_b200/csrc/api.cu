@@ -236,6 +236,13 @@ int sfb_destroy(sfb_ctx* c) {
   return SFB_OK;
 }
 
+int sfb_prox(sfb_ctx* c, void* W) {
+  if (c == nullptr || W == nullptr || !aligned(W, 16)) return SFB_ERR_ARG;
+  if (c->d.model != SFB_SC) return SFB_OK;   // h = 0 for the MLR and DML workloads: identity
+  ACC(launch_prox_unit_columns(c->stream, reinterpret_cast<float*>(W), c->d.J, c->d.D));
+  return SFB_OK;
+}
+
 int sfb_invalidate(sfb_ctx* c) {
   if (c == nullptr) return SFB_ERR_ARG;
   c->shadow_of = nullptr;

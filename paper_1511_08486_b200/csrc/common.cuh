@@ -112,6 +112,9 @@ int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, 
 // SC epilogue on dense products: u = z - x in place (u rows hold z), pad columns zero.
 int launch_finish_sc(cudaStream_t s, RowMap u, const float* Xdata, int K, int J);
 
+// Column-norm projection: every column of W with 2-norm above 1 is divided by its norm (in place).
+int launch_prox_unit_columns(cudaStream_t s, float* W, int J, int D);
+
 // W (fp32) -> bf16 shadow, round to nearest even.
 int launch_cast_bf16(cudaStream_t s, const float* W, __nv_bfloat16* Wb, long long n);
 

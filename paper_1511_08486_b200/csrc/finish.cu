@@ -235,6 +235,35 @@ __global__ void __launch_bounds__(256) finish_mlr_fused_kernel(RowMap u, const f
   }
 }
 
+// Unit-ball projection of the columns of W (sparse-coding prox).  One block owns 32 consecutive
+// columns: 32 x 8 threads walk the rows (a warp reads one 128-byte line per row), the squared norms are
+// combined in a fixed order, then the block rescales its columns (second read served by L2).  Columns
+// with norm <= 1 are not written at all.
+__global__ void __launch_bounds__(256) prox_unit_columns_kernel(float* __restrict__ W, int J, int D) {
+  __shared__ float part[8][33];
+  __shared__ float scale[32];
+  const int c = threadIdx.x & 31, r = threadIdx.x >> 5;
+  const int d = blockIdx.x * 32 + c;
+  float acc = 0.f;
+  if (d < D)
+    for (int j = r; j < J; j += 8) {
+      const float w = W[(size_t)j * D + d];
+      acc = fmaf(w, w, acc);
+    }
+  part[r][c] = acc;
+  __syncthreads();
+  if (r == 0) {
+    float n2 = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) n2 += part[q][c];
+    scale[c] = (n2 > 1.0f) ? 1.0f / sqrtf(n2) : 1.0f;
+  }
+  __syncthreads();
+  const float sc = scale[c];
+  if (d < D && sc != 1.0f)
+    for (int j = r; j < J; j += 8) W[(size_t)j * D + d] *= sc;
+}
+
 // 16-byte-vectorised row copy; rows are whole numbers of 16-byte units on both sides.
 __global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, int K, int cols) {
   const int units_dst = dst.ld * dst.es / 16;
@@ -337,6 +366,11 @@ int launch_finish_mlr_fused(cudaStream_t s, RowMap u, const float2* stats, int n
   if (smem > 48 * 1024) return SFB_ERR_SHAPE;
   if (u.es == 4) finish_mlr_fused_kernel<4><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status);
   else finish_mlr_fused_kernel<2><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_prox_unit_columns(cudaStream_t s, float* W, int J, int D) {
+  prox_unit_columns_kernel<<<(D + 31) / 32, 256, 0, s>>>(W, J, D);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

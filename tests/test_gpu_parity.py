@@ -247,3 +247,29 @@ def test_sparse_bad_index_sets_status():
         assert wl.ctx.status() & B.SFB_DEV_BAD_INDEX
     finally:
         wl.close()
+
+
+def test_sc_prox_unit_columns():
+    """Column projection after the update (Figure 3, prox): parity with the oracle, untouched columns bit-identical."""
+    cfg = scaled("C3", J=300, D=1003, P=2, B=8, density=0.05)
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        rng = np.random.default_rng(7)
+        scale = rng.uniform(0.2, 3.0, cfg["D"]).astype(np.float32)      # some columns inside, some outside the ball
+        W = (inputs["W"] * scale[None, :]).astype(np.float32)
+        wl.W.copy_(torch.from_numpy(W))
+        wl.ctx.prox(wl.W)
+        torch.cuda.synchronize()
+        got = wl.W.cpu().numpy()
+        ref = orc.prox_unit_columns(W)
+        inside = np.linalg.norm(W.astype(np.float64), axis=0) <= 1.0 - 1e-6
+        assert inside.any() and (~inside).any()
+        assert np.array_equal(got[:, inside], W[:, inside])
+        assert orc.rel_fro(got, ref) <= 1e-6
+        assert (np.linalg.norm(got.astype(np.float64), axis=0) <= 1.0 + 1e-5).all()
+        wl.ctx.prox(wl.W)                                               # idempotent up to fp32 rounding
+        torch.cuda.synchronize()
+        assert orc.rel_fro(wl.W.cpu().numpy(), ref) <= 1e-6
+    finally:
+        wl.close()

@@ -271,6 +271,21 @@ def test_sc_special_cases():
     assert np.array_equal(Wn2[:, ~used], W.astype(np.float64)[:, ~used])
 
 
+def test_sc_prox_projects_columns_onto_the_unit_ball():
+    W = np.array([[3.0, 0.3, 0.0, 1.0], [4.0, 0.4, 0.0, 0.0]])
+    Wp = orc.prox_unit_columns(W)
+    assert np.allclose(Wp[:, 0], [0.6, 0.8], atol=1e-15)           # norm 5 -> divided by 5
+    assert np.array_equal(Wp[:, 1:], W[:, 1:])                       # norms 0.5, 0, exactly 1: untouched
+    R = RNG.normal(0, 1, (9, 13))
+    Rp = orc.prox_unit_columns(R)
+    n0, n1 = np.linalg.norm(R, axis=0), np.linalg.norm(Rp, axis=0)
+    assert (n1 <= 1 + 1e-15).all() and np.allclose(n1[n0 > 1], 1.0, atol=1e-15)
+    assert np.array_equal(Rp[:, n0 <= 1], R[:, n0 <= 1])
+    assert np.allclose(orc.prox_unit_columns(Rp), Rp, atol=1e-15)   # idempotent
+    cos = (R * Rp).sum(axis=0) / (n0 * n1)
+    assert np.allclose(cos, 1.0, atol=1e-14)                          # direction preserved
+
+
 # ----------------------------------------------------------------------------- apply
 def test_apply_is_the_sum_of_outer_products_and_is_additive_linear_permutation_invariant():
     J, D, K = 5, 7, 9
