@@ -319,12 +319,12 @@ def main():
     result_host = torch.empty(128, dtype=torch.uint8).pin_memory()
     d2h = result_host.numel()
 
-    def e2e_step(t):
+    from paper_1511_08486_b200 import binding as Bd
+    host_aux = [Bd.make_aux(**{k: v for k, v in hb.items() if k != "X"}) for hb in host_batches]
+
+    def e2e_step(t):   # one C-ABI call: host inputs in, step, committed header (clock, shapes) back to the host
         b = t % wl.pool
-        for k, hv in host_batches[b].items():
-            wl.batches[b][k].copy_(hv, non_blocking=True)
-        wl.step(t, eta=eta)
-        result_host.copy_(wl.sf_buf[:128], non_blocking=True)        # the committed header (clock, shapes)
+        wl.ctx.step_host(wl.W, host_batches[b].get("X"), host_aux[b], wl.sf_buf, eta, clock=t, header_host=result_host)
     for t in range(3):
         e2e_step(t)
     barrier()

@@ -142,6 +142,16 @@ int sfb_apply(sfb_ctx* ctx, void* W, const void* sf_buf, float eta, int32_t K);
 int sfb_step(sfb_ctx* ctx, void* W, const void* X, const sfb_aux* aux, void* sf_buf, float eta, int32_t K,
              uint32_t clock);
 
+/* sfb_step for callers whose minibatch lives in HOST memory: X_host and the arrays inside aux_host
+ * are host pointers (pinned memory keeps the copies asynchronous) with the shapes sfb_step
+ * documents; they are copied to context-owned device staging buffers on the context's stream
+ * (allocated on first use, grown on demand), the step runs, and the 128-byte header the step
+ * committed to the SF buffer is copied back into header_host (may be NULL).  W and sf_buf stay
+ * device pointers.  Returns without synchronising; header_host is valid after the stream has
+ * been synchronised (sfb_status does). */
+int sfb_step_host(sfb_ctx* ctx, void* W, const void* X_host, const sfb_aux* aux_host, void* sf_buf, float eta,
+                  int32_t K, uint32_t clock, void* header_host);
+
 /* Proximal operator applied after the update (Section 2.1: prox_{eta h}; Section 3: "finally each
  * worker applies the proximal operator").  SFB_SC: h is the indicator of ||W_k||_2 <= 1 for every
  * column (atom) k, so each column whose norm exceeds 1 is divided by its norm and the others are

@@ -23,7 +23,7 @@ EXPORTS = (
     "sfb_create", "sfb_destroy", "sfb_sf_buffer_bytes", "sfb_ld", "sfb_compute_factors", "sfb_pack",
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
     "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
-    "sfb_halton_peers", "sfb_ssp_may_proceed", "sfb_prox",
+    "sfb_halton_peers", "sfb_ssp_may_proceed", "sfb_prox", "sfb_step_host",
 )
 
 
@@ -73,6 +73,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_apply.restype = C.c_int
     lib.sfb_step.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, C.c_float, C.c_int32, C.c_uint32]
     lib.sfb_step.restype = C.c_int
+    lib.sfb_step_host.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, C.c_float, C.c_int32, C.c_uint32, vp]
+    lib.sfb_step_host.restype = C.c_int
     lib.sfb_prox.argtypes = [vp, vp]
     lib.sfb_prox.restype = C.c_int
     lib.sfb_invalidate.argtypes = [vp]
@@ -205,6 +207,12 @@ class Context:
     def step(self, W, X, aux: sfb_aux, sf_buf, eta: float, K: int | None = None, clock: int = 0):
         self._chk(self._lib.sfb_step(self._h, _ptr(W), _ptr(X), C.byref(aux), _ptr(sf_buf), eta,
                                      self.K if K is None else K, clock), "sfb_step")
+
+    def step_host(self, W, X_host, aux_host: sfb_aux, sf_buf, eta: float, K: int | None = None, clock: int = 0,
+                  header_host=None):
+        """sfb_step with the minibatch in host memory (tensors on the CPU, ideally pinned)."""
+        self._chk(self._lib.sfb_step_host(self._h, _ptr(W), _ptr(X_host), C.byref(aux_host), _ptr(sf_buf), eta,
+                                          self.K if K is None else K, clock, _ptr(header_host)), "sfb_step_host")
 
     def prox(self, W):
         self._chk(self._lib.sfb_prox(self._h, _ptr(W)), "sfb_prox")

@@ -19,6 +19,8 @@ struct sfb_ctx {
   int ldz;
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
+  char* host_stage[6];      // sfb_step_host: device copies of the step's host inputs (allocated on first use)
+  size_t host_stage_bytes[6];
   __nv_bfloat16* w_shadow;  // bf16 path: bf16 copy of W, refreshed by the apply
   const void* shadow_of;    // W pointer the shadow currently mirrors (nullptr = stale)
   UmmaPlan* umma;           // tensor-core plan (tensor maps), TF32 / BF16 paths
@@ -231,6 +233,8 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->z_ws) cudaFree(c->z_ws);
   if (c->wt_ws) cudaFree(c->wt_ws);
   if (c->a_dense) cudaFree(c->a_dense);
+  for (int i = 0; i < 6; ++i)
+    if (c->host_stage[i]) cudaFree(c->host_stage[i]);
   if (c->w_shadow) cudaFree(c->w_shadow);
   delete c;
   return SFB_OK;
@@ -379,6 +383,71 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
     c->prof_n++;
   }
   return r;
+}
+
+// Copies `bytes` from host memory into staging buffer `slot` (grown on demand) on the context's stream.
+static int stage_in(sfb_ctx* c, int slot, const void* host, size_t bytes, const void** dev) {
+  if (bytes > c->host_stage_bytes[slot]) {
+    if (c->host_stage[slot]) {
+      cudaStreamSynchronize(c->stream);   // the old buffer may still be in use by an earlier step
+      cudaFree(c->host_stage[slot]);
+      c->host_stage[slot] = nullptr;
+      c->host_stage_bytes[slot] = 0;
+    }
+    if (cudaMalloc(&c->host_stage[slot], bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return SFB_ERR_ALLOC;
+    }
+    c->host_stage_bytes[slot] = bytes;
+  }
+  if (cudaMemcpyAsync(c->host_stage[slot], host, bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+    return SFB_ERR_CUDA;
+  *dev = c->host_stage[slot];
+  return SFB_OK;
+}
+
+int sfb_step_host(sfb_ctx* c, void* W, const void* X_host, const sfb_aux* aux_host, void* sf_buf, float eta, int32_t K,
+                  uint32_t clock, void* header_host) {
+  if (c == nullptr || W == nullptr || sf_buf == nullptr || aux_host == nullptr) return SFB_ERR_ARG;
+  const sfb_desc& d = c->d;
+  const size_t es = (size_t)c->l.es, Kt = (size_t)c->K;
+  sfb_aux dev_aux;
+  memset(&dev_aux, 0, sizeof(dev_aux));
+  const void* X_dev = nullptr;
+  int r;
+  if (d.model != SFB_SC) {
+    if (X_host == nullptr) return SFB_ERR_ARG;
+    if ((r = stage_in(c, 0, X_host, Kt * d.D * es, &X_dev)) != SFB_OK) return r;
+  }
+  const void* p = nullptr;
+  if (d.model == SFB_MLR) {
+    if (aux_host->labels == nullptr) return SFB_ERR_ARG;
+    if ((r = stage_in(c, 1, aux_host->labels, Kt * 4, &p)) != SFB_OK) return r;
+    dev_aux.labels = static_cast<const int32_t*>(p);
+  } else if (d.model == SFB_DML) {
+    if (aux_host->Xb == nullptr || aux_host->similar == nullptr) return SFB_ERR_ARG;
+    if ((r = stage_in(c, 1, aux_host->Xb, Kt * d.D * es, &p)) != SFB_OK) return r;
+    dev_aux.Xb = p;
+    if ((r = stage_in(c, 2, aux_host->similar, Kt, &p)) != SFB_OK) return r;
+    dev_aux.similar = static_cast<const uint8_t*>(p);
+  } else {
+    if (!aux_host->rowptr || !aux_host->idx || !aux_host->val || !aux_host->Xdata) return SFB_ERR_ARG;
+    const size_t nnz = aux_host->rowptr[Kt];   // host memory: readable here
+    if (nnz > d.nnz_capacity) return SFB_ERR_SHAPE;
+    if ((r = stage_in(c, 1, aux_host->rowptr, (Kt + 1) * 4, &p)) != SFB_OK) return r;
+    dev_aux.rowptr = static_cast<const uint32_t*>(p);
+    if ((r = stage_in(c, 2, aux_host->idx, (nnz > 0 ? nnz : 1) * 4, &p)) != SFB_OK) return r;
+    dev_aux.idx = static_cast<const uint32_t*>(p);
+    if ((r = stage_in(c, 3, aux_host->val, (nnz > 0 ? nnz : 1) * 4, &p)) != SFB_OK) return r;
+    dev_aux.val = p;
+    if ((r = stage_in(c, 4, aux_host->Xdata, Kt * d.J * 4, &p)) != SFB_OK) return r;
+    dev_aux.Xdata = p;
+  }
+  if ((r = sfb_step(c, W, X_dev, &dev_aux, sf_buf, eta, K, clock)) != SFB_OK) return r;
+  if (header_host != nullptr &&
+      cudaMemcpyAsync(header_host, sf_buf, 128, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+    return SFB_ERR_CUDA;
+  return SFB_OK;
 }
 
 }  // extern "C"

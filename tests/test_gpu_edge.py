@@ -1,0 +1,117 @@
+"""Edge cases and the host-buffer entry point, through the C ABI on the GPU."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sfb_oracle as orc
+from sfbgen import get_config, make_inputs, scaled
+from tests.test_gpu_parity import _workload, check_config
+from tests.util import to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,path,over", [
+    ("C0", "f32", {}),
+    ("C2", "f32", dict(J=40, D=300, P=2, B=6)),
+    ("C3", "f32", dict(J=64, D=400, P=2, B=4, density=0.1)),
+    ("C4", "bf16", dict(J=256, D=512, P=2, B=64, pool=1, labels="uniform")),
+])
+def test_step_host_equals_step(name, path, over):
+    """sfb_step_host (minibatch in pinned host memory) leaves exactly the W and SF buffer of sfb_step."""
+    from paper_1511_08486_b200 import binding as B
+    cfg = scaled(name, **over) if over else get_config(name)
+    cfg["path"] = path
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, path)
+    try:
+        wl.step(0, eta=0.05)
+        torch.cuda.synchronize()
+        W_ref, buf_ref = wl.W.clone(), wl.sf_buf.clone()
+        wl.reset()
+        wl.sf_buf.zero_()
+        t = wl.batches[0]
+        host = {k: v.cpu().pin_memory() for k, v in t.items() if isinstance(v, torch.Tensor)}
+        aux = B.make_aux(**{k: v for k, v in host.items() if k != "X"})
+        header = torch.zeros(128, dtype=torch.uint8).pin_memory()
+        wl.ctx.step_host(wl.W, host.get("X"), aux, wl.sf_buf, 0.05, clock=0, header_host=header)
+        assert wl.ctx.status() == 0                      # synchronises
+        assert torch.equal(wl.W, W_ref) and torch.equal(wl.sf_buf, buf_ref)
+        h = orc.parse_header(header.numpy())
+        assert h["magic"] == orc.MAGIC and h["J"] == cfg["J"] and h["P"] == cfg["P"]
+    finally:
+        wl.close()
+
+
+def test_single_worker_single_sample_and_single_class():
+    check_config(scaled("C0", J=10, D=64, P=1, B=1), "f32", eta=1.0, steps=1)
+    # J = 1: softmax is identically 1, so u = 1 - 1 = 0 and W must not move
+    cfg = scaled("C0", J=1, D=16, P=2, B=3)
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.step(0, eta=1.0)
+        torch.cuda.synchronize()
+        assert torch.equal(wl.W, wl.W0)
+        _, U, _ = orc.unpack(wl.sf_buf.cpu().numpy())
+        assert not U.any()
+    finally:
+        wl.close()
+
+
+def test_dml_all_pairs_beyond_the_margin_leaves_dissimilar_rows_zero():
+    cfg = scaled("C2", J=24, D=200, P=2, B=4)
+    cfg["w_std"] = 1.0                                    # |L d|^2 >> margin: every dissimilar pair inactive
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.compute_factors(0)
+        torch.cuda.synchronize()
+        U = to_f64(wl.U)
+        sim = inputs["similar"].astype(bool)
+        assert not U[~sim].any() and U[sim].any()
+    finally:
+        wl.close()
+
+
+def test_sparse_codes_with_empty_rows_and_an_empty_worker():
+    cfg = scaled("C3", J=48, D=300, P=3, B=4, density=0.1)
+    inputs = make_inputs(cfg)
+    rp, ix, vl = inputs["rowptr"][0].astype(np.int64), inputs["idx"][0], inputs["val"][0]
+    # empty the codes of sample 1 and of every sample of worker 2 (samples 8..11)
+    keep = np.ones(ix.size, bool)
+    for i in [1] + list(range(8, 12)):
+        keep[rp[i]:rp[i + 1]] = False
+    counts = np.diff(rp)
+    counts[[1, 8, 9, 10, 11]] = 0
+    inputs["rowptr"][0] = np.concatenate([[0], np.cumsum(counts)]).astype(np.uint32)
+    inputs["idx"][0], inputs["val"][0] = ix[keep], vl[keep]
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.step(0, eta=0.05)
+        torch.cuda.synchronize()
+        W_or, U_or, _ = orc.step(orc.MODEL_SC, inputs["W"], dict(rowptr=inputs["rowptr"][0], idx=inputs["idx"][0],
+                                                                  val=inputs["val"][0], Xdata=inputs["Xdata"][0]), 0.05)
+        W0 = inputs["W"].astype(np.float64)
+        err = np.linalg.norm((to_f64(wl.W) - W0) - (W_or - W0)) / np.linalg.norm(W_or - W0)
+        assert err <= 1e-5 + 2.0 ** -24 * np.linalg.norm(W0) / np.linalg.norm(W_or - W0)
+        h, U, (rp2, ix2, vl2) = orc.unpack(wl.sf_buf.cpu().numpy())
+        assert np.array_equal(rp2, inputs["rowptr"][0]) and np.array_equal(ix2, inputs["idx"][0])
+        assert np.allclose(U[1], -inputs["Xdata"][0][1], atol=0)       # empty code: u = -x exactly
+        assert wl.ctx.status() == 0
+    finally:
+        wl.close()
+
+
+def test_sparse_capacity_overflow_sets_status():
+    from paper_1511_08486_b200 import binding as B
+    cfg = scaled("C3", J=32, D=200, P=2, B=4, density=0.2)
+    inputs = make_inputs(cfg)
+    inputs["nnz_capacity"] = 2 * 32                         # far below the real nonzero count per worker
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.compute_factors(0)
+        wl.pack(0)
+        assert wl.ctx.status() & B.SFB_DEV_CAPACITY
+    finally:
+        wl.close()
