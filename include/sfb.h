@@ -144,8 +144,9 @@ int sfb_step(sfb_ctx* ctx, void* W, const void* X, const sfb_aux* aux, void* sf_
 
 /* sfb_step for callers whose minibatch lives in HOST memory: X_host and the arrays inside aux_host
  * are host pointers (pinned memory keeps the copies asynchronous) with the shapes sfb_step
- * documents; they are copied to context-owned device staging buffers on the context's stream
- * (allocated on first use, grown on demand), the step runs, and the 128-byte header the step
+ * documents; they are copied to context-owned device staging buffers (two sets, allocated on
+ * first use, grown on demand) on a side stream, so the copy for one call overlaps the kernels of
+ * the previous call; the step then runs on the context's stream, and the 128-byte header the step
  * committed to the SF buffer is copied back into header_host (may be NULL).  W and sf_buf stay
  * device pointers.  Returns without synchronising; header_host is valid after the stream has
  * been synchronised (sfb_status does). */

@@ -19,8 +19,14 @@ struct sfb_ctx {
   int ldz;
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
-  char* host_stage[6];      // sfb_step_host: device copies of the step's host inputs (allocated on first use)
-  size_t host_stage_bytes[6];
+  // sfb_step_host: two sets of device staging buffers for the step's host inputs (allocated on first
+  // use), filled on a side stream so that the copy of step t+1 overlaps the kernels of step t
+  char* host_stage[2][6];
+  size_t host_stage_bytes[2][6];
+  cudaStream_t copy_stream;
+  cudaEvent_t copied[2], consumed[2];
+  bool host_ready;
+  uint64_t host_steps;
   __nv_bfloat16* w_shadow;  // bf16 path: bf16 copy of W, refreshed by the apply
   const void* shadow_of;    // W pointer the shadow currently mirrors (nullptr = stale)
   UmmaPlan* umma;           // tensor-core plan (tensor maps), TF32 / BF16 paths
@@ -233,8 +239,17 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->z_ws) cudaFree(c->z_ws);
   if (c->wt_ws) cudaFree(c->wt_ws);
   if (c->a_dense) cudaFree(c->a_dense);
-  for (int i = 0; i < 6; ++i)
-    if (c->host_stage[i]) cudaFree(c->host_stage[i]);
+  for (int k = 0; k < 2; ++k)
+    for (int i = 0; i < 6; ++i)
+      if (c->host_stage[k][i]) cudaFree(c->host_stage[k][i]);
+  if (c->host_ready) {
+    cudaStreamSynchronize(c->copy_stream);
+    for (int k = 0; k < 2; ++k) {
+      cudaEventDestroy(c->copied[k]);
+      cudaEventDestroy(c->consumed[k]);
+    }
+    cudaStreamDestroy(c->copy_stream);
+  }
   if (c->w_shadow) cudaFree(c->w_shadow);
   delete c;
   return SFB_OK;
@@ -385,24 +400,25 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   return r;
 }
 
-// Copies `bytes` from host memory into staging buffer `slot` (grown on demand) on the context's stream.
-static int stage_in(sfb_ctx* c, int slot, const void* host, size_t bytes, const void** dev) {
-  if (bytes > c->host_stage_bytes[slot]) {
-    if (c->host_stage[slot]) {
+// Copies `bytes` from host memory into staging buffer `slot` of set `set` (grown on demand) on the copy stream.
+static int stage_in(sfb_ctx* c, int set, int slot, const void* host, size_t bytes, const void** dev) {
+  if (bytes > c->host_stage_bytes[set][slot]) {
+    if (c->host_stage[set][slot]) {
       cudaStreamSynchronize(c->stream);   // the old buffer may still be in use by an earlier step
-      cudaFree(c->host_stage[slot]);
-      c->host_stage[slot] = nullptr;
-      c->host_stage_bytes[slot] = 0;
+      cudaStreamSynchronize(c->copy_stream);
+      cudaFree(c->host_stage[set][slot]);
+      c->host_stage[set][slot] = nullptr;
+      c->host_stage_bytes[set][slot] = 0;
     }
-    if (cudaMalloc(&c->host_stage[slot], bytes) != cudaSuccess) {
+    if (cudaMalloc(&c->host_stage[set][slot], bytes) != cudaSuccess) {
       cudaGetLastError();
       return SFB_ERR_ALLOC;
     }
-    c->host_stage_bytes[slot] = bytes;
+    c->host_stage_bytes[set][slot] = bytes;
   }
-  if (cudaMemcpyAsync(c->host_stage[slot], host, bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+  if (cudaMemcpyAsync(c->host_stage[set][slot], host, bytes, cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess)
     return SFB_ERR_CUDA;
-  *dev = c->host_stage[slot];
+  *dev = c->host_stage[set][slot];
   return SFB_OK;
 }
 
@@ -415,35 +431,50 @@ int sfb_step_host(sfb_ctx* c, void* W, const void* X_host, const sfb_aux* aux_ho
   memset(&dev_aux, 0, sizeof(dev_aux));
   const void* X_dev = nullptr;
   int r;
+  if (!c->host_ready) {
+    if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return SFB_ERR_CUDA;
+    for (int k = 0; k < 2; ++k)
+      if (cudaEventCreateWithFlags(&c->copied[k], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&c->consumed[k], cudaEventDisableTiming) != cudaSuccess)
+        return SFB_ERR_CUDA;
+    c->host_ready = true;
+  }
+  const int set = (int)(c->host_steps & 1);
+  // this set's buffers were last read by the step two calls ago
+  if (c->host_steps >= 2 && cudaStreamWaitEvent(c->copy_stream, c->consumed[set], 0) != cudaSuccess) return SFB_ERR_CUDA;
   if (d.model != SFB_SC) {
     if (X_host == nullptr) return SFB_ERR_ARG;
-    if ((r = stage_in(c, 0, X_host, Kt * d.D * es, &X_dev)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 0, X_host, Kt * d.D * es, &X_dev)) != SFB_OK) return r;
   }
   const void* p = nullptr;
   if (d.model == SFB_MLR) {
     if (aux_host->labels == nullptr) return SFB_ERR_ARG;
-    if ((r = stage_in(c, 1, aux_host->labels, Kt * 4, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 1, aux_host->labels, Kt * 4, &p)) != SFB_OK) return r;
     dev_aux.labels = static_cast<const int32_t*>(p);
   } else if (d.model == SFB_DML) {
     if (aux_host->Xb == nullptr || aux_host->similar == nullptr) return SFB_ERR_ARG;
-    if ((r = stage_in(c, 1, aux_host->Xb, Kt * d.D * es, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 1, aux_host->Xb, Kt * d.D * es, &p)) != SFB_OK) return r;
     dev_aux.Xb = p;
-    if ((r = stage_in(c, 2, aux_host->similar, Kt, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 2, aux_host->similar, Kt, &p)) != SFB_OK) return r;
     dev_aux.similar = static_cast<const uint8_t*>(p);
   } else {
     if (!aux_host->rowptr || !aux_host->idx || !aux_host->val || !aux_host->Xdata) return SFB_ERR_ARG;
     const size_t nnz = aux_host->rowptr[Kt];   // host memory: readable here
     if (nnz > d.nnz_capacity) return SFB_ERR_SHAPE;
-    if ((r = stage_in(c, 1, aux_host->rowptr, (Kt + 1) * 4, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 1, aux_host->rowptr, (Kt + 1) * 4, &p)) != SFB_OK) return r;
     dev_aux.rowptr = static_cast<const uint32_t*>(p);
-    if ((r = stage_in(c, 2, aux_host->idx, (nnz > 0 ? nnz : 1) * 4, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 2, aux_host->idx, (nnz > 0 ? nnz : 1) * 4, &p)) != SFB_OK) return r;
     dev_aux.idx = static_cast<const uint32_t*>(p);
-    if ((r = stage_in(c, 3, aux_host->val, (nnz > 0 ? nnz : 1) * 4, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 3, aux_host->val, (nnz > 0 ? nnz : 1) * 4, &p)) != SFB_OK) return r;
     dev_aux.val = p;
-    if ((r = stage_in(c, 4, aux_host->Xdata, Kt * d.J * 4, &p)) != SFB_OK) return r;
+    if ((r = stage_in(c, set, 4, aux_host->Xdata, Kt * d.J * 4, &p)) != SFB_OK) return r;
     dev_aux.Xdata = p;
   }
+  if (cudaEventRecord(c->copied[set], c->copy_stream) != cudaSuccess) return SFB_ERR_CUDA;
+  if (cudaStreamWaitEvent(c->stream, c->copied[set], 0) != cudaSuccess) return SFB_ERR_CUDA;
   if ((r = sfb_step(c, W, X_dev, &dev_aux, sf_buf, eta, K, clock)) != SFB_OK) return r;
+  if (cudaEventRecord(c->consumed[set], c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  ++c->host_steps;
   if (header_host != nullptr &&
       cudaMemcpyAsync(header_host, sf_buf, 128, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
     return SFB_ERR_CUDA;
