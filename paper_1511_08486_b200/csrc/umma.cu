@@ -23,6 +23,12 @@
 #include "umma.cuh"
 #include "umma_api.cuh"
 
+// The apply epilogue writes the new fp32 W with TMA bulk stores from its staging blocks (fewer store
+// instructions than per-thread 16-byte stores); -DSFB_LSU_STORE_W switches back to plain stores.
+#ifndef SFB_LSU_STORE_W
+#define SFB_TMA_STORE_W 1
+#endif
+
 namespace sfb {
 
 // extra passes implemented in finish.cu
@@ -118,7 +124,8 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 //          one 3-D TMA per chunk, with zero fill on every ragged edge.
 template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
   constexpr int CH = 128 / ES;                 // values per 128-byte chunk
   constexpr int BK = CH * KA;                  // reduction steps per pipeline stage
   constexpr int UMMA_K = 32 / ES;              // reduction steps per instruction (16 bf16 / 8 tf32)
@@ -518,8 +525,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               float4 w = wv[g];
               w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
               w.z = fmaf(-p.eta, a.z, w.z); w.w = fmaf(-p.eta, a.w, w.w);
+#ifdef SFB_TMA_STORE_W
+              *reinterpret_cast<float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2)) = w;   // goes out by TMA below
+#elif !defined(SFB_EXP_SKIP_W_STORE)
               __stcs(reinterpret_cast<float4*>(rowp[g] + c), w);   // streamed: keep L2 for the factors
+#endif
+#ifdef SFB_EXP_SKIP_SHADOW_STORE
+              if (p.shadow != nullptr && w.x == 123.456f) {
+#else
               if (p.shadow != nullptr) {
+#endif
                 __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
                 uint2 pk;
                 pk.x = *reinterpret_cast<uint32_t*>(&lo);
@@ -533,6 +548,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
 #pragma unroll
         for (int g = 0; g < 8; ++g) wv[g] = wn[g];
+#ifdef SFB_TMA_STORE_W
+        if (APPLY) {   // the 32 x 32 block of new W sits in the staging block, swizzled as the tensor map expects
+          ptx::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            ptx::tma_store_2d(&tmW, stage, nt * BN + col_in_tile, mt * BM + quarter * 32);
+            ptx::tma_store_commit();
+            ptx::tma_store_wait_read();   // the block is rewritten by the next pass
+          }
+        }
+#endif
         __syncwarp();
       }
       ptx::tc_fence_before();
@@ -551,6 +577,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     printf("EXPCLK apply=%d cycles=%lld ns=%llu MHz=%.0f\n", (int)APPLY, clock64() - exp_c0, exp_t1 - exp_t0,
            1e3 * (double)(clock64() - exp_c0) / (double)(exp_t1 - exp_t0));
   }
+#endif
+#ifdef SFB_TMA_STORE_W
+  if (APPLY && warp >= 2 && lane == 0) ptx::tma_store_wait_all();
 #endif
   ptx::tc_fence_before();
   __syncthreads();
@@ -612,7 +641,8 @@ int pow2_at_least(int n) {
 }
 
 template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI>
-int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, int num_sms) {
+int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w, const GemmParams& p,
+                int num_sms) {
   constexpr int stage_bytes = (BM + BN / CG) * 128 * KA;
   constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
   constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
@@ -642,7 +672,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
   const int tiles = p.m_tiles * p.n_tiles;
   if (CG == 1) {
     const int grid = tiles < num_sms ? tiles : num_sms;
-    kernel<<<grid, NUM_THREADS, smem, s>>>(a, b, p);
+    kernel<<<grid, NUM_THREADS, smem, s>>>(a, b, w, p);
   } else {
     const int clusters = tiles < max_clusters ? tiles : max_clusters;
     cudaLaunchConfig_t cfg;
@@ -655,7 +685,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cfg.attrs = at; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kernel, a, b, p) != cudaSuccess) return SFB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kernel, a, b, w, p) != cudaSuccess) return SFB_ERR_CUDA;
   }
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
@@ -668,21 +698,22 @@ struct Variant {
 };
 
 template <int ES, bool APPLY, int EPI>
-int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p,
-                int num_sms) {
+int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w,
+                const GemmParams& p, int num_sms) {
   if (v.cg == 2) {
-    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, p, num_sms);
-    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, p, num_sms);
-    return launch_gemm<ES, APPLY, 256, 2, 1, false, EPI>(s, a, b, p, num_sms);
+    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, w, p, num_sms);
+    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, w, p, num_sms);
+    return launch_gemm<ES, APPLY, 256, 2, 1, false, EPI>(s, a, b, w, p, num_sms);
   }
-  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false, EPI>(s, a, b, p, num_sms);
-  return launch_gemm<ES, APPLY, 128, 1, 1, false, EPI>(s, a, b, p, num_sms);
+  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false, EPI>(s, a, b, w, p, num_sms);
+  return launch_gemm<ES, APPLY, 128, 1, 1, false, EPI>(s, a, b, w, p, num_sms);
 }
 
 template <bool APPLY, int EPI>
 int dispatch_gemm(cudaStream_t s, int es, const Variant& v, const CUtensorMap& a, const CUtensorMap& b,
-                  const GemmParams& p, int num_sms) {
-  return es == 2 ? dispatch_es<2, APPLY, EPI>(s, v, a, b, p, num_sms) : dispatch_es<4, APPLY, EPI>(s, v, a, b, p, num_sms);
+                  const CUtensorMap& w, const GemmParams& p, int num_sms) {
+  return es == 2 ? dispatch_es<2, APPLY, EPI>(s, v, a, b, w, p, num_sms)
+                 : dispatch_es<4, APPLY, EPI>(s, v, a, b, w, p, num_sms);
 }
 
 }  // namespace
@@ -784,8 +815,8 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, v.bn / v.cg, 1,
                        v.fold, v.ka, false))
     return SFB_ERR_CUDA;
-  return stats != nullptr ? dispatch_gemm<false, 1>(s, es, v, ta, tb, p, pl->num_sms)
-                          : dispatch_gemm<false, 0>(s, es, v, ta, tb, p, pl->num_sms);
+  return stats != nullptr ? dispatch_gemm<false, 1>(s, es, v, ta, tb, ta, p, pl->num_sms)
+                          : dispatch_gemm<false, 0>(s, es, v, ta, tb, ta, p, pl->num_sms);
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
@@ -862,7 +893,19 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   if (!encode_rows_map(&tv, es, v_rows.base, d.D, d.B, workers, (long long)v_rows.ld * es, v_rows.worker_stride, p.k_bb,
                        p.k_wp, v.fold, (v.bn / v.cg) / CH, es == 4))
     return SFB_ERR_CUDA;
-  return dispatch_gemm<true, 0>(s, es, v, tu, tv, p, pl->num_sms);
+  // fp32 W as a 2-D map with 32 x 32 boxes (128-byte swizzle) for the epilogue's TMA stores
+  CUtensorMap tw;
+  {
+    cuuint64_t dims[2] = {(cuuint64_t)d.D, (cuuint64_t)d.J};
+    cuuint64_t strides[1] = {(cuuint64_t)d.D * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    if (get_encode()(&tw, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, W, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SFB_ERR_CUDA;
+  }
+  return dispatch_gemm<true, 0>(s, es, v, tu, tv, tw, p, pl->num_sms);
 }
 
 }  // namespace sfb
