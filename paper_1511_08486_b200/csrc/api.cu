@@ -139,7 +139,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     const RowMap a = dense_codes(c);
     ACC(launch_densify_codes(c->stream, codes, a, c->K, d.D, c->dev_status));
     ACC(umma_forward_rows(c->umma, c->stream, W, a, u, c->dev_status));
-    ACC(launch_finish_sc(c->stream, u, reinterpret_cast<const float*>(aux->Xdata), c->K, d.J));
+    ACC(launch_finish_sc(c->stream, u, u, reinterpret_cast<const float*>(aux->Xdata), c->K, d.J));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {

@@ -68,10 +68,13 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
                      const int* dev_status);
 
 // MLR epilogue: u = softmax(z) - onehot(label).  z rows are fp32; u rows fp32 or bf16 (u.es).
-int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status);
+// z may be `nsplit` partial products (split s at z + s * split_stride_bytes), summed in split order.
+int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
+                      int nsplit = 1, long long split_stride_bytes = 0);
 
 // DML epilogue: u = +z (similar) or -z * [|z|^2 < margin] (dissimilar).
-int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J);
+int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
+                      int nsplit = 1, long long split_stride_bytes = 0);
 
 // Copies K rows of `cols` values from src to dst rows (same value type), zero-filling dst pad columns.
 int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols);
@@ -110,7 +113,9 @@ int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, in
 int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status);
 
 // SC epilogue on dense products: u = z - x in place (u rows hold z), pad columns zero.
-int launch_finish_sc(cudaStream_t s, RowMap u, const float* Xdata, int K, int J);
+// z: products (possibly `nsplit` partials); u = sum of partials - x.
+int launch_finish_sc(cudaStream_t s, RowMap z, RowMap u, const float* Xdata, int K, int J, int nsplit = 1,
+                     long long split_stride_bytes = 0);
 
 // Column-norm projection: every column of W with 2-norm above 1 is divided by its norm (in place).
 int launch_prox_unit_columns(cudaStream_t s, float* W, int J, int D);

@@ -43,6 +43,17 @@ __device__ float block_sum(float v, float* red) {
   return warp_sum(r);
 }
 
+// Four products starting at column j: the sum, in split order, of the partial products of a reduction
+// that the GEMM cut in `nsplit` ranges (partial s lives `stride` floats after partial s - 1).
+__device__ __forceinline__ float4 ldz4(const float* zr, int j, int nsplit, long long stride) {
+  float4 t = *reinterpret_cast<const float4*>(zr + j);
+  for (int s = 1; s < nsplit; ++s) {
+    const float4 q = *reinterpret_cast<const float4*>(zr + s * stride + j);
+    t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w;
+  }
+  return t;
+}
+
 // Stores 4 consecutive values starting at column j (j % 4 == 0, j + 3 < ld).
 __device__ __forceinline__ void store_u4(char* row, int j, float4 v, int es) {
   if (es == 4) {
@@ -58,7 +69,7 @@ __device__ __forceinline__ void store_u4(char* row, int j, float4 v, int es) {
 
 // z rows are fp32 with ld a multiple of 4; values beyond J inside the last float4 are ignored.
 __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, const int32_t* __restrict__ labels,
-                                                                 int K, int J, int cache_floats, int* dev_status) {
+                                                                 int K, int J, int cache_floats, int* dev_status, int nsplit, long long zstride) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -71,7 +82,7 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
 
   float m = -INFINITY;
   for (int q = threadIdx.x; q < J4; q += blockDim.x) {
-    float4 t = *reinterpret_cast<const float4*>(zr + q * 4);
+    float4 t = ldz4(zr, q * 4, nsplit, zstride);
     const int j = q * 4;
     if (j + 1 >= J) t.y = -INFINITY;
     if (j + 2 >= J) t.z = -INFINITY;
@@ -89,7 +100,7 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
     if (cached) {
       t = *reinterpret_cast<const float4*>(cache + j);
     } else {
-      t = *reinterpret_cast<const float4*>(zr + j);
+      t = ldz4(zr, j, nsplit, zstride);
       if (j + 1 >= J) t.y = -INFINITY;
       if (j + 2 >= J) t.z = -INFINITY;
       if (j + 3 >= J) t.w = -INFINITY;
@@ -113,7 +124,7 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
       if (cached) {
         t = *reinterpret_cast<const float4*>(cache + j);
       } else {
-        t = *reinterpret_cast<const float4*>(zr + j);
+        t = ldz4(zr, j, nsplit, zstride);
         t.x = exp2f(fmaf(t.x, kLog2e, -mb)); t.y = exp2f(fmaf(t.y, kLog2e, -mb));
         t.z = exp2f(fmaf(t.z, kLog2e, -mb)); t.w = exp2f(fmaf(t.w, kLog2e, -mb));
       }
@@ -131,7 +142,7 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
 }
 
 __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, const uint8_t* __restrict__ similar,
-                                                                 float margin, int K, int J, int cache_floats) {
+                                                                 float margin, int K, int J, int cache_floats, int nsplit, long long zstride) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -143,7 +154,7 @@ __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, co
 
   float n = 0.f;
   for (int q = threadIdx.x; q < J4; q += blockDim.x) {
-    float4 t = *reinterpret_cast<const float4*>(zr + q * 4);
+    float4 t = ldz4(zr, q * 4, nsplit, zstride);
     const int j = q * 4;
     if (j + 1 >= J) t.y = 0.f;
     if (j + 2 >= J) t.z = 0.f;
@@ -160,7 +171,7 @@ __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, co
     const int j = q * 4;
     float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
     if (q < J4 && g != 0.f) {
-      t = cached ? *reinterpret_cast<const float4*>(cache + j) : *reinterpret_cast<const float4*>(zr + j);
+      t = cached ? *reinterpret_cast<const float4*>(cache + j) : ldz4(zr, j, nsplit, zstride);
       t.x *= g; t.y *= g; t.z *= g; t.w *= g;
       if (j + 1 >= J) t.y = 0.f;
       if (j + 2 >= J) t.z = 0.f;
@@ -336,7 +347,8 @@ int fin_cache_floats(int J) {
 
 }  // namespace
 
-int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status) {
+int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
+                      int nsplit, long long split_stride_bytes) {
   const int cf = fin_cache_floats(J);
   static bool attr_done = false;
   if (!attr_done) {
@@ -344,11 +356,12 @@ int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels,
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     attr_done = true;
   }
-  finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status);
+  finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status, nsplit, split_stride_bytes / 4);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
-int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J) {
+int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
+                      int nsplit, long long split_stride_bytes) {
   const int cf = fin_cache_floats(J);
   static bool attr_done = false;
   if (!attr_done) {
@@ -356,7 +369,7 @@ int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     attr_done = true;
   }
-  finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf);
+  finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf, nsplit, split_stride_bytes / 4);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

@@ -123,14 +123,20 @@ __global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, i
   }
 }
 
-__global__ void __launch_bounds__(256) finish_sc_kernel(RowMap u, const float* __restrict__ Xdata, int K, int J) {
+__global__ void __launch_bounds__(256) finish_sc_kernel(RowMap zr, RowMap u, const float* __restrict__ Xdata, int K, int J,
+                                                        int nsplit, long long zstride) {
   const int units = u.ld >> 2;
   const long long total = (long long)K * units;
   for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
        g += (long long)gridDim.x * blockDim.x) {
     const int i = (int)(g / units), j = (int)(g % units) * 4;
     float4* p = reinterpret_cast<float4*>(u.row(i) + (size_t)j * 4);
-    float4 z = *p;
+    const float* zp = reinterpret_cast<const float*>(zr.row(i)) + j;
+    float4 z = *reinterpret_cast<const float4*>(zp);
+    for (int sp = 1; sp < nsplit; ++sp) {
+      const float4 q = *reinterpret_cast<const float4*>(zp + sp * zstride);
+      z.x += q.x; z.y += q.y; z.z += q.z; z.w += q.w;
+    }
     const float* x = Xdata + (size_t)i * J;
     z.x = (j < J) ? z.x - x[j] : 0.f;
     z.y = (j + 1 < J) ? z.y - x[j + 1] : 0.f;
@@ -303,10 +309,11 @@ int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, 
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
-int launch_finish_sc(cudaStream_t s, RowMap u, const float* Xdata, int K, int J) {
+int launch_finish_sc(cudaStream_t s, RowMap z, RowMap u, const float* Xdata, int K, int J, int nsplit,
+                     long long split_stride_bytes) {
   const long long total = (long long)K * (u.ld >> 2);
   const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
-  finish_sc_kernel<<<blocks, 256, 0, s>>>(u, Xdata, K, J);
+  finish_sc_kernel<<<blocks, 256, 0, s>>>(z, u, Xdata, K, J, nsplit, split_stride_bytes / 4);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

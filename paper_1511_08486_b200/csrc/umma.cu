@@ -47,6 +47,8 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct GemmParams {
   int m_tiles, n_tiles, k_blocks;   // m_tiles counts tiles of 128*CG rows; k_blocks counts blocks of BK reduction steps
+  int k_splits, k_per_split;        // forward only: the reduction is cut in k_splits ranges of k_per_split blocks, each
+  long long split_stride;           // range writing its partial products to z + split * split_stride bytes
   int a_policy, b_policy;   // L2 eviction policy of the operand loads (0 normal, 1 evict first, 2 evict last)
   int m_fastest;            // tile order: 1 = consecutive tiles share the B operand slab, 0 = share the A slab
   int group;                // tiles of the fast dimension walked before the slow one advances (0 = all)
@@ -176,7 +178,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (CG == 2) ptx::cluster_sync();   // the peer's barriers exist before anything is signalled remotely
   ptx::tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  const int total_work = p.m_tiles * p.n_tiles * p.k_splits;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (every CTA)
@@ -188,7 +190,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #ifdef SFB_EXP_CLOCKS
     long long exp_wait_empty = 0;
 #endif
-    for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
+    for (int work = cluster_id; work < total_work && ok; work += num_clusters) {
+      const int tile = work / p.k_splits, split = work - tile * p.k_splits;
+      const int kb_begin = split * p.k_per_split, kb_end = min(kb_begin + p.k_per_split, p.k_blocks);
       int mt, nt;
       tile_coords(p, tile, mt, nt);
       mt = mt * CG + (int)rank;                           // 128-row unit of this CTA
@@ -199,7 +203,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         else { mp0 = mt * p.m_wp; }
       }
       int row0 = 0, kp0 = 0;           // apply: first row / worker of the current reduction block
-      for (int kb = 0; kb < p.k_blocks; ++kb) {
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
 #ifdef SFB_EXP_CLOCKS
         long long w0 = clock64();
 #endif
@@ -295,7 +299,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #ifdef SFB_EXP_CLOCKS
     long long exp_wait_full = 0, exp_wait_tmem = 0;
 #endif
-    for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++it) {
+    for (int work = cluster_id; work < total_work && ok; work += num_clusters, ++it) {
+      const int split = work % p.k_splits;
+      const int kb_begin = split * p.k_per_split, kb_end = min(kb_begin + p.k_per_split, p.k_blocks);
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
 #ifdef SFB_EXP_CLOCKS
@@ -308,7 +314,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * BN;
-      for (int kb = 0; kb < p.k_blocks; ++kb) {
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
 #ifdef SFB_EXP_CLOCKS
         long long w2 = clock64();
 #endif
@@ -332,7 +338,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               const uint64_t b_desc = ptx::smem_desc(b_addr + a * (BNC * 128), 16, 1024, 2);
 #pragma unroll
               for (int k = 0; k < CH / UMMA_K; ++k) {
-                const uint32_t acc = (kb > 0 || a > 0 || k > 0) ? 1u : 0u;
+                const uint32_t acc = (kb > kb_begin || a > 0 || k > 0) ? 1u : 0u;
                 if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
                 else ptx::mma_tf32<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
               }
@@ -346,14 +352,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             constexpr uint32_t STEP = (UMMA_K * 128) >> 4;
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k) {
-              const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+              const uint32_t acc = (kb > kb_begin || k > 0) ? 1u : 0u;
               if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
               else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
             }
           }
           ptx::mma_commit<CG>(&ctl->empty[s]);                     // stage reusable once these MMAs have read it
           if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->empty[s]), 1));
-          if (kb == p.k_blocks - 1) {                              // accumulator complete, in both CTAs
+          if (kb == kb_end - 1) {                                  // accumulator complete, in both CTAs
             ptx::mma_commit<CG>(&ctl->tmem_full[buf]);
             if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_full[buf]), 1));
           }
@@ -379,7 +385,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int lrow = lane >> 3, lq = lane & 7;    // transposed assignment: row-in-group, 16-byte column
     int it = 0;
     bool ok = true;
-    for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++it) {
+    for (int work = cluster_id; work < total_work && ok; work += num_clusters, ++it) {
+      const int tile = work / p.k_splits, split = work - tile * p.k_splits;
       int mt, nt;
       tile_coords(p, tile, mt, nt);
       mt = mt * CG + (int)rank;
@@ -398,7 +405,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           int wp_, slot;
           if (p.B >= BM) { wp_ = mt / p.m_tpw; slot = (mt % p.m_tpw) * BM + r; }
           else { wp_ = mt * p.m_wp + r / p.m_bb; slot = r % p.m_bb; }
-          if (wp_ < p.P && slot < p.B) rowp[g] = reinterpret_cast<float*>(p.z.row(wp_ * p.B + slot));
+          if (wp_ < p.P && slot < p.B)
+            rowp[g] = reinterpret_cast<float*>(p.z.row(wp_ * p.B + slot) + split * p.split_stride);
         }
       }
       const int ncols = APPLY ? p.Nvalid : p.z.ld;   // multiples of 4 on these paths
@@ -669,7 +677,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
     }
     attr_done = true;
   }
-  const int tiles = p.m_tiles * p.n_tiles;
+  const int tiles = p.m_tiles * p.n_tiles * p.k_splits;
   if (CG == 1) {
     const int grid = tiles < num_sms ? tiles : num_sms;
     kernel<<<grid, NUM_THREADS, smem, s>>>(a, b, w, p);
@@ -730,6 +738,8 @@ struct UmmaPlan {
   int fold_ka;    // 128-byte atoms of the reduction index per stage in the folded kernels (SFB_FOLD_KA, default 2)
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
   int fwd_group, apply_group;   // tile-order group widths (SFB_FWD_GROUP / SFB_APPLY_GROUP override the defaults)
+  float* part_ws;               // partial products of a split reduction, [4][K][ldp] fp32 (small forward GEMMs only)
+  int ldp;
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -751,11 +761,23 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   const char* ag = getenv("SFB_APPLY_GROUP");
   p->fwd_group = fg != nullptr ? atoi(fg) : 8;
   p->apply_group = ag != nullptr ? atoi(ag) : 8;
+  p->part_ws = nullptr;
+  p->ldp = (int)pad_to(d.J, 4);
+  {   // forward GEMMs with fewer 128 x 128 tiles than half the SMs may split their reduction
+    const long long K_ = (long long)d.P * d.B;
+    const long long tiles = ((K_ + 127) / 128) * ((d.J + 127) / 128);
+    if (tiles * 2 <= p->num_sms && cudaMalloc(&p->part_ws, (size_t)4 * K_ * p->ldp * 4) != cudaSuccess) {
+      cudaGetLastError();
+      delete p;
+      return SFB_ERR_ALLOC;
+    }
+  }
   p->stats = nullptr;
   if (d.model == SFB_MLR) {
     const size_t parts = 2 * (size_t)((d.J + 127) / 128);
     if (cudaMalloc(&p->stats, (size_t)d.P * d.B * parts * sizeof(float2)) != cudaSuccess) {
       cudaGetLastError();
+      if (p->part_ws) cudaFree(p->part_ws);
       delete p;
       return SFB_ERR_ALLOC;
     }
@@ -766,6 +788,7 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
 
 void umma_plan_destroy(UmmaPlan* p) {
   if (p->stats) cudaFree(p->stats);
+  if (p->part_ws) cudaFree(p->part_ws);
   delete p;
 }
 
@@ -782,7 +805,8 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
 
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
 int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
-                      float2* stats, int* n_parts_out, int* part_cols_out) {
+                      float2* stats, int* n_parts_out, int* part_cols_out, int* k_splits_out, int max_splits,
+                      long long split_stride) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   GemmParams p;
@@ -796,6 +820,20 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
   p.n_tiles = (d.J + v.bn - 1) / v.bn;
   p.k_blocks = (d.D + CH * v.ka - 1) / (CH * v.ka);
+  // Few tiles and a long reduction (e.g. 1024 samples x 1000 classes over 20000 features): cut the
+  // reduction so that every SM gets work; the partial products are summed, in a fixed order, by the
+  // finishing pass.  Only when the caller provides the partial buffers (k_splits_out != nullptr).
+  p.k_splits = 1;
+  if (k_splits_out != nullptr && stats == nullptr) {
+    const int tiles = p.m_tiles * p.n_tiles;
+    int ks = pl->num_sms / (tiles > 0 ? tiles : 1);
+    if (ks > 4) ks = 4;
+    if (ks > max_splits) ks = max_splits;
+    if (ks >= 2 && p.k_blocks >= 32 * ks) p.k_splits = ks;
+    *k_splits_out = p.k_splits;
+  }
+  p.k_per_split = (p.k_blocks + p.k_splits - 1) / p.k_splits;
+  p.split_stride = split_stride;
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
   p.m_fastest = ((long long)d.J * d.D > (long long)d.P * d.B * d.D) ? 1 : 0;
   p.a_policy = p.m_fastest ? 2 : 0;   // the operand whose slab changes every tile is re-read all along: keep it
@@ -833,6 +871,25 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     RowMap zz = bf16 ? z : u;   // fp32 products: workspace when u is bf16, else u itself (finished in place)
     // the GEMM epilogue leaves exp(z - local max) in u and (max, sum) per half tile; the finishing
     // pass rescales to the softmax and subtracts the one-hot label, in place
+    if (pl->part_ws != nullptr) {
+      // few tiles: split reduction into the partial buffers, then the plain softmax pass sums them
+      RowMap pz;
+      pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
+      pz.worker_stride = (long long)d.B * pl->ldp * 4;
+      const long long sstride = (long long)K * pl->ldp * 4;
+      int ks = 1;
+      if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr, nullptr,
+                                 &ks, 4, sstride)) < 0)
+        return r;
+      launches += r;
+      if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
+      launches += r;
+      if (v.base != nullptr) {
+        if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
+        launches += r;
+      }
+      return launches;
+    }
     int n_parts = 0, part_cols = 0;
     (void)zz;
     if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
@@ -852,6 +909,17 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   if ((r = launch_diff_rows(s, reinterpret_cast<const float*>(X), reinterpret_cast<const float*>(aux->Xb), v, K, d.D)) < 0)
     return r;
   launches += r;
+  if (pl->part_ws != nullptr) {
+    RowMap pz;
+    pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
+    pz.worker_stride = (long long)d.B * pl->ldp * 4;
+    const long long sstride = (long long)K * pl->ldp * 4;
+    int ks = 1;
+    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, 4, sstride)) < 0) return r;
+    launches += r;
+    if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
+    return launches + r;
+  }
   if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr)) < 0) return r;
   launches += r;
   if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
@@ -874,6 +942,7 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   else { p.k_bb = pow2_at_least(d.B); p.k_wp = BK / p.k_bb; p.k_bpw = 1; p.k_blocks = (workers + p.k_wp - 1) / p.k_wp; }
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
   p.n_tiles = (d.D + v.bn - 1) / v.bn;
+  p.k_splits = 1; p.k_per_split = p.k_blocks;
   p.Mvalid = d.J; p.Nvalid = d.D;
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
   p.a_policy = p.m_fastest ? 2 : 0;
