@@ -19,6 +19,7 @@ struct sfb_ctx {
   int ldz;
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
+  void* csc_ws;             // SC, fp32 path: scratch of the atom-major re-sort of the codes (when K fits)
   // sfb_step_host: two sets of device staging buffers for the step's host inputs (allocated on first
   // use), filled on a side stream so that the copy of step t+1 overlaps the kernels of step t
   char* host_stage[2][6];
@@ -209,6 +210,8 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
   if (ok) ok = cudaMemsetAsync(c->dev_status, 0, 256, c->stream) == cudaSuccess;
   if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_F32)
     ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
+  if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_F32 && sc_csc_supported(c->K))
+    ok = cudaMalloc(&c->csc_ws, (size_t)sc_csc_workspace_bytes(c->K, desc->D, (long long)desc->nnz_capacity)) == cudaSuccess;
   if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_TF32)
     ok = cudaMalloc(&c->a_dense, (size_t)c->K * c->l.ldv * 4) == cudaSuccess;
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
@@ -239,6 +242,7 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->z_ws) cudaFree(c->z_ws);
   if (c->wt_ws) cudaFree(c->wt_ws);
   if (c->a_dense) cudaFree(c->a_dense);
+  if (c->csc_ws) cudaFree(c->csc_ws);
   for (int k = 0; k < 2; ++k)
     for (int i = 0; i < 6; ++i)
       if (c->host_stage[k][i]) cudaFree(c->host_stage[k][i]);
@@ -345,7 +349,10 @@ int sfb_pack(sfb_ctx* c, const void* U, const void* V, const sfb_aux* aux, void*
 static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check) {
   const sfb_desc& d = c->d;
   if (check) ACC(launch_check_header(c->stream, sf_buf, d, c->l, c->dev_status));
-  if (d.v_sparse && d.path == SFB_PATH_F32) {
+  if (d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
+    ACC(launch_sc_apply_csc(c->stream, reinterpret_cast<float*>(W), stream_codes(c, sf_buf), stream_u(c, sf_buf), K, d.J,
+                            d.D, eta, (long long)d.nnz_capacity, c->csc_ws, c->dev_status));
+  } else if (d.v_sparse && d.path == SFB_PATH_F32) {
     ACC(launch_sc_apply(c->stream, reinterpret_cast<float*>(W), stream_codes(c, sf_buf), stream_u(c, sf_buf), K, d.J,
                         d.D, eta, c->dev_status, c->dev_status));
   } else if (d.v_sparse) {

@@ -109,6 +109,13 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
 int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                     const int* dev_status_ro, int* dev_status);
 
+// The same update through an atom-major (CSC) re-sort of the codes and shared-memory u columns (faster;
+// needs sc_csc_supported(K) and a workspace of sc_csc_workspace_bytes(K, D, nnz_capacity) bytes).
+long long sc_csc_workspace_bytes(int K, int D, long long nnz_capacity);
+bool sc_csc_supported(int K);
+int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
+                        long long nnz_capacity, void* workspace, const int* dev_status_ro);
+
 // Dense fp32 rows a_i of the CSR codes (zeros elsewhere), for the tensor-core sparse-coding path.
 int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status);
 

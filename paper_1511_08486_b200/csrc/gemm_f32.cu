@@ -53,7 +53,7 @@ __device__ __forceinline__ void mma_tile(const float (*As)[64 * MI + 4], const f
 // Tile rows = samples i (BM = 64*MI), tile columns = classes j (BN = 64*NI), reduction over d.
 // Both operands are contiguous along d, so tiles are transposed while being stored to shared memory.
 template <int MI, int NI>
-__global__ void __launch_bounds__(256) forward_f32_kernel(const float* __restrict__ W, const float* __restrict__ X,
+__global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __restrict__ W, const float* __restrict__ X,
                                                           const float* __restrict__ Xb, int K, int J, int D,
                                                           RowMap z, RowMap v) {
   constexpr int BM = 64 * MI, BN = 64 * NI;
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(256) forward_f32_kernel(const float* __restric
 // Tile rows = rows j of W (BM), tile columns = columns d of W (BN), reduction over the K factors.
 // U rows are contiguous along j and V rows along d: tiles go to shared memory as they are.
 template <int MI, int NI>
-__global__ void __launch_bounds__(256) apply_f32_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
+__global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
                                                         int D, float eta, const int* __restrict__ dev_status) {
   constexpr int BM = 64 * MI, BN = 64 * NI;
   __shared__ __align__(16) float As[BK][BM + 4];
