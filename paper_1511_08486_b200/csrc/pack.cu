@@ -81,6 +81,7 @@ __global__ void __launch_bounds__(256) pack_csr_kernel(char* buf, long long stre
                                                        const uint32_t* __restrict__ idx, const float* __restrict__ val,
                                                        int* dev_status) {
   const int p = blockIdx.x;
+  const int part = blockIdx.y, parts = gridDim.y;   // the worker's words are spread over gridDim.y blocks
   char* vb = buf + streams_off + (long long)p * stream_stride + u_bytes;
   uint32_t* rp = reinterpret_cast<uint32_t*>(vb);
   uint32_t* ix = reinterpret_cast<uint32_t*>(vb + rp_bytes);
@@ -88,9 +89,9 @@ __global__ void __launch_bounds__(256) pack_csr_kernel(char* buf, long long stre
   const uint32_t base = rowptr[(size_t)p * B];
   const uint32_t nnz_true = rowptr[(size_t)(p + 1) * B] - base;
   const uint32_t nnz = nnz_true < (uint32_t)cap_p ? nnz_true : (uint32_t)cap_p;
-  if (nnz_true > (uint32_t)cap_p && threadIdx.x == 0) atomicOr(dev_status, SFB_DEV_CAPACITY);
+  if (nnz_true > (uint32_t)cap_p && threadIdx.x == 0 && part == 0) atomicOr(dev_status, SFB_DEV_CAPACITY);
   const int rp_words = (int)(rp_bytes / 4);
-  for (int t = threadIdx.x; t < rp_words; t += blockDim.x) {
+  for (int t = part * blockDim.x + threadIdx.x; t < rp_words; t += parts * blockDim.x) {
     uint32_t r = 0u;
     if (t <= B) {
       r = rowptr[(size_t)p * B + t] - base;
@@ -100,7 +101,7 @@ __global__ void __launch_bounds__(256) pack_csr_kernel(char* buf, long long stre
   }
   const int idx_words = (int)(idx_bytes / 4);
   bool bad = false;
-  for (int t = threadIdx.x; t < idx_words; t += blockDim.x) {
+  for (int t = part * blockDim.x + threadIdx.x; t < idx_words; t += parts * blockDim.x) {
     uint32_t c = 0u;
     float a = 0.f;
     if ((uint32_t)t < nnz) {
@@ -129,7 +130,8 @@ int launch_check_header(cudaStream_t s, const void* sf_buf, const sfb_desc& d, c
 
 int launch_pack_csr(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, const uint32_t* rowptr,
                     const uint32_t* idx, const float* val, int* dev_status) {
-  pack_csr_kernel<<<d.P, 256, 0, s>>>(reinterpret_cast<char*>(sf_buf), l.streams_off, l.stream_stride, l.u_bytes,
+  const int parts = (l.cap_p + 2047) / 2048 < 1 ? 1 : ((l.cap_p + 2047) / 2048 > 64 ? 64 : (l.cap_p + 2047) / 2048);
+  pack_csr_kernel<<<dim3(d.P, parts), 256, 0, s>>>(reinterpret_cast<char*>(sf_buf), l.streams_off, l.stream_stride, l.u_bytes,
                                       l.rp_bytes, l.idx_bytes, d.B, l.cap_p, d.D, rowptr, idx, val, dev_status);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }

@@ -59,10 +59,15 @@ __global__ void __launch_bounds__(256) csc_chunk_offsets_kernel(int nchunks, int
   const int d = blockIdx.x * 256 + threadIdx.x;
   if (d >= D) return;
   int run = 0;
-  for (int c = 0; c < nchunks; ++c) {
-    const int t = cnt[(size_t)c * D + d];
-    cnt[(size_t)c * D + d] = run;
-    run += t;
+  for (int c0 = 0; c0 < nchunks; c0 += 8) {   // eight independent loads in flight, then the running sum
+    int t[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t[q] = (c0 + q < nchunks) ? cnt[(size_t)(c0 + q) * D + d] : 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (c0 + q < nchunks) cnt[(size_t)(c0 + q) * D + d] = run;
+      run += t[q];
+    }
   }
   total[d] = run;
 }
