@@ -273,3 +273,8 @@ def test_sc_prox_unit_columns():
         assert orc.rel_fro(wl.W.cpu().numpy(), ref) <= 1e-6
     finally:
         wl.close()
+
+
+def test_c1_hundred_steps_f32():
+    # C1's own schedule on the fp32 path: 100 steps, pool of 8 minibatches, eta = 1e-2
+    check_config(get_config("C1"), "f32", eta=1e-2, steps=100)

@@ -72,3 +72,14 @@ def test_tf32_sparse_coding_dense_alternative():
     check_config(_cfg("C3", "tf32", J=70, D=332, P=3, B=5, density=0.1), "tf32", eta=1e-2, steps=2)
     check_config(_cfg("C3", "tf32", J=512, D=2000, P=4, B=32), "tf32", eta=1e-3, steps=2)
     check_config(_cfg("C3", "tf32"), "tf32", eta=1e-4, steps=1)
+
+
+def test_tf32_c1_hundred_steps():
+    # the workload's own schedule: 100 steps over a pool of 8 minibatches, eta = 1e-2, free-running
+    # against the oracle's trajectory (the oracle keeps W in fp64; the tolerance is on W_100 - W_0)
+    check_config(_cfg("C1", "tf32"), "tf32", eta=1e-2, steps=100)
+
+
+def test_bf16_c4_reduced_fifty_steps():
+    # C4's 50-step schedule at a reduced shape the oracle finishes in seconds (J = 4096, K = 512)
+    check_config(_cfg("C4", "bf16", J=4096, D=8192, P=16, B=32), "bf16", eta=1e-3, steps=50)
