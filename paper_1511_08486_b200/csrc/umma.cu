@@ -711,9 +711,11 @@ int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CU
   if (v.cg == 2) {
     if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, w, p, num_sms);
     if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, w, p, num_sms);
+    if (v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, false, EPI>(s, a, b, w, p, num_sms);
     return launch_gemm<ES, APPLY, 256, 2, 1, false, EPI>(s, a, b, w, p, num_sms);
   }
   if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false, EPI>(s, a, b, w, p, num_sms);
+  if (v.ka == 2) return launch_gemm<ES, APPLY, 128, 1, 2, false, EPI>(s, a, b, w, p, num_sms);
   return launch_gemm<ES, APPLY, 128, 1, 1, false, EPI>(s, a, b, w, p, num_sms);
 }
 
@@ -799,7 +801,9 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
   // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
   v.cg = (v.bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
   v.fold = v.cg == 2 && pl->fold_ok && dims_chunk_aligned;
-  v.ka = v.fold ? pl->fold_ka : 1;
+  // two 128-byte atoms of reduction per stage wherever three such stages fit in shared memory: the
+  // per-stage barrier round trip, not the number of TMA instructions, is what costs
+  v.ka = (v.cg == 2 || v.bn == 128) ? pl->fold_ka : 1;
   return v;
 }
 
