@@ -6,11 +6,12 @@
 // atom with a counting sort that is deterministic: counts per (chunk of 8 samples, atom) by integer
 // atomics, prefix sums over chunks and atoms, then every chunk places its samples one after the other,
 // so inside a column the entries are in sample order whatever the thread schedule.
-// The apply gives each thread block 32 rows of W and keeps the matching 32 columns of ALL u_i in shared
-// memory (K x 128 bytes).  A warp takes 32 consecutive atoms: for each atom it walks the column's
-// entries (coalesced loads, broadcast by shuffles), accumulating a_id * u_i[j0 + lane] from shared
-// memory, parks the 32 sums in a private 32 x 33 tile, and finally updates W with 128-byte row segments.
-// W and U are each read once; no floating-point atomics; every element of W has one owner and a fixed
+// The apply gives each thread block 64 rows of W and keeps the matching 64 columns of a slice of the
+// u_i in shared memory (the samples are taken in as few slices as fit).  A warp takes 16 consecutive
+// atoms: for each atom it walks the slice's entries of the column (coalesced loads staged through a
+// small per-warp strip), accumulating a_id * u_i[j0 + 2 lane .. + 1] from shared memory, parks the sums
+// in a private 16 x 65 tile, and finally updates W with 64-byte row segments.
+// U is read once and W once per slice; no floating-point atomics; every element of W has one owner and a fixed
 // summation order (bit-reproducible); atoms nobody uses get W + (-eta * 0) = W, bit-identical.
 #include "common.cuh"
 
@@ -18,7 +19,6 @@ namespace sfb {
 namespace {
 
 constexpr int CSC_CHUNK = 8;    // samples per chunk of the counting sort
-constexpr int CSC_JT = 32;      // rows of W per block of the apply
 
 struct CsrRow2 {
   const uint32_t* idx;
@@ -132,76 +132,111 @@ __global__ void __launch_bounds__(256) csc_fill_kernel(CsrView codes, int K, int
   }
 }
 
-// grid = ceil(J / 32); dynamic shared memory: K * 32 floats (u columns) + warps * 32 * 33 floats (tiles)
+constexpr int CSC2_JT = 64;     // rows of W per block of the two-rows-per-lane apply
+constexpr int CSC2_AB = 16;     // atoms per warp block there
+constexpr int CSC2_WARP_FLOATS = 64 + CSC2_AB * 65;   // entry strip (32 x 8 bytes) + [16][65] tile
+
+// Two rows of W per lane, the samples taken in `passes` slices so that a slice of the u columns
+// (Kh x 256 bytes) fits in shared memory.  Shared-memory bandwidth bounds this kernel: per entry and 64 rows
+// it costs half a broadcast read of the strip (two entries per 16-byte load) and one 256-byte read of u.
+// grid = (ceil(J / 64), atom splits).  cnt holds, after the fill, for every (chunk, atom) the number of
+// entries of the column that belong to samples before the END of the chunk, which gives the slice bounds.
 __global__ void __launch_bounds__(512) csc_apply_kernel(float* __restrict__ W, RowMap u, int K, int J, int D, float eta,
-                                                        const int* __restrict__ colptr, const int* __restrict__ ent_i,
-                                                        const float* __restrict__ ent_a,
-                                                        const int* __restrict__ status_ro) {
+                                                         const int* __restrict__ colptr, const int* __restrict__ cnt,
+                                                         const int* __restrict__ ent_i, const float* __restrict__ ent_a,
+                                                         int passes, int Kh, const int* __restrict__ status_ro) {
   extern __shared__ __align__(16) float smem[];
   if (status_ro != nullptr && (*status_ro & SFB_DEV_BAD_HEADER)) return;
-  float* Us = smem;                                   // [K][32]
+  float* Us = smem;                                   // [Kh][64]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  float* T = smem + (size_t)K * 32 + warp * (32 * 33 + 64);   // [32][33] + entry strip, private to the warp
-  const int j0 = blockIdx.x * CSC_JT;
-  const bool jok = j0 + lane < J;
-  for (int i = warp; i < K; i += nwarps)
-    Us[i * 32 + lane] = jok ? reinterpret_cast<const float*>(u.row(i))[j0 + lane] : 0.f;
-  __syncthreads();
-
-  const int nblocks = (D + 31) / 32;
-  for (int ab = warp; ab < nblocks; ab += nwarps) {
-    const int d0 = ab * 32;
-    const int dn = min(32, D - d0);
-    // column boundaries of the 32 atoms: lane holds colptr[d0 + lane] and the end of the last one
-    const int cp = colptr[min(d0 + lane, D)];
-    const int cp_next = colptr[min(d0 + 32, D)];
-    // per atom: rounds of 32 entries staged in a per-warp shared-memory strip (one coalesced load per
-    // round, the next round's load already in flight), then one broadcast read + one u read + one FMA
-    // per entry, four running sums
-    int2* strip = reinterpret_cast<int2*>(T + 32 * 33);           // 32 (sample, value) pairs
-    int pre_i = 0;
-    float pre_a = 0.f;
-    {
-      const int b0 = __shfl_sync(0xffffffffu, cp, 0);
-      if (b0 + lane < cp_next) { pre_i = ent_i[b0 + lane]; pre_a = ent_a[b0 + lane]; }
+  float* region = smem + (size_t)Kh * 64 + warp * CSC2_WARP_FLOATS;
+  int2* strip = reinterpret_cast<int2*>(region);
+  const int4* strip4 = reinterpret_cast<const int4*>(region);
+  float* T = region + 64;
+  const int j0 = blockIdx.x * CSC2_JT;
+  const int jn = min(CSC2_JT, J - j0);
+  const int nnz = colptr[D];
+  const int nchunks = (K + CSC_CHUNK - 1) / CSC_CHUNK;
+  const int nblocks = (D + CSC2_AB - 1) / CSC2_AB;
+  for (int h = 0; h < passes; ++h) {
+    const int i_lo = h * Kh;
+    if (i_lo >= K) break;
+    const int i_n = min(Kh, K - i_lo);
+    __syncthreads();                                  // the previous slice is no longer read
+    for (int i = warp; i < i_n; i += nwarps) {
+      const float* ur = reinterpret_cast<const float*>(u.row(i_lo + i)) + j0;
+      float2 v = make_float2(0.f, 0.f);
+      if (2 * lane + 1 < jn) v = *reinterpret_cast<const float2*>(ur + 2 * lane);
+      else if (2 * lane < jn) v.x = ur[2 * lane];
+      *reinterpret_cast<float2*>(Us + i * 64 + 2 * lane) = v;
     }
-    for (int dd = 0; dd < dn; ++dd) {
-      const int beg = __shfl_sync(0xffffffffu, cp, dd);
-      const int stop = (dd < 31) ? __shfl_sync(0xffffffffu, cp, dd + 1) : cp_next;
-      float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-      for (int base = beg; base < stop; base += 32) {
-        // the prefetched values are those of [base, base + 32) of the contiguous entry range
-        strip[lane] = make_int2(base + lane < stop ? pre_i : 0, __float_as_int(base + lane < stop ? pre_a : 0.f));
-        const int nxt = (base + 32 < stop) ? base + 32 : stop;    // next round: same atom, or the next atom's start
-        if (nxt + lane < cp_next) { pre_i = ent_i[nxt + lane]; pre_a = ent_a[nxt + lane]; }
-        __syncwarp();
+    __syncthreads();
+    const int c_lo = i_lo / CSC_CHUNK;                               // Kh is a multiple of the chunk size
+    const int c_hi = min(nchunks, (i_lo + Kh) / CSC_CHUNK);
+    for (int ab = blockIdx.y + gridDim.y * warp; ab < nblocks; ab += gridDim.y * nwarps) {
+      const int d0 = ab * CSC2_AB;
+      const int dn = min(CSC2_AB, D - d0);
+      int lo = nnz, hi = nnz;                                        // entry range of atom d0 + lane in this slice
+      if (lane < dn) {
+        const int d = d0 + lane, cp = colptr[d];
+        lo = (c_lo == 0) ? cp : cp + cnt[(size_t)(c_lo - 1) * D + d];
+        hi = cp + cnt[(size_t)(c_hi - 1) * D + d];
+      }
+      int pre_i = 0;
+      float pre_a = 0.f;
+      {
+        const int b0 = __shfl_sync(0xffffffffu, lo, 0);
+        if (b0 + lane < nnz) { pre_i = ent_i[b0 + lane]; pre_a = ent_a[b0 + lane]; }
+      }
+      for (int dd = 0; dd < dn; ++dd) {
+        const int beg = __shfl_sync(0xffffffffu, lo, dd);
+        const int stop = __shfl_sync(0xffffffffu, hi, dd);
+        const int next_beg = __shfl_sync(0xffffffffu, lo, dd + 1);   // lane 16 and up hold nnz: nothing to fetch
+        float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
+        if (beg >= stop && next_beg + lane < nnz) { pre_i = ent_i[next_beg + lane]; pre_a = ent_a[next_beg + lane]; }
+        for (int base = beg; base < stop; base += 32) {
+          const bool ok = base + lane < stop;
+          strip[lane] = make_int2(ok ? pre_i - i_lo : 0, __float_as_int(ok ? pre_a : 0.f));
+          const int nxt = (base + 32 < stop) ? base + 32 : next_beg;
+          if (nxt + lane < nnz) { pre_i = ent_i[nxt + lane]; pre_a = ent_a[nxt + lane]; }
+          __syncwarp();
 #pragma unroll
-        for (int k = 0; k < 32; k += 4) {
-          const int2 e0 = strip[k], e1 = strip[k + 1], e2 = strip[k + 2], e3 = strip[k + 3];
-          acc0 = fmaf(__int_as_float(e0.y), Us[e0.x * 32 + lane], acc0);
-          acc1 = fmaf(__int_as_float(e1.y), Us[e1.x * 32 + lane], acc1);
-          acc2 = fmaf(__int_as_float(e2.y), Us[e2.x * 32 + lane], acc2);
-          acc3 = fmaf(__int_as_float(e3.y), Us[e3.x * 32 + lane], acc3);
+          for (int k = 0; k < 16; k += 2) {
+            const int4 p = strip4[k], q = strip4[k + 1];
+            const float2 u0 = *reinterpret_cast<const float2*>(Us + p.x * 64 + 2 * lane);
+            const float2 u1 = *reinterpret_cast<const float2*>(Us + p.z * 64 + 2 * lane);
+            const float2 u2 = *reinterpret_cast<const float2*>(Us + q.x * 64 + 2 * lane);
+            const float2 u3 = *reinterpret_cast<const float2*>(Us + q.z * 64 + 2 * lane);
+            acc0.x = fmaf(__int_as_float(p.y), u0.x, acc0.x); acc0.y = fmaf(__int_as_float(p.y), u0.y, acc0.y);
+            acc1.x = fmaf(__int_as_float(p.w), u1.x, acc1.x); acc1.y = fmaf(__int_as_float(p.w), u1.y, acc1.y);
+            acc2.x = fmaf(__int_as_float(q.y), u2.x, acc2.x); acc2.y = fmaf(__int_as_float(q.y), u2.y, acc2.y);
+            acc3.x = fmaf(__int_as_float(q.w), u3.x, acc3.x); acc3.y = fmaf(__int_as_float(q.w), u3.y, acc3.y);
+          }
+          __syncwarp();
         }
-        __syncwarp();
+        T[dd * 65 + 2 * lane] = (acc0.x + acc1.x) + (acc2.x + acc3.x);
+        T[dd * 65 + 2 * lane + 1] = (acc0.y + acc1.y) + (acc2.y + acc3.y);
       }
-      T[dd * 33 + lane] = (acc0 + acc1) + (acc2 + acc3);
-    }
-    __syncwarp();
-    // W[j0 + jj][d0 + lane] -= eta * T[lane][jj]: 128-byte row segments, 8 rows fetched at a time
-    if (lane < dn) {
-      const int jn = min(32, J - j0);
-      for (int jb = 0; jb < jn; jb += 8) {
-        float wv[8];
+      __syncwarp();
+      // W[j0 + jj][d0 + a] -= eta * T[a][jj]: a warp instruction covers two rows x 16 atoms (64-byte segments)
+      const int a = lane & 15, q = lane >> 4;
+      if (a < dn) {
+        for (int jb = 0; jb < jn; jb += 16) {
+          float wv[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          wv[q] = (jb + q < jn) ? W[(size_t)(j0 + jb + q) * D + d0 + lane] : 0.f;
+          for (int t = 0; t < 8; ++t) {
+            const int jj = jb + 2 * t + q;
+            wv[t] = (jj < jn) ? W[(size_t)(j0 + jj) * D + d0 + a] : 0.f;
+          }
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          if (jb + q < jn) W[(size_t)(j0 + jb + q) * D + d0 + lane] = fmaf(-eta, T[lane * 33 + jb + q], wv[q]);
+          for (int t = 0; t < 8; ++t) {
+            const int jj = jb + 2 * t + q;
+            if (jj < jn) W[(size_t)(j0 + jj) * D + d0 + a] = fmaf(-eta, T[a * 65 + jj], wv[t]);
+          }
+        }
       }
+      __syncwarp();
     }
-    __syncwarp();
   }
 }
 
@@ -213,8 +248,8 @@ long long sc_csc_workspace_bytes(int K, int D, long long nnz_capacity) {
   return pad_to((nchunks * D + D + D + 1) * 4, 256) + pad_to(nnz_capacity * 4, 256) * 2;
 }
 
-// The u columns of all K samples must fit in shared memory next to the warps' tiles.
-bool sc_csc_supported(int K) { return (long long)K * 128 + 16 * (32 * 33 + 64) * 4 <= 220 * 1024; }
+// The sliced kernel takes any K (more slices); the bound only keeps the chunk tables small.
+bool sc_csc_supported(int K) { return K <= (1 << 14); }
 
 int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                         long long nnz_capacity, void* workspace, const int* dev_status_ro) {
@@ -231,14 +266,24 @@ int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K
   csc_scan_kernel<<<1, 1024, 0, s>>>(D, total, colptr);
   csc_fill_kernel<<<nchunks, 256, 0, s>>>(codes, K, D, cnt, colptr, ent_i, ent_a);
   const int threads = 512;
-  const size_t smem = (size_t)K * 128 + (size_t)(threads / 32) * (32 * 33 + 64) * 4;
   static bool attr_done = false;
   if (!attr_done) {
     cudaFuncSetAttribute(csc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     attr_done = true;
   }
-  csc_apply_kernel<<<(J + CSC_JT - 1) / CSC_JT, threads, smem, s>>>(W, u, K, J, D, eta, colptr, ent_i, ent_a,
-                                                                  dev_status_ro);
+  // slices of the samples: the fewest that let Kh x 256 bytes of u sit beside the warps' tiles
+  const long long tiles = (long long)(threads / 32) * CSC2_WARP_FLOATS * 4;
+  const int kh_max = (int)((220 * 1024 - tiles) / 256) / CSC_CHUNK * CSC_CHUNK;
+  const int passes = (K + kh_max - 1) / kh_max;
+  const int Kh = ((K + passes - 1) / passes + CSC_CHUNK - 1) / CSC_CHUNK * CSC_CHUNK;
+  const int nj = (J + CSC2_JT - 1) / CSC2_JT;
+  const int nblocks = (D + CSC2_AB - 1) / CSC2_AB;
+  int splits = 148 / nj;                            // atom splits: fill the SMs when J / 64 alone does not
+  if (splits > nblocks / (threads / 32)) splits = nblocks / (threads / 32);
+  if (splits < 1) splits = 1;
+  const size_t smem = (size_t)Kh * 256 + (size_t)tiles;
+  csc_apply_kernel<<<dim3(nj, splits), threads, smem, s>>>(W, u, K, J, D, eta, colptr, cnt, ent_i, ent_a, passes, Kh,
+                                                           dev_status_ro);
   return cudaGetLastError() == cudaSuccess ? 5 : SFB_ERR_CUDA;
 }
 

@@ -178,6 +178,12 @@ def test_c3_sc_scaled_f32():
     check_config(scaled("C3", J=512, D=2000, P=4, B=32), "f32", eta=1e-3, steps=2)
 
 
+def test_c3_sc_many_samples_f32():
+    """K beyond one shared-memory slice of the scatter apply: two ragged slices, then three."""
+    check_config(scaled("C3", J=100, D=310, P=2, B=515, density=0.03), "f32", eta=1e-3, steps=1)
+    check_config(scaled("C3", J=72, D=200, P=4, B=400, density=0.03), "f32", eta=1e-3, steps=1)
+
+
 def test_c3_sc_full_f32():
     check_config(get_config("C3"), "f32", eta=1e-4, steps=1)
 
