@@ -160,6 +160,18 @@ int sfb_step_host(sfb_ctx* ctx, void* W, const void* X_host, const sfb_aux* aux_
  * SFB_OK without launching).  W [J][D] fp32 in place. */
 int sfb_prox(sfb_ctx* ctx, void* W);
 
+/* Minibatch objective at W, the function whose gradient the sufficient factors of this minibatch carry
+ * (Section 3, problem (P): the sum over the minibatch of f_i(W a_i); the update of Section 3 is a gradient
+ * step on it).  SFB_MLR: sum_i logsumexp(W x_i) - (W x_i)[y_i].  SFB_DML: sum_i 1/2 |L d_i|^2 for a similar
+ * pair, 1/2 max(0, margin - |L d_i|^2) for a dissimilar one.  SFB_SC: sum_i 1/2 |W a_i - x_i|^2.
+ * Arguments as sfb_compute_factors; loss: DEVICE pointer to one double (8-byte aligned), written on the
+ * context's stream.  The products are formed in the context's math path (SFB_DML always on the fp32
+ * path), reduced per sample in fp32 and over the samples in fp64, in a fixed order (bit-reproducible).
+ * A monitoring helper outside the step: W, the SF buffer and the step's state are untouched.  The first
+ * call allocates K x J floats of workspace (SFB_ERR_ALLOC if that fails); later calls allocate nothing.
+ * A label outside [0, J) contributes 0 and sets SFB_DEV_BAD_LABEL. */
+int sfb_loss(sfb_ctx* ctx, const void* W, const void* X, const sfb_aux* aux, double* loss);
+
 /* Tells the context that W was changed by someone else, so a cached bf16 shadow is stale. */
 int sfb_invalidate(sfb_ctx* ctx);
 

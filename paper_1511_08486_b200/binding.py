@@ -24,6 +24,7 @@ EXPORTS = (
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
     "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
     "sfb_halton_peers", "sfb_ssp_may_proceed", "sfb_prox", "sfb_step_host",
+    "sfb_loss",
 )
 
 
@@ -77,6 +78,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_step_host.restype = C.c_int
     lib.sfb_prox.argtypes = [vp, vp]
     lib.sfb_prox.restype = C.c_int
+    lib.sfb_loss.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp]
+    lib.sfb_loss.restype = C.c_int
     lib.sfb_invalidate.argtypes = [vp]
     lib.sfb_invalidate.restype = C.c_int
     lib.sfb_status.argtypes = [vp, C.POINTER(C.c_int32)]
@@ -216,6 +219,10 @@ class Context:
 
     def prox(self, W):
         self._chk(self._lib.sfb_prox(self._h, _ptr(W)), "sfb_prox")
+
+    def loss(self, W, X, aux: sfb_aux, out):
+        """Minibatch objective at W into `out` (one float64 on the device); asynchronous."""
+        self._chk(self._lib.sfb_loss(self._h, _ptr(W), _ptr(X), C.byref(aux), _ptr(out)), "sfb_loss")
 
     def invalidate(self):
         self._chk(self._lib.sfb_invalidate(self._h), "sfb_invalidate")

@@ -20,6 +20,8 @@ struct sfb_ctx {
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
   void* csc_ws;             // SC, fp32 path: scratch of the atom-major re-sort of the codes (when K fits)
+  float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
+  float* loss_i;            // sfb_loss: per-sample objective [K]
   // sfb_step_host: two sets of device staging buffers for the step's host inputs (allocated on first
   // use), filled on a side stream so that the copy of step t+1 overlaps the kernels of step t
   char* host_stage[2][6];
@@ -243,6 +245,8 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->wt_ws) cudaFree(c->wt_ws);
   if (c->a_dense) cudaFree(c->a_dense);
   if (c->csc_ws) cudaFree(c->csc_ws);
+  if (c->loss_rows) cudaFree(c->loss_rows);
+  if (c->loss_i) cudaFree(c->loss_i);
   for (int k = 0; k < 2; ++k)
     for (int i = 0; i < 6; ++i)
       if (c->host_stage[k][i]) cudaFree(c->host_stage[k][i]);
@@ -263,6 +267,46 @@ int sfb_prox(sfb_ctx* c, void* W) {
   if (c == nullptr || W == nullptr || !aligned(W, 16)) return SFB_ERR_ARG;
   if (c->d.model != SFB_SC) return SFB_OK;   // h = 0 for the MLR and DML workloads: identity
   ACC(launch_prox_unit_columns(c->stream, reinterpret_cast<float*>(W), c->d.J, c->d.D));
+  return SFB_OK;
+}
+
+int sfb_loss(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, double* loss) {
+  if (c == nullptr || W == nullptr || loss == nullptr) return SFB_ERR_ARG;
+  if (!aligned(W, 16) || !aligned(loss, 8)) return SFB_ERR_ARG;
+  int r = check_aux(c, aux);
+  if (r != SFB_OK) return r;
+  const sfb_desc& d = c->d;
+  if (d.model != SFB_SC && (X == nullptr || !aligned(X, 16))) return SFB_ERR_ARG;
+  const int ldl = (d.J + 3) & ~3;
+  if (c->loss_rows == nullptr) {
+    bool ok = cudaMalloc(&c->loss_rows, (size_t)c->K * ldl * 4) == cudaSuccess;
+    if (ok) ok = cudaMalloc(&c->loss_i, (size_t)c->K * 4) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      if (c->loss_rows) cudaFree(c->loss_rows);
+      c->loss_rows = nullptr;
+      return SFB_ERR_ALLOC;
+    }
+  }
+  const RowMap rows = caller_rows(c->loss_rows, ldl, d.B, 4);
+  const RowMap none = caller_rows(nullptr, c->l.ldv, d.B, c->l.es);
+  if (d.model == SFB_SC) {
+    // u_i = W a_i - x_i by the path's own forward (sparse gather, or dense tf32 rows)
+    r = factors_into(c, W, X, aux, rows, none, global_codes(aux, d.B));
+    if (r < 0) return r;
+  } else if (d.path == SFB_PATH_F32 || d.model == SFB_DML) {
+    const float* Xb = (d.model == SFB_DML) ? reinterpret_cast<const float*>(aux->Xb) : nullptr;
+    ACC(launch_forward_f32(c->stream, reinterpret_cast<const float*>(W), reinterpret_cast<const float*>(X), Xb, c->K,
+                           d.J, d.D, rows, none));
+  } else {
+    r = ensure_shadow(c, W);
+    if (r < 0) return r;
+    const bool bf16 = d.path == SFB_PATH_BF16;
+    ACC(umma_forward_rows(c->umma, c->stream, bf16 ? (const void*)c->w_shadow : W, caller_rows(X, d.D, d.B, c->l.es),
+                          rows, c->dev_status));
+  }
+  ACC(launch_sample_loss(c->stream, d.model, rows, aux->labels, aux->similar, d.margin, c->K, d.J, c->loss_i, loss,
+                         c->dev_status));
   return SFB_OK;
 }
 

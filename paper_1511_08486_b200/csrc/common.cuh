@@ -126,6 +126,10 @@ int launch_finish_sc(cudaStream_t s, RowMap z, RowMap u, const float* Xdata, int
 
 // Column-norm projection: every column of W with 2-norm above 1 is divided by its norm (in place).
 int launch_prox_unit_columns(cudaStream_t s, float* W, int J, int D);
+// Minibatch objective: per-sample values from the fp32 rows (z_i for MLR / DML, u_i for SC) into loss_i[K],
+// then their fp64 sum into *total (device).  Two launches.
+int launch_sample_loss(cudaStream_t s, int model, RowMap rows, const int32_t* labels, const uint8_t* similar, float margin,
+                       int K, int J, float* loss_i, double* total, int* dev_status);
 
 // W (fp32) -> bf16 shadow, round to nearest even.
 int launch_cast_bf16(cudaStream_t s, const float* W, __nv_bfloat16* Wb, long long n);

@@ -79,5 +79,12 @@ class DeviceWorkload:
         t = self.batches[t_idx % self.pool]
         self.ctx.step(self.W, t["X"], t["aux"], self.sf_buf, self.cfg["eta"] if eta is None else eta, K, clock=t_idx)
 
+    def loss(self, b: int = 0):
+        """Minibatch objective of batch b at the current W: a one-element float64 device tensor (asynchronous)."""
+        t = self.batches[b % self.pool]
+        out = torch.zeros(1, dtype=torch.float64, device=self.W.device)
+        self.ctx.loss(self.W, t["X"], t["aux"], out)
+        return out
+
     def close(self):
         self.ctx.destroy()

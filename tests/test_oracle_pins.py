@@ -386,3 +386,30 @@ def test_pack_sparse_v_roundtrip():
     with pytest.raises(ValueError):
         orc.pack(orc.MODEL_SC, orc.DTYPE_F32, cfg["J"], cfg["D"], cfg["P"], cfg["B"], U,
                  csr=(rowptr, idx, val), nnz_capacity=cfg["P"])
+
+
+def test_losses_closed_forms():
+    """Values the definitions fix: W = 0 gives K log J (uniform softmax); L = 0 gives margin / 2 per
+    dissimilar pair and 0 per similar pair; a dictionary that reproduces the data exactly gives 0, and
+    W = 0 gives half the squared norm of the data.  dml_loss also against the loop version."""
+    rng = np.random.default_rng(11)
+    K, J, D = 7, 5, 9
+    X = rng.standard_normal((K, D)).astype(np.float32)
+    y = rng.integers(0, J, K).astype(np.int32)
+    assert abs(orc.mlr_loss(np.zeros((J, D), np.float32), X, y) - K * np.log(J)) <= 1e-12
+    Xa, Xb = X, rng.standard_normal((K, D)).astype(np.float32)
+    sim = np.array([1, 0, 1, 0, 0, 1, 0], np.uint8)
+    assert abs(orc.dml_loss(np.zeros((J, D), np.float32), Xa, Xb, sim, 1.5) - 0.5 * 1.5 * 4) <= 1e-12
+    L = (0.2 * rng.standard_normal((J, D))).astype(np.float32)
+    want = loop_dml_loss(L.astype(np.float64).tolist(), Xa.astype(np.float64).tolist(), Xb.astype(np.float64).tolist(),
+                         sim.tolist(), 1.0)
+    assert abs(orc.dml_loss(L, Xa, Xb, sim, 1.0) - want) <= 1e-10
+    # sparse coding: codes with two nonzeros per sample, data = W a exactly (small integers: exact in fp32)
+    W = rng.integers(-3, 4, (J, D)).astype(np.float32)
+    rowptr = np.arange(0, 2 * K + 1, 2).astype(np.uint32)
+    idx = np.concatenate([np.sort(rng.choice(D, 2, replace=False)) for _ in range(K)]).astype(np.uint32)
+    val = rng.integers(1, 4, 2 * K).astype(np.float32)
+    A = orc.csr_to_dense(rowptr, idx, val, D)
+    Xd = (A @ W.T.astype(np.float64)).astype(np.float32)
+    assert orc.sc_loss(W, rowptr, idx, val, Xd) == 0.0
+    assert abs(orc.sc_loss(np.zeros_like(W), rowptr, idx, val, Xd) - 0.5 * float((Xd.astype(np.float64) ** 2).sum())) <= 1e-9
