@@ -214,6 +214,126 @@ def workload_name(cfg, path):
             f"K={cfg['K']} path={path}")
 
 
+def run_bsp(args, cfg, inputs, wl, path, rank, world, local_rank, barrier):
+    """One job over all ranks: rank r computes the factors of its P / world workers, the worker streams are
+    all-gathered in place (NCCL), every rank applies all K pairs to its own copy of W.  K samples per step in
+    total, whatever the number of ranks (strong scaling)."""
+    import torch
+    from paper_1511_08486_b200.bsp import BspSfb, exchange_bytes
+    from paper_1511_08486_b200.workload import shard_batch
+    dev = wl.W.device
+    stream = torch.cuda.current_stream()
+    K, eta = cfg["K"], cfg["eta"]
+    bsp = BspSfb(wl.ctx, wl.desc, wl.sf_buf)
+    shards = [shard_batch(t, cfg["model"], bsp.first, bsp.n_workers, cfg["B"]) for t in wl.batches]
+    step_bytes = 4.0 * cfg["J"] * cfg["D"] + wl.ctx.sf_buffer_bytes
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < (252 << 20) else None
+
+    def step(t):
+        s = shards[t % wl.pool]
+        bsp.step(wl.W, s["X"], s["aux"], eta, clock=t)
+
+    wl.reset()
+    for t in range(max(args.warmup, 3)):
+        step(t)
+    barrier()
+    l0 = wl.ctx.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    ms = 0.0
+    with ClockSampler(local_rank) as clocks:
+        if flush is None:
+            ev[0].record(stream)
+            for t in range(args.steps):
+                step(args.warmup + t)
+            ev[1].record(stream)
+            barrier()
+            ms = ev[0].elapsed_time(ev[1])
+        else:
+            for t in range(args.steps):
+                flush.fill_(t & 1)
+                barrier()
+                ev[0].record(stream)
+                step(args.warmup + t)
+                ev[1].record(stream)
+                torch.cuda.synchronize()
+                ms += ev[0].elapsed_time(ev[1])
+            barrier()
+    launches = wl.ctx.launch_count() - l0
+    status = wl.ctx.status()
+
+    # stages, timed apart: factors of the shard / exchange / header + apply
+    from paper_1511_08486_b200.bsp import all_gather_streams
+    st = [0.0, 0.0, 0.0]
+    nprof = min(args.steps, 16)
+    for t in range(nprof):
+        s = shards[t % wl.pool]
+        barrier()
+        ev[0].record(stream)
+        wl.ctx.factors_shard(wl.W, s["X"], s["aux"], wl.sf_buf, bsp.first, bsp.n_workers)
+        ev[1].record(stream)
+        if world > 1:
+            all_gather_streams(wl.sf_buf, bsp.streams_off, bsp.stream_stride, cfg["P"])
+        ev[2].record(stream)
+        wl.ctx.commit_header(wl.sf_buf, t)
+        wl.ctx.apply(wl.W, wl.sf_buf, eta)
+        ev[3].record(stream)
+        torch.cuda.synchronize()
+        for k in range(3):
+            st[k] += ev[k].elapsed_time(ev[k + 1]) / nprof
+
+    # end to end: the shard's minibatch starts in pinned host memory, the committed header comes back
+    host = [{k: v.cpu().pin_memory() for k, v in s.items() if isinstance(v, torch.Tensor)} for s in shards]
+    stage = [{k: torch.empty_like(v, device=dev) for k, v in h.items()} for h in host]
+    from paper_1511_08486_b200 import binding as Bd
+    stage_aux = [Bd.make_aux(**{k: v for k, v in sg.items() if k != "X"}) for sg in stage]
+    h2d = sum(v.numel() * v.element_size() for v in host[0].values())
+    header = torch.empty(128, dtype=torch.uint8).pin_memory()
+
+    def e2e_step(t):
+        b = t % wl.pool
+        for k, v in host[b].items():
+            stage[b][k].copy_(v, non_blocking=True)
+        bsp.step(wl.W, stage[b].get("X"), stage_aux[b], eta, clock=t)
+        header.copy_(wl.sf_buf[:128], non_blocking=True)
+    for t in range(3):
+        e2e_step(t)
+    barrier()
+    ev[0].record(stream)
+    for t in range(args.steps):
+        e2e_step(args.warmup + t)
+    ev[1].record(stream)
+    barrier()
+    e2e_ms = ev[0].elapsed_time(ev[1])
+    ms, e2e_ms, st[0], st[1], st[2] = max_over_ranks([ms, e2e_ms, st[0], st[1], st[2]], device=dev)
+    if rank != 0:
+        return None
+    peaks = load_peaks()
+    alg = algorithmic(cfg, path, inputs)
+    xb = exchange_bytes(cfg["P"], world, bsp.stream_stride)
+    out = {
+        "metric": METRIC, "value": whole_job_throughput(K, args.steps, ms, 1), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": path, "data": "synthetic",
+        "config": {"workload": workload_name(cfg, path), "parallelism": f"bsp sfb: {cfg['P']} workers over {world} gpu(s)",
+                   "l2": "per-step footprint larger than L2" if flush is None else "L2 flushed between steps",
+                   "eta": eta, "pool": cfg["pool"]},
+        "e2e": {"value": whole_job_throughput(K, args.steps, e2e_ms, 1), "unit": UNIT, "h2d_bytes_per_step": h2d * world,
+                "d2h_bytes_per_step": 128 * world},
+        "gpu_launches": int(launches), "device_status": status,
+        "stages_ms": {"factors": st[0], "exchange": st[1], "apply": st[2], "steps_recorded": nprof},
+        "exchange_bytes_per_step": xb,
+        "clocks": clocks.summary(),
+    }
+    if alg is not None and not alg["sparse"] and path != "f32":
+        scale = 1.0 if path == "bf16" else 0.5
+        peak = peaks["bf16_sustained"] * scale
+        tf = alg["flops"] / (st[2] * 1e-3) / 1e12
+        out["roofline"] = {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                           "traffic": None, "kernel": "umma_gemm_kernel (apply)",
+                           "peak_source": f"{peaks['source']} cuBLAS bf16 sustained" + ("" if path == "bf16" else " x 0.5 (tf32)")}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -223,6 +343,9 @@ def main():
     ap.add_argument("--config", default="C4")
     ap.add_argument("--path", default=None, help="f32 | tf32 | bf16 (default: the configuration's own)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "bsp"],
+                    help="N > 1: independent replicas of the whole path (default), or ONE job whose P workers are split "
+                         "over the ranks with an all-gather of the worker streams per step (sufficient factor broadcasting)")
     for dim in ("J", "D", "P", "B"):
         ap.add_argument(f"--{dim}", type=int, default=None, help=f"override {dim} (smaller cases for profiler captures)")
     args = ap.parse_args()
@@ -265,6 +388,15 @@ def main():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.mode == "bsp":
+        out = run_bsp(args, cfg, inputs, wl, path, rank, world, local_rank, barrier)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
+        wl.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # L2 flush buffer for workloads whose per-step footprint is below L2
     step_bytes = 4.0 * cfg["J"] * cfg["D"] + wl.ctx.sf_buffer_bytes
@@ -365,7 +497,7 @@ def main():
             if alg["sparse"]:
                 gbs = alg["bytes"] / (a_ms * 1e-3) / 1e9
                 out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                   "frac": gbs / peaks["hbm_gbs"], "traffic": traffic, "kernel": "sc_apply_kernel",
+                                   "frac": gbs / peaks["hbm_gbs"], "traffic": traffic, "kernel": "csc_apply_kernel",
                                    "peak_source": f"{peaks['source']} HBM copy bandwidth"}
             elif path == "f32":
                 out["roofline"] = {"bound": "alu", "achieved": apply_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",

@@ -153,6 +153,33 @@ int sfb_step(sfb_ctx* ctx, void* W, const void* X, const sfb_aux* aux, void* sf_
 int sfb_step_host(sfb_ctx* ctx, void* W, const void* X_host, const sfb_aux* aux_host, void* sf_buf, float eta,
                   int32_t K, uint32_t clock, void* header_host);
 
+/* The step as P real workers take it (Section 3, "Sufficient factor broadcasting": every worker computes
+ * the SF pairs of its own data shard against its full local copy of W, broadcasts them to all other
+ * workers, and applies every worker's pairs to its copy; BSP, Section 4: all workers apply the same set of
+ * pairs at every clock).  A process that owns workers [first_worker, first_worker + n_workers) of the P
+ * in the descriptor calls, per clock,
+ *   1. sfb_factors_shard: the pairs of ITS n_workers * B samples, written straight into those workers'
+ *      streams of the P-worker SF buffer (X, aux: the shard's minibatch only, laid out as for
+ *      sfb_compute_factors with P = n_workers; SFB_SC row pointers start at 0).  Other streams untouched.
+ *   2. the exchange (the caller's: the worker streams are contiguous and equally long, so an all-gather
+ *      over bytes [streams_off, streams_off + P * stream_stride) of the buffer, each process contributing
+ *      the streams it owns, in place, is the whole broadcast; header words 40..47 and 56..63 hold
+ *      stream_stride and streams_off, see sfb_sf_buffer_layout).
+ *   3. sfb_commit_header (header and directory, identical on every process; the SFB_SC directory takes each
+ *      worker's nonzero count from the stream it received) and sfb_apply with K = P * B.
+ * With one process owning all P workers the three calls leave exactly the W and SF buffer of sfb_step.
+ * The factors of a worker do not depend on which other workers share its process, except through the
+ * tile geometry the library picks for the shard's size (a split reduction, the width of the partial
+ * softmax tiles): bit-identical in most configurations, always far inside the path's tolerance.
+ * Returns SFB_ERR_ARG for a worker range outside [0, P).  Nothing is exchanged by the library. */
+int sfb_factors_shard(sfb_ctx* ctx, const void* W, const void* X, const sfb_aux* aux, void* sf_buf,
+                      int32_t first_worker, int32_t n_workers);
+int sfb_commit_header(sfb_ctx* ctx, void* sf_buf, uint32_t clock);
+
+/* Byte range of the worker streams inside the SF buffer of a descriptor: streams_off = offset of worker
+ * 0's stream, stream_stride = bytes per worker stream (both multiples of 128).  Host-only arithmetic. */
+int sfb_sf_buffer_layout(const sfb_desc* desc, uint64_t* streams_off, uint64_t* stream_stride);
+
 /* Proximal operator applied after the update (Section 2.1: prox_{eta h}; Section 3: "finally each
  * worker applies the proximal operator").  SFB_SC: h is the indicator of ||W_k||_2 <= 1 for every
  * column (atom) k, so each column whose norm exceeds 1 is divided by its norm and the others are

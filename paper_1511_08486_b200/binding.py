@@ -24,7 +24,7 @@ EXPORTS = (
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
     "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
     "sfb_halton_peers", "sfb_ssp_may_proceed", "sfb_prox", "sfb_step_host",
-    "sfb_loss",
+    "sfb_loss", "sfb_factors_shard", "sfb_commit_header", "sfb_sf_buffer_layout",
 )
 
 
@@ -80,6 +80,12 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_prox.restype = C.c_int
     lib.sfb_loss.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp]
     lib.sfb_loss.restype = C.c_int
+    lib.sfb_factors_shard.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, C.c_int32, C.c_int32]
+    lib.sfb_factors_shard.restype = C.c_int
+    lib.sfb_commit_header.argtypes = [vp, vp, C.c_uint32]
+    lib.sfb_commit_header.restype = C.c_int
+    lib.sfb_sf_buffer_layout.argtypes = [C.POINTER(sfb_desc), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    lib.sfb_sf_buffer_layout.restype = C.c_int
     lib.sfb_invalidate.argtypes = [vp]
     lib.sfb_invalidate.restype = C.c_int
     lib.sfb_status.argtypes = [vp, C.POINTER(C.c_int32)]
@@ -129,6 +135,15 @@ def make_aux(labels=None, Xb=None, similar=None, rowptr=None, idx=None, val=None
 
 def sfb_sf_buffer_bytes(desc: sfb_desc) -> int:
     return int(load_library().sfb_sf_buffer_bytes(C.byref(desc)))
+
+
+def sfb_sf_buffer_layout(desc: sfb_desc) -> tuple[int, int]:
+    """(streams_off, stream_stride) in bytes: where the worker streams sit inside the SF buffer."""
+    off, stride = C.c_uint64(0), C.c_uint64(0)
+    r = load_library().sfb_sf_buffer_layout(C.byref(desc), C.byref(off), C.byref(stride))
+    if r != SFB_OK:
+        raise SfbError(r, "sfb_sf_buffer_layout")
+    return int(off.value), int(stride.value)
 
 
 def sfb_ld(desc: sfb_desc) -> tuple[int, int]:
@@ -219,6 +234,13 @@ class Context:
 
     def prox(self, W):
         self._chk(self._lib.sfb_prox(self._h, _ptr(W)), "sfb_prox")
+
+    def factors_shard(self, W, X, aux: sfb_aux, sf_buf, first_worker: int, n_workers: int):
+        self._chk(self._lib.sfb_factors_shard(self._h, _ptr(W), _ptr(X), C.byref(aux), _ptr(sf_buf), first_worker,
+                                              n_workers), "sfb_factors_shard")
+
+    def commit_header(self, sf_buf, clock: int = 0):
+        self._chk(self._lib.sfb_commit_header(self._h, _ptr(sf_buf), clock), "sfb_commit_header")
 
     def loss(self, W, X, aux: sfb_aux, out):
         """Minibatch objective at W into `out` (one float64 on the device); asynchronous."""

@@ -130,26 +130,29 @@ int ensure_shadow(sfb_ctx* c, const void* W) {
 }
 
 // Factors of one minibatch written through the row maps u / v (v.base == nullptr: v not wanted).
-int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, RowMap u, RowMap v, CsrView codes) {
+// workers > 0: the minibatch holds only that many workers' samples and u / v / codes start at the first of them.
+int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, RowMap u, RowMap v, CsrView codes,
+                 int workers = 0) {
   const sfb_desc& d = c->d;
+  const int K = workers > 0 ? workers * d.B : c->K;
   const float* Wf = reinterpret_cast<const float*>(W);
   if (d.model == SFB_SC && d.path == SFB_PATH_F32) {
-    ACC(launch_sc_forward_ws(c->stream, Wf, c->wt_ws, codes, reinterpret_cast<const float*>(aux->Xdata), u, c->K, d.J,
+    ACC(launch_sc_forward_ws(c->stream, Wf, c->wt_ws, codes, reinterpret_cast<const float*>(aux->Xdata), u, K, d.J,
                              d.D, c->dev_status));
     return SFB_OK;
   }
   if (d.model == SFB_SC) {   // dense alternative: the codes as dense tf32 rows through the tensor-core GEMM
     const RowMap a = dense_codes(c);
-    ACC(launch_densify_codes(c->stream, codes, a, c->K, d.D, c->dev_status));
-    ACC(umma_forward_rows(c->umma, c->stream, W, a, u, c->dev_status));
-    ACC(launch_finish_sc(c->stream, u, u, reinterpret_cast<const float*>(aux->Xdata), c->K, d.J));
+    ACC(launch_densify_codes(c->stream, codes, a, K, d.D, c->dev_status));
+    ACC(umma_forward_rows(c->umma, c->stream, W, a, u, c->dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers));
+    ACC(launch_finish_sc(c->stream, u, u, reinterpret_cast<const float*>(aux->Xdata), K, d.J));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {
     const float* Xb = (d.model == SFB_DML) ? reinterpret_cast<const float*>(aux->Xb) : nullptr;
-    ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, c->K, d.J, d.D, u, v));
-    if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, u, u, aux->labels, c->K, d.J, c->dev_status));
-    else ACC(launch_finish_dml(c->stream, u, u, aux->similar, d.margin, c->K, d.J));
+    ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, K, d.J, d.D, u, v));
+    if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, u, u, aux->labels, K, d.J, c->dev_status));
+    else ACC(launch_finish_dml(c->stream, u, u, aux->similar, d.margin, K, d.J));
     return SFB_OK;
   }
   // tensor-core paths
@@ -157,7 +160,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     const int r = ensure_shadow(c, W);
     if (r < 0) return r;
   }
-  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, z_rows(c), c->dev_status));
+  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, z_rows(c), c->dev_status, workers));
   return SFB_OK;
 }
 
@@ -181,6 +184,16 @@ const char* sfb_strerror(int code) {
 size_t sfb_sf_buffer_bytes(const sfb_desc* desc) {
   if (check_desc(desc) != SFB_OK) return 0;
   return (size_t)make_layout(*desc).total_bytes;
+}
+
+int sfb_sf_buffer_layout(const sfb_desc* desc, uint64_t* streams_off, uint64_t* stream_stride) {
+  if (streams_off == nullptr || stream_stride == nullptr) return SFB_ERR_ARG;
+  const int r = check_desc(desc);
+  if (r != SFB_OK) return r;
+  const Layout l = make_layout(*desc);
+  *streams_off = (uint64_t)l.streams_off;
+  *stream_stride = (uint64_t)l.stream_stride;
+  return SFB_OK;
 }
 
 int sfb_ld(const sfb_desc* desc, int32_t* ldu, int32_t* ldv) {
@@ -410,6 +423,35 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
     ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status));
     if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
   }
+  return SFB_OK;
+}
+
+int sfb_factors_shard(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, void* sf_buf, int32_t first_worker,
+                      int32_t n_workers) {
+  if (c == nullptr || W == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
+  if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
+  const sfb_desc& d = c->d;
+  if (first_worker < 0 || n_workers <= 0 || first_worker > d.P - n_workers) return SFB_ERR_ARG;
+  int r = check_aux(c, aux);
+  if (r != SFB_OK) return r;
+  if (d.model != SFB_SC && (X == nullptr || !aligned(X, 16))) return SFB_ERR_ARG;
+  // the shard's streams: every offset below is relative to the first of them
+  char* shard = reinterpret_cast<char*>(sf_buf) + (long long)first_worker * c->l.stream_stride;
+  CsrView codes;
+  memset(&codes, 0, sizeof(codes));
+  if (d.v_sparse) {
+    sfb_desc ds = d;
+    ds.P = n_workers;
+    ACC(launch_pack_csr(c->stream, shard, ds, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
+                        c->dev_status));
+    codes = stream_codes(c, shard);
+  }
+  return factors_into(c, W, X, aux, stream_u(c, shard), d.v_sparse ? RowMap() : stream_v(c, shard), codes, n_workers);
+}
+
+int sfb_commit_header(sfb_ctx* c, void* sf_buf, uint32_t clock) {
+  if (c == nullptr || sf_buf == nullptr || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
+  ACC(launch_write_header(c->stream, sf_buf, c->d, c->l, clock, nullptr));
   return SFB_OK;
 }
 

@@ -53,6 +53,8 @@ __global__ void write_header_kernel(char* buf, HeaderImage h, long long u_bytes,
           if (rowptr != nullptr) {
             const uint32_t n = rowptr[(p + 1) * h.B] - rowptr[p * h.B];
             val = n < h.cap_p ? n : h.cap_p;
+          } else if (h.flags & 1u) {   // no global row pointers: the count the worker's own stream carries
+            val = reinterpret_cast<const uint32_t*>(buf + v_off)[h.B];
           }
           break;
         case 4: val = (uint32_t)(u_off & 0xffffffffu); break;

@@ -810,15 +810,16 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
 int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
                       float2* stats, int* n_parts_out, int* part_cols_out, int* k_splits_out, int max_splits,
-                      long long split_stride) {
+                      long long split_stride, int workers) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
+  const int P = workers > 0 ? workers : d.P;     // a shard of the workers, or all of them
   GemmParams p;
   memset(&p, 0, sizeof(p));
-  p.B = d.B; p.P = d.P;
+  p.B = d.B; p.P = P;
   int m_units;
-  if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; m_units = d.P * p.m_tpw; }
-  else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; m_units = (d.P + p.m_wp - 1) / p.m_wp; }
+  if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; m_units = P * p.m_tpw; }
+  else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; m_units = (P + p.m_wp - 1) / p.m_wp; }
   // folding walks the reduction index (D) in 128-byte atoms: rows must be whole atoms long
   const Variant v = pick_variant(pl, m_units, d.J, (d.D % CH) == 0 && (a.ld % CH) == 0);
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
@@ -839,7 +840,7 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.k_per_split = (p.k_blocks + p.k_splits - 1) / p.k_splits;
   p.split_stride = split_stride;
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
-  p.m_fastest = ((long long)d.J * d.D > (long long)d.P * d.B * d.D) ? 1 : 0;
+  p.m_fastest = ((long long)d.J * d.D > (long long)P * d.B * d.D) ? 1 : 0;
   p.a_policy = p.m_fastest ? 2 : 0;   // the operand whose slab changes every tile is re-read all along: keep it
   p.b_policy = p.m_fastest ? 0 : 2;
   p.group = pl->fwd_group;
@@ -851,7 +852,7 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   if (n_parts_out != nullptr) *n_parts_out = p.n_parts;
   if (part_cols_out != nullptr) *part_cols_out = v.bn / 2;
   CUtensorMap ta, tb;
-  if (!encode_rows_map(&ta, es, a.base, d.D, d.B, d.P, (long long)a.ld * es, a.worker_stride, p.m_bb, p.m_wp, v.fold,
+  if (!encode_rows_map(&ta, es, a.base, d.D, d.B, P, (long long)a.ld * es, a.worker_stride, p.m_bb, p.m_wp, v.fold,
                        v.ka, false))
     return SFB_ERR_CUDA;
   if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, v.bn / v.cg, 1,
@@ -862,9 +863,9 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
-                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status) {
+                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status, int workers) {
   const sfb_desc& d = pl->d;
-  const int K = d.P * d.B;
+  const int K = (workers > 0 ? workers : d.P) * d.B;
   int launches = 0, r;
   RowMap x_rows;
   x_rows.base = const_cast<char*>(reinterpret_cast<const char*>(X));
@@ -880,10 +881,10 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
       RowMap pz;
       pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
       pz.worker_stride = (long long)d.B * pl->ldp * 4;
-      const long long sstride = (long long)K * pl->ldp * 4;
+      const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
       int ks = 1;
       if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr, nullptr,
-                                 &ks, 4, sstride)) < 0)
+                                 &ks, 4, sstride, workers)) < 0)
         return r;
       launches += r;
       if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
@@ -897,7 +898,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     int n_parts = 0, part_cols = 0;
     (void)zz;
     if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
-                               &part_cols)) < 0)
+                               &part_cols, nullptr, 1, 0, workers)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status)) < 0) return r;
@@ -917,14 +918,15 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     RowMap pz;
     pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
-    const long long sstride = (long long)K * pl->ldp * 4;
+    const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, 4, sstride)) < 0) return r;
+    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, 4, sstride, workers)) < 0)
+      return r;
     launches += r;
     if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
     return launches + r;
   }
-  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr)) < 0) return r;
+  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers)) < 0) return r;
   launches += r;
   if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
   return launches + r;

@@ -13,13 +13,14 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
 void umma_plan_destroy(UmmaPlan* p);
 
 // z = W a on the tensor cores followed by the model epilogue; factors go through u / v row maps.
+// workers > 0: only that many workers' samples (X, aux, u, v start at the first of them).
 int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
-                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status);
+                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status, int workers = 0);
 
 // Z rows (fp32) = A rows (the path's value type) times Wop^T on the tensor cores; no epilogue beyond the store.
 int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
                       float2* stats = nullptr, int* n_parts_out = nullptr, int* part_cols_out = nullptr,
-                      int* k_splits_out = nullptr, int max_splits = 1, long long split_stride = 0);
+                      int* k_splits_out = nullptr, int max_splits = 1, long long split_stride = 0, int workers = 0);
 
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
 // u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).

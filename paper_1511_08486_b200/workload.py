@@ -15,6 +15,33 @@ def bf16_tensor(bits: np.ndarray, device) -> torch.Tensor:
     return torch.from_numpy(bits.view(np.int16).copy()).to(device).view(torch.bfloat16)
 
 
+def shard_batch(t: dict, model: str, first_worker: int, n_workers: int, Bsz: int) -> dict:
+    """The part of a device minibatch `t` that belongs to workers [first_worker, first_worker + n_workers).
+
+    Fresh contiguous tensors (so every pointer is aligned) plus the matching `aux`; sparse codes get
+    row pointers that start at 0.  Copies only: what a process of a multi-process run would hold.
+    """
+    lo, hi = first_worker * Bsz, (first_worker + n_workers) * Bsz
+    s = {}
+    if model == "mlr":
+        s["X"], s["labels"] = t["X"][lo:hi].clone(), t["labels"][lo:hi].clone()
+        s["aux"] = B.make_aux(labels=s["labels"])
+    elif model == "dml":
+        s["X"], s["Xb"], s["similar"] = t["X"][lo:hi].clone(), t["Xb"][lo:hi].clone(), t["similar"][lo:hi].clone()
+        s["aux"] = B.make_aux(Xb=s["Xb"], similar=s["similar"])
+    else:
+        rp = t["rowptr"][lo:hi + 1].clone()
+        e0, e1 = int(rp[0].item()), int(rp[-1].item())
+        s["X"] = None
+        s["rowptr"] = rp - e0
+        # keep at least one element so that the pointers are valid for a shard without nonzeros
+        s["idx"] = t["idx"][e0:max(e1, e0 + 1)].clone() if t["idx"].numel() > e0 else torch.zeros_like(t["idx"][:1])
+        s["val"] = t["val"][e0:max(e1, e0 + 1)].clone() if t["val"].numel() > e0 else torch.zeros_like(t["val"][:1])
+        s["Xdata"] = t["Xdata"][lo:hi].clone()
+        s["aux"] = B.make_aux(rowptr=s["rowptr"], idx=s["idx"], val=s["val"], Xdata=s["Xdata"])
+    return s
+
+
 class DeviceWorkload:
     """Device copies of the inputs of configuration `cfg`, a context, and the SF buffer."""
 
