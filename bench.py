@@ -32,6 +32,7 @@ if ROOT not in sys.path:
 
 METRIC = "SF-step samples/s"
 UNIT = "samples/s"
+SMEM_TBS = 148 * 128 * 1.965e9 / 1e12           # shared-memory load path of the whole chip
 DATASHEET_BF16_TFLOPS = 2250.0
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 lanes x 2 flop x max SM clock
 
@@ -136,7 +137,7 @@ def algorithmic(cfg, path, inputs=None):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one apply launch, from the ncu captures summarised
 # under profiles/ (captured at J = 8192 and scaled by J where the full launch is too large to capture).
-NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 4.03e9}
+NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 4.03e9, ("C3", "f32"): 6.28e8}
 
 
 def oracle_step_time(cfg, inputs, sample_workers: int):
@@ -499,6 +500,11 @@ def main():
                 out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": gbs / peaks["hbm_gbs"], "traffic": traffic, "kernel": "csc_apply_kernel",
                                    "peak_source": f"{peaks['source']} HBM copy bandwidth"}
+                # what the counters show as the limiter: every multiply-add takes 4 bytes of u from shared memory
+                smem_tbs = 2.0 * alg["flops"] / (a_ms * 1e-3) / 1e12
+                out["roofline"]["secondary"] = {"bound": "shared-memory operand reads", "achieved": smem_tbs,
+                                                "peak": SMEM_TBS, "unit": "TB/s", "frac": smem_tbs / SMEM_TBS,
+                                                "peak_source": "148 SMs x 128 B/clk x 1.965 GHz"}
             elif path == "f32":
                 out["roofline"] = {"bound": "alu", "achieved": apply_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
                                    "frac": apply_tflops / FP32_FMA_TFLOPS, "traffic": None,
