@@ -20,6 +20,8 @@ struct sfb_ctx {
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
   void* csc_ws;             // SC, fp32 path: scratch of the atom-major re-sort of the codes (when K fits)
+  float* f32_part;          // fp32 dense path: partial products [splits][K][ldp] of a split forward reduction
+  int ldp, f32_splits;
   float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
   float* loss_i;            // sfb_loss: per-sample objective [K]
   // sfb_step_host: two sets of device staging buffers for the step's host inputs (allocated on first
@@ -150,9 +152,15 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
   }
   if (d.path == SFB_PATH_F32) {
     const float* Xb = (d.model == SFB_DML) ? reinterpret_cast<const float*>(aux->Xb) : nullptr;
-    ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, K, d.J, d.D, u, v));
-    if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, u, u, aux->labels, K, d.J, c->dev_status));
-    else ACC(launch_finish_dml(c->stream, u, u, aux->similar, d.margin, K, d.J));
+    // partial products of a split reduction live in the context's workspace, laid out like caller rows
+    const RowMap part = caller_rows(c->f32_part, c->ldp, d.B, 4);
+    const long long sstride = (long long)c->K * c->ldp * 4;
+    int ks = 1;
+    ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, K, d.J, d.D, u, v, part, sstride,
+                           c->f32_splits, &ks));
+    const RowMap zsrc = ks > 1 ? part : u;
+    if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, zsrc, u, aux->labels, K, d.J, c->dev_status, ks, sstride));
+    else ACC(launch_finish_dml(c->stream, zsrc, u, aux->similar, d.margin, K, d.J, ks, sstride));
     return SFB_OK;
   }
   // tensor-core paths
@@ -229,6 +237,12 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     ok = cudaMalloc(&c->csc_ws, (size_t)sc_csc_workspace_bytes(c->K, desc->D, (long long)desc->nnz_capacity)) == cudaSuccess;
   if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_TF32)
     ok = cudaMalloc(&c->a_dense, (size_t)c->K * c->l.ldv * 4) == cudaSuccess;
+  if (ok && desc->model != SFB_SC && desc->path == SFB_PATH_F32) {
+    const int ks = forward_f32_splits(c->K, desc->J, desc->D);
+    c->ldp = (desc->J + 3) & ~3;
+    c->f32_splits = ks;
+    if (ks > 1) ok = cudaMalloc(&c->f32_part, (size_t)ks * c->K * c->ldp * 4) == cudaSuccess;
+  }
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -258,6 +272,7 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->wt_ws) cudaFree(c->wt_ws);
   if (c->a_dense) cudaFree(c->a_dense);
   if (c->csc_ws) cudaFree(c->csc_ws);
+  if (c->f32_part) cudaFree(c->f32_part);
   if (c->loss_rows) cudaFree(c->loss_rows);
   if (c->loss_i) cudaFree(c->loss_i);
   for (int k = 0; k < 2; ++k)

@@ -60,8 +60,13 @@ static inline Layout make_layout(const sfb_desc& d) {
 // Z[i][j] = sum_d A[i][d] * W[j][d] on fp32 CUDA cores, written as fp32 rows through `z`.
 // A = X, or X - Xb (element-wise fp32 subtraction) when Xb != nullptr.  When `v` has a base, the
 // operand rows (X, or the difference) are also written there (the factor v), pad columns zero.
+// With a `part` row map (fp32 rows, split_stride bytes between partial buffers) and nsplit_out, a problem
+// with few tiles has its reduction cut into *nsplit_out ranges whose partial products go to `part` instead
+// of `z` (the finishing pass sums them in range order); forward_f32_splits tells how many in advance.
+int forward_f32_splits(int K, int J, int D);
 int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
-                       RowMap z, RowMap v);
+                       RowMap z, RowMap v, RowMap part = RowMap(), long long split_stride = 0, int max_splits = 1,
+                       int* nsplit_out = nullptr);
 
 // W[j][d] -= eta * sum_{i<K} U[i][j] * V[i][d] on fp32 CUDA cores (fixed summation order).
 int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J, int D, float eta,

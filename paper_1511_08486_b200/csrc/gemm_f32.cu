@@ -55,7 +55,7 @@ __device__ __forceinline__ void mma_tile(const float (*As)[64 * MI + 4], const f
 template <int MI, int NI>
 __global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __restrict__ W, const float* __restrict__ X,
                                                           const float* __restrict__ Xb, int K, int J, int D,
-                                                          RowMap z, RowMap v) {
+                                                          RowMap z, RowMap v, int d_per_split, long long split_stride) {
   constexpr int BM = 64 * MI, BN = 64 * NI;
   __shared__ __align__(16) float As[BK][BM + 4];
   __shared__ __align__(16) float Bs[BK][BN + 4];
@@ -106,11 +106,15 @@ __global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __rest
     }
   };
 
-  fetch(0);
-  for (int d0 = 0; d0 < D; d0 += BK) {
+  // blockIdx.z takes the reduction range [d_lo, d_hi) and writes its partial products split_stride bytes
+  // after the previous range's (one range: the whole reduction, written to z itself)
+  const int d_lo = blockIdx.z * d_per_split;
+  const int d_hi = min(D, d_lo + d_per_split);
+  fetch(d_lo);
+  for (int d0 = d_lo; d0 < d_hi; d0 += BK) {
     stash();
     __syncthreads();
-    if (d0 + BK < D) fetch(d0 + BK);
+    if (d0 + BK < d_hi) fetch(d0 + BK);
     mma_tile<MI, NI>(As, Bs, ty, tx, acc);
     __syncthreads();
   }
@@ -123,7 +127,7 @@ __global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __rest
     for (int a = 0; a < 4; ++a) {
       const int i = i0 + mi * 64 + ty * 4 + a;
       if (i >= K) continue;
-      float* zr = reinterpret_cast<float*>(z.row(i));
+      float* zr = reinterpret_cast<float*>(z.row(i) + blockIdx.z * split_stride);
 #pragma unroll
       for (int ni = 0; ni < NI; ++ni) {
         const int j = j0 + ni * 64 + tx * 4;
@@ -214,15 +218,34 @@ __global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W
 
 }  // namespace
 
-int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
-                       RowMap z, RowMap v) {
+// Few 128 x 128 tiles and a long reduction (e.g. 1024 samples x 1000 classes over 20000 features): the
+// reduction is cut into up to 4 ranges so that every SM has two blocks of the large-tile kernel.
+int forward_f32_splits(int K, int J, int D) {
   const long long big_tiles = (long long)((K + 127) / 128) * ((J + 127) / 128);
-  if (big_tiles >= 148) {
+  if (big_tiles >= 148) return 1;
+  long long ks = (2 * 148) / big_tiles;
+  if (ks > 4) ks = 4;
+  while (ks > 1 && D / ks < 512) --ks;
+  return (int)ks;
+}
+
+int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
+                       RowMap z, RowMap v, RowMap part, long long split_stride, int max_splits, int* nsplit_out) {
+  if (nsplit_out != nullptr) *nsplit_out = 1;
+  const long long big_tiles = (long long)((K + 127) / 128) * ((J + 127) / 128);
+  int ks = (part.base != nullptr && nsplit_out != nullptr) ? forward_f32_splits(K, J, D) : 1;
+  if (ks > max_splits) ks = max_splits;       // the partial buffers the caller owns
+  if (ks > 1) {
+    const int per = ((D + ks - 1) / ks + BK - 1) / BK * BK;
+    dim3 grid((J + 127) / 128, (K + 127) / 128, ks);
+    forward_f32_kernel<2, 2><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, part, v, per, split_stride);
+    *nsplit_out = ks;
+  } else if (big_tiles >= 148) {
     dim3 grid((J + 127) / 128, (K + 127) / 128);
-    forward_f32_kernel<2, 2><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, z, v);
+    forward_f32_kernel<2, 2><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, z, v, D, 0);
   } else {
     dim3 grid((J + 63) / 64, (K + 63) / 64);
-    forward_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, z, v);
+    forward_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, X, Xb, K, J, D, z, v, D, 0);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
