@@ -216,6 +216,97 @@ __global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W
     }
 }
 
+// ---- apply, large tiles: the factor rows go to shared memory as they are, so they are fetched with
+// 16-byte asynchronous copies (zero-filled beyond K, J and D) through a ring of PIPE stages: one barrier
+// per reduction step, no staging registers.
+constexpr int PIPE = 4;
+constexpr int PIPE_STAGE_FLOATS = 2 * BK * (128 + 4);
+
+__device__ __forceinline__ void cp_async16_zfill(float* dst_smem, const void* src, int src_bytes) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst_smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
+                                                             int D, float eta, const int* __restrict__ dev_status) {
+  constexpr int BM = 128, BN = 128;
+  extern __shared__ __align__(16) float ring[];
+  if (dev_status != nullptr && (*dev_status & SFB_DEV_BAD_HEADER)) return;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int j0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
+  const int lr = tid >> 5, lc = (tid & 31) * 4;   // loader: factor rows lr and lr + 8 of the step, 4 columns at lc
+  // bytes of this thread's 16-byte piece that exist (the rest is zero-filled); a piece with nothing to read
+  // still needs a valid aligned address: column 0 of a valid row
+  const int ju = j0 + lc, dv = d0 + lc;
+  const int u_bytes = max(0, min(16, (J - ju) * 4)), v_bytes = max(0, min(16, (D - dv) * 4));
+  const size_t u_off = u_bytes > 0 ? (size_t)ju * 4 : 0, v_off = v_bytes > 0 ? (size_t)dv * 4 : 0;
+
+  auto issue = [&](int stage, int k0) {
+    float* As = ring + stage * PIPE_STAGE_FLOATS;
+    float* Bs = As + BK * (BM + 4);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int r = lr + 8 * h, i = k0 + r;
+      const bool ok = i < K;
+      const int ii = ok ? i : 0;
+      cp_async16_zfill(As + r * (BM + 4) + lc, u.row(ii) + u_off, ok ? u_bytes : 0);
+      cp_async16_zfill(Bs + r * (BN + 4) + lc, v.row(ii) + v_off, ok ? v_bytes : 0);
+    }
+  };
+
+  float acc[8][8];
+#pragma unroll
+  for (int m = 0; m < 8; ++m)
+#pragma unroll
+    for (int n = 0; n < 8; ++n) acc[m][n] = 0.f;
+
+  const int nk = (K + BK - 1) / BK;
+#pragma unroll
+  for (int st = 0; st < PIPE - 1; ++st) {
+    if (st < nk) issue(st, st * BK);
+    cp_async_commit();
+  }
+  for (int kt = 0; kt < nk; ++kt) {
+    cp_async_wait<PIPE - 2>();       // this thread's pieces of step kt have landed
+    __syncthreads();                 // ... everybody's have, and everybody is done with step kt - 1
+    const int nxt = kt + PIPE - 1;
+    if (nxt < nk) issue(nxt % PIPE, nxt * BK);
+    cp_async_commit();
+    const float* As = ring + (kt % PIPE) * PIPE_STAGE_FLOATS;
+    mma_tile<2, 2>(reinterpret_cast<const float(*)[BM + 4]>(As), reinterpret_cast<const float(*)[BN + 4]>(As + BK * (BM + 4)),
+                   ty, tx, acc);
+  }
+  cp_async_wait<0>();
+
+  const bool vec_ok = (D & 3) == 0;
+#pragma unroll
+  for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int j = j0 + mi * 64 + ty * 4 + a;
+      if (j >= J) continue;
+      float* wr = W + (size_t)j * D;
+#pragma unroll
+      for (int ni = 0; ni < 2; ++ni) {
+        const int d = d0 + ni * 64 + tx * 4;
+        const float* c = acc[mi * 4 + a] + ni * 4;
+        if (vec_ok && d + 3 < D) {
+          float4 w = *reinterpret_cast<float4*>(wr + d);
+          w.x = fmaf(-eta, c[0], w.x); w.y = fmaf(-eta, c[1], w.y);
+          w.z = fmaf(-eta, c[2], w.z); w.w = fmaf(-eta, c[3], w.w);
+          *reinterpret_cast<float4*>(wr + d) = w;
+        } else {
+#pragma unroll
+          for (int b = 0; b < 4; ++b)
+            if (d + b < D) wr[d + b] = fmaf(-eta, c[b], wr[d + b]);
+        }
+      }
+    }
+}
+
 }  // namespace
 
 // Few 128 x 128 tiles and a long reduction (e.g. 1024 samples x 1000 classes over 20000 features): the
@@ -255,7 +346,12 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
   const long long big_tiles = (long long)((J + 127) / 128) * ((D + 127) / 128);
   if (big_tiles >= 148) {
     dim3 grid((D + 127) / 128, (J + 127) / 128);
-    apply_f32_kernel<2, 2><<<grid, 256, 0, s>>>(W, u, v, K, J, D, eta, dev_status);
+    static bool attr_done = false;
+    if (!attr_done) {
+      cudaFuncSetAttribute(apply_f32_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE * PIPE_STAGE_FLOATS * 4);
+      attr_done = true;
+    }
+    apply_f32_pipe_kernel<<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(W, u, v, K, J, D, eta, dev_status);
   } else {
     dim3 grid((D + 63) / 64, (J + 63) / 64);
     apply_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, u, v, K, J, D, eta, dev_status);
