@@ -165,10 +165,17 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def pick_sample_workers(cfg):
-    """Workers whose samples make up the oracle's bounded sample (~10-30 s of host work)."""
+def pick_sample_workers(cfg, budget=1.5e12):
+    """Workers whose samples make up the oracle's bounded sample.
+
+    budget: fp64 flops of one sampled oracle step.  The reference arm repeats the step `--steps` times, so it
+    takes the default (a few seconds per step on the GPU machine's host); the cpu_baseline leg times ONE step and
+    asks for more (10-30 s).  The sparse-coding oracle spends its time in per-sample scatter loops, not flops:
+    a quarter of the workers there.
+    """
+    if cfg["model"] == "sc":
+        return max(1, cfg["P"] // 4)
     flops_per_worker = 4.0 * cfg["J"] * cfg["D"] * cfg["B"]           # forward + apply, fp64
-    budget = 1.5e12                                                    # ~15 s at ~100 GFLOP/s
     return int(max(1, min(cfg["P"], budget // max(flops_per_worker, 1.0))))
 
 
@@ -520,7 +527,7 @@ def main():
             out["apply_tflops"] = apply_tflops
             out["forward_tflops"] = fwd_tflops
         if not args.no_cpu_baseline:
-            sw = pick_sample_workers(cfg)
+            sw = pick_sample_workers(cfg, budget=6e12)
             dt, n = oracle_step_time(cfg, inputs, sw)
             out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                    "sample": f"one oracle step on {sw} of {cfg['P']} workers' samples ({n} of {K}) at full J x D, {dt:.1f} s"}

@@ -25,6 +25,11 @@
  *     index out of range or unsorted, SF-buffer header not matching the descriptor, CSR capacity
  *     exceeded) set bits of a sticky device status word and make the kernel that found them skip
  *     the affected writes; nothing traps.  Read the word with sfb_status.
+ *   - A context is not thread-safe: calls on one context come from one host thread at a time.  Different
+ *     contexts are independent (also on different devices of one process; a context belongs to the
+ *     device that was current in sfb_create, which must be current again for every call on it).
+ *   - "allocates only in sfb_create" has two stated exceptions, both on first use: the staging buffers
+ *     of sfb_step_host and the workspace of sfb_loss.
  *   - W is J x D, row-major fp32, updated in place.  Samples are rows: X is [K][D].
  *   - Sample i belongs to worker p = i / B, slot i % B.
  *

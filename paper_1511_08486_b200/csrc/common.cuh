@@ -55,6 +55,20 @@ static inline Layout make_layout(const sfb_desc& d) {
   return l;
 }
 
+// cudaFuncSetAttribute acts on the current device only: first() is true once per device (ordinals 0..63)
+// for the static object it is called on.  A repeated call from a racing thread would set the same value.
+struct PerDeviceOnce {
+  unsigned long long done = 0;
+  bool first() {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (done & bit) return false;
+    done |= bit;
+    return true;
+  }
+};
+
 // ---- kernel launchers (each returns the number of kernels it launched, or a negative SFB_ERR_*) ----
 
 // Z[i][j] = sum_d A[i][d] * W[j][d] on fp32 CUDA cores, written as fp32 rows through `z`.

@@ -350,11 +350,10 @@ int fin_cache_floats(int J) {
 int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
                       int nsplit, long long split_stride_bytes) {
   const int cf = fin_cache_floats(J);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;   // function attributes are per device
+  if (attr_once.first()) {
     cudaFuncSetAttribute(finish_mlr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
-    attr_done = true;
   }
   finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status, nsplit, split_stride_bytes / 4);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
@@ -363,11 +362,10 @@ int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels,
 int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
                       int nsplit, long long split_stride_bytes) {
   const int cf = fin_cache_floats(J);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;   // function attributes are per device
+  if (attr_once.first()) {
     cudaFuncSetAttribute(finish_mlr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
-    attr_done = true;
   }
   finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf, nsplit, split_stride_bytes / 4);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;

@@ -346,10 +346,9 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
   const long long big_tiles = (long long)((J + 127) / 128) * ((D + 127) / 128);
   if (big_tiles >= 148) {
     dim3 grid((D + 127) / 128, (J + 127) / 128);
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;   // function attributes are per device
+    if (attr_once.first()) {
       cudaFuncSetAttribute(apply_f32_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE * PIPE_STAGE_FLOATS * 4);
-      attr_done = true;
     }
     apply_f32_pipe_kernel<<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(W, u, v, K, J, D, eta, dev_status);
   } else {

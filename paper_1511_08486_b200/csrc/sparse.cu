@@ -319,11 +319,10 @@ int launch_finish_sc(cudaStream_t s, RowMap z, RowMap u, const float* Xdata, int
 
 int launch_sc_apply(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                     const int* dev_status_ro, int* /*dev_status*/) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;   // function attributes are per device
+  if (attr_once.first()) {
     cudaFuncSetAttribute(sc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SLAB_D * SLAB_J * 4);
     cudaFuncSetAttribute(sc_apply_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    attr_done = true;
   }
   dim3 grid((D + SLAB_D - 1) / SLAB_D, (J + SLAB_J - 1) / SLAB_J);
   sc_apply_kernel<<<grid, SLAB_T, SLAB_D * SLAB_J * 4, s>>>(W, codes, u, K, J, D, eta, dev_status_ro);

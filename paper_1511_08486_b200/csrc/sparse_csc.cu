@@ -266,10 +266,9 @@ int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K
   csc_scan_kernel<<<1, 1024, 0, s>>>(D, total, colptr);
   csc_fill_kernel<<<nchunks, 256, 0, s>>>(codes, K, D, cnt, colptr, ent_i, ent_a);
   const int threads = 512;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;   // function attributes are per device
+  if (attr_once.first()) {
     cudaFuncSetAttribute(csc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-    attr_done = true;
   }
   // slices of the samples: the fewest that let Kh x 256 bytes of u sit beside the warps' tiles
   const long long tiles = (long long)(threads / 32) * CSC2_WARP_FLOATS * 4;

@@ -655,9 +655,9 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
   constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
   constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
   auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD, EPI>;
-  static bool attr_done = false;
+  static PerDeviceOnce attr_once;   // function attributes are per device
   static int max_clusters = 0;
-  if (!attr_done) {
+  if (attr_once.first()) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return SFB_ERR_CUDA;
     if (CG == 2) {   // how many CTA pairs the device can hold at once
@@ -675,7 +675,6 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
         max_clusters = num_sms / 2;
       }
     }
-    attr_done = true;
   }
   const int tiles = p.m_tiles * p.n_tiles * p.k_splits;
   if (CG == 1) {
