@@ -727,6 +727,8 @@ int dispatch_gemm(cudaStream_t s, int es, const Variant& v, const CUtensorMap& a
 
 }  // namespace
 
+constexpr int MAX_SPLITS = 8;   // ranges a forward reduction may be cut into (partial buffers of the plan)
+
 struct UmmaPlan {
   sfb_desc d;
   Layout l;
@@ -739,7 +741,7 @@ struct UmmaPlan {
   int fold_ka;    // 128-byte atoms of the reduction index per stage in the folded kernels (SFB_FOLD_KA, default 2)
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
   int fwd_group, apply_group;   // tile-order group widths (SFB_FWD_GROUP / SFB_APPLY_GROUP override the defaults)
-  float* part_ws;               // partial products of a split reduction, [4][K][ldp] fp32 (small forward GEMMs only)
+  float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
   int ldp;
 };
 
@@ -764,10 +766,10 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   p->apply_group = ag != nullptr ? atoi(ag) : 8;
   p->part_ws = nullptr;
   p->ldp = (int)pad_to(d.J, 4);
-  {   // forward GEMMs with fewer 128 x 128 tiles than half the SMs may split their reduction
+  {   // forward GEMMs whose 128 x 128 tiles do not fill the SMs may split their reduction
     const long long K_ = (long long)d.P * d.B;
     const long long tiles = ((K_ + 127) / 128) * ((d.J + 127) / 128);
-    if (tiles * 2 <= p->num_sms && cudaMalloc(&p->part_ws, (size_t)4 * K_ * p->ldp * 4) != cudaSuccess) {
+    if (tiles < p->num_sms && cudaMalloc(&p->part_ws, (size_t)MAX_SPLITS * K_ * p->ldp * 4) != cudaSuccess) {
       cudaGetLastError();
       delete p;
       return SFB_ERR_ALLOC;
@@ -794,11 +796,36 @@ void umma_plan_destroy(UmmaPlan* p) {
 }
 
 // Tile shape and kernel variant for an M x N output (M counted in 128-row units).
-static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_chunk_aligned) {
+// max_splits > 1: the caller can take partial products, so a problem with few tiles may cut its reduction
+// (k_atoms 128-byte atoms long) into *splits ranges.  CTA pairs on 256 x 256 tiles need half the operand
+// traffic per flop of single 128 x 128 tiles, so they are preferred as soon as pairs x ranges fill the SMs.
+static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_chunk_aligned, int k_atoms = 0,
+                            int max_splits = 1, int* splits = nullptr) {
   Variant v;
+  if (splits != nullptr) *splits = 1;
   v.bn = (N > 128 && (long long)m_units * ((N + 255) / 256) >= pl->num_sms) ? 256 : 128;
   // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
   v.cg = (v.bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
+  if (max_splits > 1 && splits != nullptr && v.cg == 1) {
+    const int k_blocks = (k_atoms + pl->fold_ka - 1) / pl->fold_ka;
+    auto ranges = [&](long long tiles, int slots) {
+      long long ks = slots / (tiles > 0 ? tiles : 1);
+      if (ks > max_splits) ks = max_splits;
+      while (ks > 1 && k_blocks < 16 * ks) --ks;
+      return (int)(ks < 1 ? 1 : ks);
+    };
+    const long long t_pair = (long long)((m_units + 1) / 2) * ((N + 255) / 256);
+    const int ks_pair = ranges(t_pair, pl->num_sms / 2);
+    const long long t_one = (long long)m_units * ((N + 127) / 128);
+    const int ks_one = ranges(t_one, pl->num_sms);
+    if (pl->pair_ok && N > 128 && m_units >= 2 && 4 * t_pair * ks_pair >= 3 * (pl->num_sms / 2)) {
+      v.bn = 256; v.cg = 2;
+      *splits = ks_pair;
+    } else if (t_one < pl->num_sms) {
+      v.bn = 128; v.cg = 1;
+      *splits = ks_one;
+    }
+  }
   v.fold = v.cg == 2 && pl->fold_ok && dims_chunk_aligned;
   // two 128-byte atoms of reduction per stage wherever three such stages fit in shared memory: the
   // per-stage barrier round trip, not the number of TMA instructions, is what costs
@@ -820,22 +847,18 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   if (d.B >= BM) { p.m_bb = BM; p.m_wp = 1; p.m_tpw = (d.B + BM - 1) / BM; m_units = P * p.m_tpw; }
   else { p.m_bb = pow2_at_least(d.B); p.m_wp = BM / p.m_bb; p.m_tpw = 1; m_units = (P + p.m_wp - 1) / p.m_wp; }
   // folding walks the reduction index (D) in 128-byte atoms: rows must be whole atoms long
-  const Variant v = pick_variant(pl, m_units, d.J, (d.D % CH) == 0 && (a.ld % CH) == 0);
+  const bool may_split = k_splits_out != nullptr && stats == nullptr && max_splits > 1;
+  int ks_pick = 1;
+  const Variant v = pick_variant(pl, m_units, d.J, (d.D % CH) == 0 && (a.ld % CH) == 0, (d.D + CH - 1) / CH,
+                                 may_split ? (max_splits < MAX_SPLITS ? max_splits : MAX_SPLITS) : 1, &ks_pick);
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
   p.n_tiles = (d.J + v.bn - 1) / v.bn;
   p.k_blocks = (d.D + CH * v.ka - 1) / (CH * v.ka);
   // Few tiles and a long reduction (e.g. 1024 samples x 1000 classes over 20000 features): cut the
   // reduction so that every SM gets work; the partial products are summed, in a fixed order, by the
   // finishing pass.  Only when the caller provides the partial buffers (k_splits_out != nullptr).
-  p.k_splits = 1;
-  if (k_splits_out != nullptr && stats == nullptr) {
-    const int tiles = p.m_tiles * p.n_tiles;
-    int ks = pl->num_sms / (tiles > 0 ? tiles : 1);
-    if (ks > 4) ks = 4;
-    if (ks > max_splits) ks = max_splits;
-    if (ks >= 2 && p.k_blocks >= 32 * ks) p.k_splits = ks;
-    *k_splits_out = p.k_splits;
-  }
+  p.k_splits = may_split ? ks_pick : 1;
+  if (k_splits_out != nullptr) *k_splits_out = p.k_splits;
   p.k_per_split = (p.k_blocks + p.k_splits - 1) / p.k_splits;
   p.split_stride = split_stride;
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
@@ -883,7 +906,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
       const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
       int ks = 1;
       if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr, nullptr,
-                                 &ks, 4, sstride, workers)) < 0)
+                                 &ks, MAX_SPLITS, sstride, workers)) < 0)
         return r;
       launches += r;
       if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
@@ -919,7 +942,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, 4, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
