@@ -743,6 +743,11 @@ struct UmmaPlan {
   int fwd_group, apply_group;   // tile-order group widths (SFB_FWD_GROUP / SFB_APPLY_GROUP override the defaults)
   float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
   int ldp;
+  // MLR: the factor v is a copy of x that nothing in the factor stage reads, so it runs on a side stream
+  // next to the forward GEMM (fork / join by events; SFB_NO_SIDE_COPY=1 keeps it on the main stream)
+  cudaStream_t side;
+  cudaEvent_t fork, join;
+  bool side_ok;
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -775,6 +780,23 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
       return SFB_ERR_ALLOC;
     }
   }
+  p->side_ok = false;
+  {
+    const char* ns = getenv("SFB_NO_SIDE_COPY");
+    if (d.model == SFB_MLR && !(ns != nullptr && ns[0] == '1')) {
+      p->side_ok = cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking) == cudaSuccess;
+      if (p->side_ok) {
+        const bool e1 = cudaEventCreateWithFlags(&p->fork, cudaEventDisableTiming) == cudaSuccess;
+        const bool e2 = e1 && cudaEventCreateWithFlags(&p->join, cudaEventDisableTiming) == cudaSuccess;
+        if (!e2) {
+          if (e1) cudaEventDestroy(p->fork);
+          cudaStreamDestroy(p->side);
+          cudaGetLastError();
+          p->side_ok = false;
+        }
+      }
+    }
+  }
   p->stats = nullptr;
   if (d.model == SFB_MLR) {
     const size_t parts = 2 * (size_t)((d.J + 127) / 128);
@@ -790,6 +812,12 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
 }
 
 void umma_plan_destroy(UmmaPlan* p) {
+  if (p->side_ok) {
+    cudaStreamSynchronize(p->side);
+    cudaEventDestroy(p->fork);
+    cudaEventDestroy(p->join);
+    cudaStreamDestroy(p->side);
+  }
   if (p->stats) cudaFree(p->stats);
   if (p->part_ws) cudaFree(p->part_ws);
   delete p;
@@ -895,6 +923,20 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   x_rows.worker_stride = (long long)d.B * d.D * pl->es;
   if (d.model == SFB_MLR) {
     const bool bf16 = d.path == SFB_PATH_BF16;
+    bool forked = false;
+    if (v.base != nullptr && pl->side_ok) {   // v = x on the side stream, joined before this call returns its work
+      if (cudaEventRecord(pl->fork, s) != cudaSuccess || cudaStreamWaitEvent(pl->side, pl->fork, 0) != cudaSuccess)
+        return SFB_ERR_CUDA;
+      if ((r = launch_copy_rows(pl->side, x_rows, v, K, d.D)) < 0) return r;
+      launches += r;
+      if (cudaEventRecord(pl->join, pl->side) != cudaSuccess) return SFB_ERR_CUDA;
+      forked = true;
+    }
+    auto finish_v = [&]() -> int {
+      if (forked) return cudaStreamWaitEvent(s, pl->join, 0) == cudaSuccess ? 0 : SFB_ERR_CUDA;
+      if (v.base == nullptr) return 0;
+      return launch_copy_rows(s, x_rows, v, K, d.D);
+    };
     RowMap zz = bf16 ? z : u;   // fp32 products: workspace when u is bf16, else u itself (finished in place)
     // the GEMM epilogue leaves exp(z - local max) in u and (max, sum) per half tile; the finishing
     // pass rescales to the softmax and subtracts the one-hot label, in place
@@ -911,11 +953,8 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
       launches += r;
       if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
       launches += r;
-      if (v.base != nullptr) {
-        if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
-        launches += r;
-      }
-      return launches;
+      if ((r = finish_v()) < 0) return r;
+      return launches + r;
     }
     int n_parts = 0, part_cols = 0;
     (void)zz;
@@ -925,11 +964,8 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     launches += r;
     if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status)) < 0) return r;
     launches += r;
-    if (v.base != nullptr) {
-      if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
-      launches += r;
-    }
-    return launches;
+    if ((r = finish_v()) < 0) return r;
+    return launches + r;
   }
   // DML (TF32): the pair differences are the factor v and the GEMM operand
   if (v.base == nullptr) return SFB_ERR_ARG;
