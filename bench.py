@@ -279,7 +279,7 @@ def run_bsp(args, cfg, inputs, wl, path, rank, world, local_rank, barrier):
         ev[0].record(stream)
         wl.ctx.factors_shard(wl.W, s["X"], s["aux"], wl.sf_buf, bsp.first, bsp.n_workers)
         ev[1].record(stream)
-        if world > 1:
+        if bsp.in_group:
             all_gather_streams(wl.sf_buf, bsp.streams_off, bsp.stream_stride, cfg["P"])
         ev[2].record(stream)
         wl.ctx.commit_header(wl.sf_buf, t)
@@ -383,7 +383,8 @@ def main():
 
     build_library()
     torch.cuda.set_device(local_rank)
-    if world > 1:
+    in_group = world > 1 or (args.mode == "bsp" and "RANK" in os.environ)   # bsp under a launcher: NCCL even for one rank
+    if in_group:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
@@ -402,7 +403,7 @@ def main():
         if rank == 0:
             print(json.dumps(out), flush=True)
         wl.close()
-        if world > 1:
+        if in_group:
             dist.destroy_process_group()
         return
 

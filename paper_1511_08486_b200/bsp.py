@@ -41,8 +41,6 @@ def all_gather_streams(sf_buf: torch.Tensor, streams_off: int, stream_stride: in
     sf_buf: 1-D uint8 tensor holding the SF buffer (device memory with NCCL, host memory with gloo).
     """
     world = dist.get_world_size(group)
-    if world == 1:
-        return
     first, n = worker_range(P, world, dist.get_rank(group))
     streams = sf_buf[streams_off:streams_off + P * stream_stride]
     mine = streams[first * stream_stride:(first + n) * stream_stride]
@@ -58,7 +56,8 @@ class BspSfb:
         from . import binding as B
         self.ctx, self.desc, self.sf_buf, self.group = ctx, desc, sf_buf, group
         self.streams_off, self.stream_stride = B.sfb_sf_buffer_layout(desc)
-        if dist.is_available() and dist.is_initialized():
+        self.in_group = dist.is_available() and dist.is_initialized()
+        if self.in_group:
             self.world, self.rank = dist.get_world_size(group), dist.get_rank(group)
         else:
             self.world, self.rank = 1, 0
@@ -70,7 +69,7 @@ class BspSfb:
 
     def step(self, W, X_shard, aux_shard, eta: float, clock: int = 0) -> None:
         self.ctx.factors_shard(W, X_shard, aux_shard, self.sf_buf, self.first, self.n_workers)
-        if self.world > 1:
+        if self.in_group:       # also with a group of one process: the collective then has nothing to move
             all_gather_streams(self.sf_buf, self.streams_off, self.stream_stride, self.desc.P, self.group)
         self.ctx.commit_header(self.sf_buf, clock)
         self.ctx.apply(W, self.sf_buf, eta)

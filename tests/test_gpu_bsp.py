@@ -110,3 +110,24 @@ def test_shard_range_errors():
                 wl.ctx.factors_shard(wl.W, t["X"], t["aux"], wl.sf_buf, first, n)
     finally:
         wl.close()
+
+
+def test_bsp_bench_under_a_launcher_runs_the_nccl_exchange():
+    """One rank under torch.distributed.run: the in-place NCCL all-gather of the stream region really runs
+    (a group of one), and the bench line reports the job as one sharded job."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "1", "--master-addr",
+           "127.0.0.1", "--master-port", "29533", "bench.py", "--gpus", "1", "--mode", "bsp", "--config", "C1", "--path",
+           "tf32", "--J", "200", "--D", "1024", "--P", "4", "--B", "128", "--steps", "3", "--warmup", "3",
+           "--no-cpu-baseline"]
+    res = subprocess.run(cmd, cwd=root, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = [l for l in res.stdout.splitlines() if l.startswith("{")][-1]
+    out = json.loads(line)
+    assert out["scaling"] == "strong" and out["device_status"] == 0 and out["gpu_launches"] > 0
+    assert out["config"]["parallelism"].startswith("bsp sfb")
+    assert set(out["stages_ms"]) >= {"factors", "exchange", "apply"}
