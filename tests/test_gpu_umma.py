@@ -83,3 +83,11 @@ def test_tf32_c1_hundred_steps():
 def test_bf16_c4_reduced_fifty_steps():
     # C4's 50-step schedule at a reduced shape the oracle finishes in seconds (J = 4096, K = 512)
     check_config(_cfg("C4", "bf16", J=4096, D=8192, P=16, B=32), "bf16", eta=1e-3, steps=50)
+
+
+def test_pair_tiles_with_split_reduction_and_ragged_edges():
+    """Forward GEMMs small enough to take CTA pairs with several reduction ranges: an odd number of 128-row
+    units (the last pair is half empty), class counts that are no multiple of the tile, tf32 and bf16."""
+    check_config(_cfg("C1", "tf32", J=1000, D=8192, P=3, B=128, pool=1), "tf32", eta=0.5, steps=2)
+    check_config(_cfg("C2", "tf32", J=520, D=8192, P=5, B=100), "tf32", eta=1e-5, steps=1)
+    check_config(_cfg("C4", "bf16", J=1000, D=16384, P=3, B=128, pool=1, labels="uniform"), "bf16", eta=0.5, steps=2)
