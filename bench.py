@@ -137,7 +137,8 @@ def algorithmic(cfg, path, inputs=None):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one apply launch, from the ncu captures summarised
 # under profiles/ (captured at J = 8192 and scaled by J where the full launch is too large to capture).
-NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 4.03e9, ("C3", "f32"): 6.28e8}
+NCU_APPLY_TRAFFIC_BYTES = {("C4", "bf16"): 4.03e9, ("C3", "f32"): 6.28e8, ("C1", "tf32"): 2.03e8, ("C2", "tf32"): 1.21e8,
+                           ("C1", "f32"): 3.39e8, ("C2", "f32"): 1.95e8}
 
 
 def oracle_step_time(cfg, inputs, sample_workers: int):
@@ -515,8 +516,8 @@ def main():
                                                 "peak_source": "148 SMs x 128 B/clk x 1.965 GHz"}
             elif path == "f32":
                 out["roofline"] = {"bound": "alu", "achieved": apply_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
-                                   "frac": apply_tflops / FP32_FMA_TFLOPS, "traffic": None,
-                                   "kernel": "apply_f32_kernel", "peak_source": "148 SMs x 128 FMA lanes x 1.965 GHz"}
+                                   "frac": apply_tflops / FP32_FMA_TFLOPS, "traffic": traffic,
+                                   "kernel": "apply_f32_pipe_kernel", "peak_source": "148 SMs x 128 FMA lanes x 1.965 GHz"}
             else:
                 scale = 1.0 if path == "bf16" else 0.5          # tf32 nominal rate is half of bf16
                 peak = peaks["bf16_sustained"] * scale
