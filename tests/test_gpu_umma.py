@@ -91,3 +91,9 @@ def test_pair_tiles_with_split_reduction_and_ragged_edges():
     check_config(_cfg("C1", "tf32", J=1000, D=8192, P=3, B=128, pool=1), "tf32", eta=0.5, steps=2)
     check_config(_cfg("C2", "tf32", J=520, D=8192, P=5, B=100), "tf32", eta=1e-5, steps=1)
     check_config(_cfg("C4", "bf16", J=1000, D=16384, P=3, B=128, pool=1, labels="uniform"), "bf16", eta=0.5, steps=2)
+
+
+def test_tf32_large_mlr_fused_softmax_epilogue():
+    """A C4-shaped problem on the tf32 path: CTA pairs, folded loads and the fused exp / partial-sum epilogue
+    with fp32 factors (the bf16 path's kernels instantiated for 4-byte values)."""
+    check_config(_cfg("C4", "tf32", J=4096, D=4096, P=8, B=128, pool=1), "tf32", eta=1e-3, steps=2)
