@@ -352,6 +352,9 @@ def main():
     ap.add_argument("--config", default="C4")
     ap.add_argument("--path", default=None, help="f32 | tf32 | bf16 (default: the configuration's own)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="record sfb_step into one CUDA graph per pool minibatch and replay it (launch-bound small "
+                         "configurations; the header's clock is then the recorded one)")
     ap.add_argument("--mode", default="replicas", choices=["replicas", "bsp"],
                     help="N > 1: independent replicas of the whole path (default), or ONE job whose P workers are split "
                          "over the ranks with an all-gather of the worker streams per step (sufficient factor broadcasting)")
@@ -390,6 +393,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
     inputs = make_inputs(cfg)
+    if args.graph:            # capture needs a stream of its own; the context takes the current stream
+        torch.cuda.set_stream(torch.cuda.Stream(device=dev))
     wl = DeviceWorkload(cfg, inputs, path=path, device=dev)
     K, eta = cfg["K"], cfg["eta"]
     stream = torch.cuda.current_stream()
@@ -412,16 +417,35 @@ def main():
     step_bytes = 4.0 * cfg["J"] * cfg["D"] + wl.ctx.sf_buffer_bytes
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < (252 << 20) else None
 
+    graphs = []
+
+    def one_step(t):
+        if graphs:
+            graphs[t % wl.pool].replay()
+        else:
+            wl.step(t, eta=eta)
+
     def run_steps(n, t0=0):
         for t in range(n):
             if flush is not None:
                 flush.fill_(t & 1)
-            wl.step(t0 + t, eta=eta)
+            one_step(t0 + t)
 
     # ---- device-resident timing ----------------------------------------------------------------
     wl.reset()
     run_steps(max(args.warmup, 3))
     barrier()
+    if args.graph and args.mode == "replicas":
+        for b in range(wl.pool):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                wl.step(b, eta=eta)
+            graphs.append(g)
+        launches_per_step = wl.ctx.launch_count()
+        wl.step(0, eta=eta)
+        launches_per_step = wl.ctx.launch_count() - launches_per_step      # what one replay launches
+        run_steps(3)
+        barrier()
     l0 = wl.ctx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local_rank) as clocks:
@@ -436,13 +460,15 @@ def main():
             for t in range(args.steps):
                 flush.fill_(t & 1)
                 ev0.record(stream)
-                wl.step(args.warmup + t, eta=eta)
+                one_step(args.warmup + t)
                 ev1.record(stream)
                 torch.cuda.synchronize()
                 ms += ev0.elapsed_time(ev1)
             barrier()
-    launches = wl.ctx.launch_count() - l0
+    launches = wl.ctx.launch_count() - l0 if not graphs else launches_per_step * args.steps
     status = wl.ctx.status()
+    graphs_used = bool(graphs)
+    graphs.clear()            # stages and the end-to-end leg below run eagerly
 
     # ---- per-stage timing (events recorded inside sfb_step, same workload) ------------------------
     wl.ctx.profile(True)
@@ -492,7 +518,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": workload_name(cfg, path), "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "per-step footprint larger than L2" if flush is None else "L2 flushed between steps",
-                       "eta": eta, "pool": cfg["pool"]},
+                       "eta": eta, "pool": cfg["pool"], "cuda_graph": graphs_used},
             "e2e": {"value": whole_job_throughput(K, args.steps, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "last_clock_read_back": clock_of_last},
             "gpu_launches": int(launches),

@@ -28,6 +28,10 @@
  *   - A context is not thread-safe: calls on one context come from one host thread at a time.  Different
  *     contexts are independent (also on different devices of one process; a context belongs to the
  *     device that was current in sfb_create, which must be current again for every call on it).
+ *   - sfb_compute_factors, sfb_pack, sfb_apply, sfb_step, sfb_factors_shard and sfb_commit_header only enqueue
+ *     kernels (and event fork / join with a side stream of the context); after one ordinary call, which does
+ *     the one-time kernel attribute set-up, a call may be recorded into a CUDA graph by capturing the context's
+ *     stream and replayed (pointers and the clock are then the recorded ones).
  *   - "allocates only in sfb_create" has two stated exceptions, both on first use: the staging buffers
  *     of sfb_step_host and the workspace of sfb_loss.
  *   - W is J x D, row-major fp32, updated in place.  Samples are rows: X is [K][D].
