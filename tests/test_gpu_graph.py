@@ -49,3 +49,50 @@ def test_captured_step_replays_to_the_same_weights(name, path, over):
         finally:
             torch.cuda.synchronize()
             wl.close()
+
+
+@pytest.mark.parametrize("name,path,over", [CASES[1], CASES[2], CASES[4]])
+def test_captured_stage_calls_replay_to_the_same_weights(name, path, over):
+    """The separate entry points in one graph: factors + pack + apply, and shard factors + header + apply."""
+    from paper_1511_08486_b200.workload import DeviceWorkload
+    cfg = scaled(name, **over)
+    cfg["path"] = path
+    cfg["pool"] = 1
+    inputs = make_inputs(cfg)
+    eta = 1e-3
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        wl = DeviceWorkload(cfg, inputs, path=path, stream=side.cuda_stream)
+        try:
+            t = wl.batches[0]
+
+            def staged():
+                wl.compute_factors(0)
+                wl.pack(0, clock=0)
+                wl.apply(eta)
+
+            def sharded():
+                wl.ctx.factors_shard(wl.W, t["X"], t["aux"], wl.sf_buf, 0, cfg["P"])
+                wl.ctx.commit_header(wl.sf_buf, 0)
+                wl.ctx.apply(wl.W, wl.sf_buf, eta)
+
+            for fn in (staged, sharded):
+                wl.reset()
+                for _ in range(3):
+                    fn()
+                side.synchronize()
+                W_eager = wl.W.clone()
+                wl.reset()
+                fn()
+                side.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    fn()
+                graph.replay()
+                graph.replay()
+                torch.cuda.synchronize()
+                assert wl.ctx.status() == 0
+                assert torch.equal(wl.W, W_eager)
+        finally:
+            torch.cuda.synchronize()
+            wl.close()
