@@ -90,7 +90,8 @@ enum {
   SFB_DEV_BAD_INDEX = 2,    /* CSR column >= D or not strictly ascending: that entry is skipped */
   SFB_DEV_BAD_HEADER = 4,   /* SF buffer header does not match the descriptor: apply leaves W untouched */
   SFB_DEV_CAPACITY = 8,     /* a worker's nonzeros exceed cap_p: that stream's codes are truncated */
-  SFB_DEV_TIMEOUT = 16      /* a bounded device-side wait ran out */
+  SFB_DEV_TIMEOUT = 16      /* a bounded device-side wait (about a second) ran out: the launch completed, its
+                               output is not to be used; the context stays usable */
 };
 
 typedef struct sfb_desc {

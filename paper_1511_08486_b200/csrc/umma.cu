@@ -43,7 +43,7 @@ constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
 constexpr int RING_BYTES = 192 * 1024;   // shared memory given to the operand ring
 constexpr int MAX_STAGES = 8;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = 1u << 20;   // polls of a bounded wait: a failed poll suspends about 1.4 us, so about 1.4 s
 
 struct GemmParams {
   int m_tiles, n_tiles, k_blocks;   // m_tiles counts tiles of 128*CG rows; k_blocks counts blocks of BK reduction steps
@@ -65,6 +65,7 @@ struct GemmParams {
   int n_parts;
   const int* status_ro;
   int* status;
+  int lose_signal;          // test hook: the first pair / CTA drops its first "stage free" signal (see UmmaPlan)
 };
 
 struct SharedCtl {
@@ -357,8 +358,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
             }
           }
-          ptx::mma_commit<CG>(&ctl->empty[s]);                     // stage reusable once these MMAs have read it
-          if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->empty[s]), 1));
+          // (test hook: one lost signal, so that the producer's bounded wait runs out and the abort path is taken)
+          const bool lost = p.lose_signal != 0 && cluster_id == 0 && it == 0 && kb == kb_begin;
+          if (!lost) {
+            ptx::mma_commit<CG>(&ctl->empty[s]);                   // stage reusable once these MMAs have read it
+            if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->empty[s]), 1));
+          }
           if (kb == kb_end - 1) {                                  // accumulator complete, in both CTAs
             ptx::mma_commit<CG>(&ctl->tmem_full[buf]);
             if (CG == 2) ptx::mma_commit_addr<CG>(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_full[buf]), 1));
@@ -748,6 +753,9 @@ struct UmmaPlan {
   cudaStream_t side;
   cudaEvent_t fork, join;
   bool side_ok;
+  // SFB_TEST_LOSE_SIGNAL=1 at plan creation: the first GEMM launched through this plan loses one pipeline
+  // signal in its first CTA (pair), which must end in SFB_DEV_TIMEOUT after the bounded wait, not in a hang
+  int lose_signal;
 };
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
@@ -765,6 +773,8 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   p->fold_ok = !(no_fold != nullptr && no_fold[0] == '1');
   const char* ka = getenv("SFB_FOLD_KA");
   p->fold_ka = (ka != nullptr && ka[0] == '1') ? 1 : 2;
+  const char* ls = getenv("SFB_TEST_LOSE_SIGNAL");
+  p->lose_signal = (ls != nullptr && ls[0] == '1') ? 1 : 0;
   const char* fg = getenv("SFB_FWD_GROUP");
   const char* ag = getenv("SFB_APPLY_GROUP");
   p->fwd_group = fg != nullptr ? atoi(fg) : 8;
@@ -896,6 +906,8 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.group = pl->fwd_group;
   p.z = z;
   p.status = dev_status;
+  p.lose_signal = pl->lose_signal;
+  pl->lose_signal = 0;
   p.Nvalid = d.J;
   p.stats = stats;
   p.n_parts = 2 * p.n_tiles;
@@ -1018,6 +1030,8 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   p.eta = eta;
   p.status_ro = dev_status;
   p.status = const_cast<int*>(dev_status);
+  p.lose_signal = pl->lose_signal;
+  pl->lose_signal = 0;
   CUtensorMap tu, tv;
   // only the first `workers` streams are visible to the maps, so zero fill covers a ragged last block
   if (!encode_rows_map(&tu, es, u_rows.base, d.J, d.B, workers, (long long)u_rows.ld * es, u_rows.worker_stride, p.k_bb,
