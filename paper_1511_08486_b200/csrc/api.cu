@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/sfb.h: argument checks, workspace, kernel sequencing.
 // Every step of the path runs in the CUDA kernels of this library; there is no CPU fallback.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -20,6 +21,11 @@ struct sfb_ctx {
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
   void* csc_ws;             // SC, fp32 path: scratch of the atom-major re-sort of the codes (when K fits)
+  // sfb_step: work that does not depend on the factors (codes into the buffer, header, atom-major re-sort of
+  // the codes) runs on this stream beside the forward pass, forked and joined by events
+  cudaStream_t aux;
+  cudaEvent_t aux_fork, aux_join;
+  bool aux_ok;
   float* f32_part;          // fp32 dense path: partial products [splits][K][ldp] of a split forward reduction
   int ldp, f32_splits;
   float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
@@ -243,6 +249,19 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     c->f32_splits = ks;
     if (ks > 1) ok = cudaMalloc(&c->f32_part, (size_t)ks * c->K * c->ldp * 4) == cudaSuccess;
   }
+  if (ok) {
+    const char* na = getenv("SFB_NO_AUX_STREAM");
+    if (!(na != nullptr && na[0] == '1') && cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) == cudaSuccess) {
+      const bool e1 = cudaEventCreateWithFlags(&c->aux_fork, cudaEventDisableTiming) == cudaSuccess;
+      const bool e2 = e1 && cudaEventCreateWithFlags(&c->aux_join, cudaEventDisableTiming) == cudaSuccess;
+      c->aux_ok = e2;
+      if (!e2) {
+        if (e1) cudaEventDestroy(c->aux_fork);
+        cudaStreamDestroy(c->aux);
+        cudaGetLastError();
+      }
+    }
+  }
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -263,6 +282,12 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
 int sfb_destroy(sfb_ctx* c) {
   if (c == nullptr) return SFB_ERR_ARG;
   cudaStreamSynchronize(c->stream);
+  if (c->aux_ok) {
+    cudaStreamSynchronize(c->aux);
+    cudaEventDestroy(c->aux_fork);
+    cudaEventDestroy(c->aux_join);
+    cudaStreamDestroy(c->aux);
+  }
   if (c->umma) umma_plan_destroy(c->umma);
   if (c->prof_have_events)
     for (int i = 0; i < 128; ++i)
@@ -418,12 +443,15 @@ int sfb_pack(sfb_ctx* c, const void* U, const void* V, const sfb_aux* aux, void*
   return SFB_OK;
 }
 
-static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check) {
+// csc_built: the atom-major re-sort of this buffer's codes for these K samples is already in the workspace
+static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check, bool csc_built = false) {
   const sfb_desc& d = c->d;
   if (check) ACC(launch_check_header(c->stream, sf_buf, d, c->l, c->dev_status));
   if (d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
-    ACC(launch_sc_apply_csc(c->stream, reinterpret_cast<float*>(W), stream_codes(c, sf_buf), stream_u(c, sf_buf), K, d.J,
-                            d.D, eta, (long long)d.nnz_capacity, c->csc_ws, c->dev_status));
+    if (!csc_built)
+      ACC(launch_sc_csc_build(c->stream, stream_codes(c, sf_buf), K, d.D, (long long)d.nnz_capacity, c->csc_ws));
+    ACC(launch_sc_csc_apply(c->stream, reinterpret_cast<float*>(W), stream_u(c, sf_buf), K, d.J, d.D, eta,
+                            (long long)d.nnz_capacity, c->csc_ws, c->dev_status));
   } else if (d.v_sparse && d.path == SFB_PATH_F32) {
     ACC(launch_sc_apply(c->stream, reinterpret_cast<float*>(W), stream_codes(c, sf_buf), stream_u(c, sf_buf), K, d.J,
                         d.D, eta, c->dev_status, c->dev_status));
@@ -491,16 +519,33 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   memset(&codes, 0, sizeof(codes));
   const int slot = c->prof_n % 128;
   if (c->profiling) cudaEventRecord(c->prof_ev[slot][0], c->stream);
-  if (d.v_sparse) {
-    ACC(launch_pack_csr(c->stream, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
-                        c->dev_status));
-    codes = stream_codes(c, sf_buf);   // the forward reads the codes it just committed to the buffer
+  // What does not depend on the factors goes to the auxiliary stream, beside the forward pass: the codes into
+  // the buffer, header and directory, and the atom-major re-sort of the codes for the scatter apply.
+  bool forked = false;
+  if (c->aux_ok) {
+    if (cudaEventRecord(c->aux_fork, c->stream) != cudaSuccess || cudaStreamWaitEvent(c->aux, c->aux_fork, 0) != cudaSuccess)
+      return SFB_ERR_CUDA;
+    forked = true;
   }
+  cudaStream_t hs = forked ? c->aux : c->stream;
+  bool csc_built = false;
+  if (d.v_sparse) {
+    ACC(launch_pack_csr(hs, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
+                        c->dev_status));
+    // the forward reads the codes it just committed to the buffer, or, beside the packing, the caller's arrays
+    codes = forked ? global_codes(aux, d.B) : stream_codes(c, sf_buf);
+  }
+  ACC(launch_write_header(hs, sf_buf, d, c->l, clock, d.v_sparse ? aux->rowptr : nullptr));
+  if (forked && d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
+    ACC(launch_sc_csc_build(hs, stream_codes(c, sf_buf), K, d.D, (long long)d.nnz_capacity, c->csc_ws));
+    csc_built = true;
+  }
+  if (forked && cudaEventRecord(c->aux_join, c->aux) != cudaSuccess) return SFB_ERR_CUDA;
   r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes);
   if (r < 0) return r;
-  ACC(launch_write_header(c->stream, sf_buf, d, c->l, clock, d.v_sparse ? aux->rowptr : nullptr));
+  if (forked && cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess) return SFB_ERR_CUDA;
   if (c->profiling) cudaEventRecord(c->prof_ev[slot][1], c->stream);
-  r = apply_from(c, W, sf_buf, eta, K, false);
+  r = apply_from(c, W, sf_buf, eta, K, false, csc_built);
   if (c->profiling) {
     cudaEventRecord(c->prof_ev[slot][2], c->stream);
     c->prof_n++;

@@ -134,6 +134,11 @@ long long sc_csc_workspace_bytes(int K, int D, long long nnz_capacity);
 bool sc_csc_supported(int K);
 int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                         long long nnz_capacity, void* workspace, const int* dev_status_ro);
+// The two halves of launch_sc_apply_csc: the re-sort reads only the codes (it can run beside the forward
+// pass), the update needs u and the workspace the re-sort filled.
+int launch_sc_csc_build(cudaStream_t s, CsrView codes, int K, int D, long long nnz_capacity, void* workspace);
+int launch_sc_csc_apply(cudaStream_t s, float* W, RowMap u, int K, int J, int D, float eta, long long nnz_capacity,
+                        void* workspace, const int* dev_status_ro);
 
 // Dense fp32 rows a_i of the CSR codes (zeros elsewhere), for the tensor-core sparse-coding path.
 int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status);

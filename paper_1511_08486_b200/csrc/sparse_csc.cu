@@ -251,25 +251,44 @@ long long sc_csc_workspace_bytes(int K, int D, long long nnz_capacity) {
 // The sliced kernel takes any K (more slices); the bound only keeps the chunk tables small.
 bool sc_csc_supported(int K) { return K <= (1 << 14); }
 
-int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
-                        long long nnz_capacity, void* workspace, const int* dev_status_ro) {
+namespace {
+struct CscScratch {
+  int* cnt; int* total; int* colptr; int* ent_i; float* ent_a;
+};
+CscScratch csc_scratch(void* workspace, int K, int D, long long nnz_capacity) {
   const int nchunks = (K + CSC_CHUNK - 1) / CSC_CHUNK;
-  int* cnt = reinterpret_cast<int*>(workspace);
-  int* total = cnt + (size_t)nchunks * D;
-  int* colptr = total + D;
+  CscScratch w;
+  w.cnt = reinterpret_cast<int*>(workspace);
+  w.total = w.cnt + (size_t)nchunks * D;
+  w.colptr = w.total + D;
   char* ent_base = reinterpret_cast<char*>(workspace) + pad_to(((long long)nchunks * D + D + D + 1) * 4, 256);
-  int* ent_i = reinterpret_cast<int*>(ent_base);
-  float* ent_a = reinterpret_cast<float*>(ent_base + pad_to(nnz_capacity * 4, 256));
-  if (cudaMemsetAsync(cnt, 0, (size_t)nchunks * D * 4, s) != cudaSuccess) return SFB_ERR_CUDA;
-  csc_count_kernel<<<K, 256, 0, s>>>(codes, K, D, cnt);
-  csc_chunk_offsets_kernel<<<(D + 255) / 256, 256, 0, s>>>(nchunks, D, cnt, total);
-  csc_scan_kernel<<<1, 1024, 0, s>>>(D, total, colptr);
-  csc_fill_kernel<<<nchunks, 256, 0, s>>>(codes, K, D, cnt, colptr, ent_i, ent_a);
+  w.ent_i = reinterpret_cast<int*>(ent_base);
+  w.ent_a = reinterpret_cast<float*>(ent_base + pad_to(nnz_capacity * 4, 256));
+  return w;
+}
+}  // namespace
+
+// Atom-major re-sort of the codes into the workspace.  Reads the codes only (not u), so it may run beside
+// the forward pass that produces u.
+int launch_sc_csc_build(cudaStream_t s, CsrView codes, int K, int D, long long nnz_capacity, void* workspace) {
+  const int nchunks = (K + CSC_CHUNK - 1) / CSC_CHUNK;
+  const CscScratch w = csc_scratch(workspace, K, D, nnz_capacity);
+  if (cudaMemsetAsync(w.cnt, 0, (size_t)nchunks * D * 4, s) != cudaSuccess) return SFB_ERR_CUDA;
+  csc_count_kernel<<<K, 256, 0, s>>>(codes, K, D, w.cnt);
+  csc_chunk_offsets_kernel<<<(D + 255) / 256, 256, 0, s>>>(nchunks, D, w.cnt, w.total);
+  csc_scan_kernel<<<1, 1024, 0, s>>>(D, w.total, w.colptr);
+  csc_fill_kernel<<<nchunks, 256, 0, s>>>(codes, K, D, w.cnt, w.colptr, w.ent_i, w.ent_a);
+  return cudaGetLastError() == cudaSuccess ? 4 : SFB_ERR_CUDA;
+}
+
+// The update from a workspace that launch_sc_csc_build filled for the same K, D and codes.
+int launch_sc_csc_apply(cudaStream_t s, float* W, RowMap u, int K, int J, int D, float eta, long long nnz_capacity,
+                        void* workspace, const int* dev_status_ro) {
+  const CscScratch w = csc_scratch(workspace, K, D, nnz_capacity);
   const int threads = 512;
   static PerDeviceOnce attr_once;   // function attributes are per device
-  if (attr_once.first()) {
+  if (attr_once.first())
     cudaFuncSetAttribute(csc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-  }
   // slices of the samples: the fewest that let Kh x 256 bytes of u sit beside the warps' tiles
   const long long tiles = (long long)(threads / 32) * CSC2_WARP_FLOATS * 4;
   const int kh_max = (int)((220 * 1024 - tiles) / 256) / CSC_CHUNK * CSC_CHUNK;
@@ -281,9 +300,17 @@ int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K
   if (splits > nblocks / (threads / 32)) splits = nblocks / (threads / 32);
   if (splits < 1) splits = 1;
   const size_t smem = (size_t)Kh * 256 + (size_t)tiles;
-  csc_apply_kernel<<<dim3(nj, splits), threads, smem, s>>>(W, u, K, J, D, eta, colptr, cnt, ent_i, ent_a, passes, Kh,
-                                                           dev_status_ro);
-  return cudaGetLastError() == cudaSuccess ? 5 : SFB_ERR_CUDA;
+  csc_apply_kernel<<<dim3(nj, splits), threads, smem, s>>>(W, u, K, J, D, eta, w.colptr, w.cnt, w.ent_i, w.ent_a, passes,
+                                                          Kh, dev_status_ro);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
+                        long long nnz_capacity, void* workspace, const int* dev_status_ro) {
+  const int a = launch_sc_csc_build(s, codes, K, D, nnz_capacity, workspace);
+  if (a < 0) return a;
+  const int b2 = launch_sc_csc_apply(s, W, u, K, J, D, eta, nnz_capacity, workspace, dev_status_ro);
+  return b2 < 0 ? b2 : a + b2;
 }
 
 }  // namespace sfb
