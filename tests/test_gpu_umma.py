@@ -97,3 +97,10 @@ def test_tf32_large_mlr_fused_softmax_epilogue():
     """A C4-shaped problem on the tf32 path: CTA pairs, folded loads and the fused exp / partial-sum epilogue
     with fp32 factors (the bf16 path's kernels instantiated for 4-byte values)."""
     check_config(_cfg("C4", "tf32", J=4096, D=4096, P=8, B=128, pool=1), "tf32", eta=1e-3, steps=2)
+
+
+def test_many_workers_and_long_reductions():
+    """K far beyond the benchmark shapes: 256 workers x 256 pairs on the bf16 path (65536 rank-one terms per
+    update), and 256 workers x 64 pairs on the tf32 path (reduction blocks that span two workers)."""
+    check_config(_cfg("C4", "bf16", J=256, D=256, P=256, B=256, pool=1, labels="uniform"), "bf16", eta=1e-3, steps=1)
+    check_config(_cfg("C2", "tf32", J=128, D=256, P=256, B=64), "tf32", eta=1e-6, steps=1)
