@@ -184,6 +184,13 @@ def test_c3_sc_many_samples_f32():
     check_config(scaled("C3", J=72, D=200, P=4, B=400, density=0.03), "f32", eta=1e-3, steps=1)
 
 
+def test_many_workers_f32():
+    """K far beyond the benchmark shapes on the CUDA-core paths: 16384 samples (MLR), 4096 coded samples
+    (seven shared-memory slices of the scatter apply)."""
+    check_config(scaled("C1", J=100, D=260, P=64, B=256), "f32", eta=1e-3, steps=1)
+    check_config(scaled("C3", J=64, D=256, P=64, B=64, density=0.05), "f32", eta=1e-4, steps=1)
+
+
 def test_c3_sc_full_f32():
     check_config(get_config("C3"), "f32", eta=1e-4, steps=1)
 
