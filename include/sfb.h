@@ -173,7 +173,7 @@ int sfb_step_host(sfb_ctx* ctx, void* W, const void* X_host, const sfb_aux* aux_
  *      sfb_compute_factors with P = n_workers; SFB_SC row pointers start at 0).  Other streams untouched.
  *   2. the exchange (the caller's: the worker streams are contiguous and equally long, so an all-gather
  *      over bytes [streams_off, streams_off + P * stream_stride) of the buffer, each process contributing
- *      the streams it owns, in place, is the whole broadcast; header words 40..47 and 56..63 hold
+ *      the streams it owns, in place, is the whole broadcast; header bytes 40..47 and 56..63 hold
  *      stream_stride and streams_off, see sfb_sf_buffer_layout).
  *   3. sfb_commit_header (header and directory, identical on every process; the SFB_SC directory takes each
  *      worker's nonzero count from the stream it received) and sfb_apply with K = P * B.
