@@ -844,7 +844,7 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
   v.bn = (N > 128 && (long long)m_units * ((N + 255) / 256) >= pl->num_sms) ? 256 : 128;
   // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
   v.cg = (v.bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
-  if (max_splits > 1 && splits != nullptr && v.cg == 1) {
+  if (v.cg == 1 && k_atoms > 0) {
     const int k_blocks = (k_atoms + pl->fold_ka - 1) / pl->fold_ka;
     auto ranges = [&](long long tiles, int slots) {
       long long ks = slots / (tiles > 0 ? tiles : 1);
@@ -856,10 +856,12 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
     const int ks_pair = ranges(t_pair, pl->num_sms / 2);
     const long long t_one = (long long)m_units * ((N + 127) / 128);
     const int ks_one = ranges(t_one, pl->num_sms);
+    // pairs that fill three quarters of the machine beat single tiles that fill all of it: the single
+    // 128 x 128 tiles are bound by the operand feed (about 50 % tensor-pipe activity with fp32 operands)
     if (pl->pair_ok && N > 128 && m_units >= 2 && 4 * t_pair * ks_pair >= 3 * (pl->num_sms / 2)) {
       v.bn = 256; v.cg = 2;
-      *splits = ks_pair;
-    } else if (t_one < pl->num_sms) {
+      if (splits != nullptr) *splits = ks_pair;
+    } else if (t_one < pl->num_sms && splits != nullptr && max_splits > 1) {
       v.bn = 128; v.cg = 1;
       *splits = ks_one;
     }
