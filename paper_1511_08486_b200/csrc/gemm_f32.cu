@@ -26,9 +26,12 @@ __device__ __forceinline__ float4 ld4_guard(const float* row, int c, int cols, b
   return r;
 }
 
-template <int MI, int NI>
+// PACKED: the multiply-adds as packed fp32 pairs (two independent round-to-nearest FMAs per instruction: half
+// the issue slots of scalar FFMA for the same arithmetic, bit-identical results).  It pays in the apply kernels;
+// the forward kernel, which also holds its operand prefetch in registers, measured slower with it.
+template <int MI, int NI, bool PACKED>
 __device__ __forceinline__ void mma_tile(const float (*As)[64 * MI + 4], const float (*Bs)[64 * NI + 4], int ty,
-                                         int tx, float (&acc)[4 * MI][4 * NI]) {
+                                         int tx, float2 (&acc)[4 * MI][2 * NI]) {
 #pragma unroll
   for (int k = 0; k < BK; ++k) {
     float a[4 * MI], b[4 * NI];
@@ -43,9 +46,18 @@ __device__ __forceinline__ void mma_tile(const float (*As)[64 * MI + 4], const f
       b[ni * 4 + 0] = t.x; b[ni * 4 + 1] = t.y; b[ni * 4 + 2] = t.z; b[ni * 4 + 3] = t.w;
     }
 #pragma unroll
-    for (int m = 0; m < 4 * MI; ++m)
+    for (int m = 0; m < 4 * MI; ++m) {
+      const float2 aa = make_float2(a[m], a[m]);
 #pragma unroll
-      for (int n = 0; n < 4 * NI; ++n) acc[m][n] = fmaf(a[m], b[n], acc[m][n]);
+      for (int n = 0; n < 2 * NI; ++n) {
+        if (PACKED) {
+          acc[m][n] = __ffma2_rn(aa, make_float2(b[2 * n], b[2 * n + 1]), acc[m][n]);
+        } else {
+          acc[m][n].x = fmaf(a[m], b[2 * n], acc[m][n].x);
+          acc[m][n].y = fmaf(a[m], b[2 * n + 1], acc[m][n].y);
+        }
+      }
+    }
   }
 }
 
@@ -65,11 +77,11 @@ __global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __rest
   const bool write_v = (v.base != nullptr) && (blockIdx.x == 0);
   const int lr = tid >> 2, lc = (tid & 3) * 4;   // loader: row within 64, first of 4 reduction columns
 
-  float acc[4 * MI][4 * NI];
+  float2 acc[4 * MI][2 * NI];
 #pragma unroll
   for (int m = 0; m < 4 * MI; ++m)
 #pragma unroll
-    for (int n = 0; n < 4 * NI; ++n) acc[m][n] = 0.f;
+    for (int n = 0; n < 2 * NI; ++n) acc[m][n] = make_float2(0.f, 0.f);
 
   float4 pa[MI], pb[NI];
   auto fetch = [&](int d0) {
@@ -115,7 +127,7 @@ __global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __rest
     stash();
     __syncthreads();
     if (d0 + BK < d_hi) fetch(d0 + BK);
-    mma_tile<MI, NI>(As, Bs, ty, tx, acc);
+    mma_tile<MI, NI, false>(As, Bs, ty, tx, acc);
     __syncthreads();
   }
   // The factor v has pad columns [D, ldv): the last loader step wrote zeros there only when
@@ -132,8 +144,8 @@ __global__ void __launch_bounds__(256, 2) forward_f32_kernel(const float* __rest
       for (int ni = 0; ni < NI; ++ni) {
         const int j = j0 + ni * 64 + tx * 4;
         if (j < z.ld)   // ld is a multiple of 4, so the whole float4 is inside the row; columns >= J hold 0
-          *reinterpret_cast<float4*>(zr + j) = make_float4(acc[mi * 4 + a][ni * 4 + 0], acc[mi * 4 + a][ni * 4 + 1],
-                                                           acc[mi * 4 + a][ni * 4 + 2], acc[mi * 4 + a][ni * 4 + 3]);
+          *reinterpret_cast<float4*>(zr + j) = make_float4(acc[mi * 4 + a][ni * 2].x, acc[mi * 4 + a][ni * 2].y,
+                                                           acc[mi * 4 + a][ni * 2 + 1].x, acc[mi * 4 + a][ni * 2 + 1].y);
       }
     }
 }
@@ -152,11 +164,11 @@ __global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W
   const int j0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
   const int lr = tid >> 4, lc = (tid & 15) * 4;   // loader: factor row within 16, first of 4 columns
 
-  float acc[4 * MI][4 * NI];
+  float2 acc[4 * MI][2 * NI];
 #pragma unroll
   for (int m = 0; m < 4 * MI; ++m)
 #pragma unroll
-    for (int n = 0; n < 4 * NI; ++n) acc[m][n] = 0.f;
+    for (int n = 0; n < 2 * NI; ++n) acc[m][n] = make_float2(0.f, 0.f);
 
   float4 pa[MI], pb[NI];
   auto fetch = [&](int k0) {
@@ -186,7 +198,7 @@ __global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W
     stash();
     __syncthreads();
     if (k0 + BK < K) fetch(k0 + BK);
-    mma_tile<MI, NI>(As, Bs, ty, tx, acc);
+    mma_tile<MI, NI, true>(As, Bs, ty, tx, acc);
     __syncthreads();
   }
 
@@ -201,7 +213,8 @@ __global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W
 #pragma unroll
       for (int ni = 0; ni < NI; ++ni) {
         const int d = d0 + ni * 64 + tx * 4;
-        const float* c = acc[mi * 4 + a] + ni * 4;
+        const float c[4] = {acc[mi * 4 + a][ni * 2].x, acc[mi * 4 + a][ni * 2].y, acc[mi * 4 + a][ni * 2 + 1].x,
+                            acc[mi * 4 + a][ni * 2 + 1].y};
         if (vec_ok && d + 3 < D) {
           float4 w = *reinterpret_cast<float4*>(wr + d);
           w.x = fmaf(-eta, c[0], w.x); w.y = fmaf(-eta, c[1], w.y);
@@ -257,11 +270,11 @@ __global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restric
     }
   };
 
-  float acc[8][8];
+  float2 acc[8][4];
 #pragma unroll
   for (int m = 0; m < 8; ++m)
 #pragma unroll
-    for (int n = 0; n < 8; ++n) acc[m][n] = 0.f;
+    for (int n = 0; n < 4; ++n) acc[m][n] = make_float2(0.f, 0.f);
 
   const int nk = (K + BK - 1) / BK;
 #pragma unroll
@@ -276,7 +289,7 @@ __global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restric
     if (nxt < nk) issue(nxt % PIPE, nxt * BK);
     cp_async_commit();
     const float* As = ring + (kt % PIPE) * PIPE_STAGE_FLOATS;
-    mma_tile<2, 2>(reinterpret_cast<const float(*)[BM + 4]>(As), reinterpret_cast<const float(*)[BN + 4]>(As + BK * (BM + 4)),
+    mma_tile<2, 2, true>(reinterpret_cast<const float(*)[BM + 4]>(As), reinterpret_cast<const float(*)[BN + 4]>(As + BK * (BM + 4)),
                    ty, tx, acc);
   }
   cp_async_wait<0>();
@@ -292,7 +305,8 @@ __global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restric
 #pragma unroll
       for (int ni = 0; ni < 2; ++ni) {
         const int d = d0 + ni * 64 + tx * 4;
-        const float* c = acc[mi * 4 + a] + ni * 4;
+        const float c[4] = {acc[mi * 4 + a][ni * 2].x, acc[mi * 4 + a][ni * 2].y, acc[mi * 4 + a][ni * 2 + 1].x,
+                            acc[mi * 4 + a][ni * 2 + 1].y};
         if (vec_ok && d + 3 < D) {
           float4 w = *reinterpret_cast<float4*>(wr + d);
           w.x = fmaf(-eta, c[0], w.x); w.y = fmaf(-eta, c[1], w.y);
