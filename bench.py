@@ -33,6 +33,7 @@ if ROOT not in sys.path:
 METRIC = "SF-step samples/s"
 UNIT = "samples/s"
 SMEM_TBS = 148 * 128 * 1.965e9 / 1e12           # shared-memory load path of the whole chip
+L2_TBS = 148 * 64 * 1.965e9 / 1e12              # L2 -> SM read path of the whole chip
 DATASHEET_BF16_TFLOPS = 2250.0
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 lanes x 2 flop x max SM clock
 
@@ -554,6 +555,21 @@ def main():
                                    "frac_of_datasheet": apply_tflops / (DATASHEET_BF16_TFLOPS * scale)}
             out["apply_tflops"] = apply_tflops
             out["forward_tflops"] = fwd_tflops
+            # the factor stage (forward contraction + finishing passes) against the bound of its contraction
+            if alg["sparse"]:
+                l2_tbs = 2.0 * alg["flops"] / (f_ms * 1e-3) / 1e12     # every multiply-add gathers 4 bytes of W from L2
+                out["roofline_factors"] = {"bound": "l2", "achieved": l2_tbs, "peak": L2_TBS, "unit": "TB/s",
+                                           "frac": l2_tbs / L2_TBS, "kernel": "sc_forward_kernel",
+                                           "peak_source": "148 SMs x 64 B/clk x 1.965 GHz"}
+            elif path == "f32":
+                out["roofline_factors"] = {"bound": "alu", "achieved": fwd_tflops, "peak": FP32_FMA_TFLOPS,
+                                           "unit": "TFLOP/s", "frac": fwd_tflops / FP32_FMA_TFLOPS,
+                                           "kernel": "forward_f32_kernel + finishing pass"}
+            else:
+                scale = 1.0 if path == "bf16" else 0.5
+                out["roofline_factors"] = {"bound": "tensor", "achieved": fwd_tflops, "peak": peaks["bf16_sustained"] * scale,
+                                           "unit": "TFLOP/s", "frac": fwd_tflops / (peaks["bf16_sustained"] * scale),
+                                           "kernel": "umma_gemm_kernel (forward) + finishing pass"}
         if not args.no_cpu_baseline:
             sw = pick_sample_workers(cfg, budget=6e12)
             dt, n = oracle_step_time(cfg, inputs, sw)
