@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 METRIC = "SF-step samples/s"
 UNIT = "samples/s"
 SMEM_TBS = 148 * 128 * 1.965e9 / 1e12           # shared-memory load path of the whole chip
-L2_TBS = 148 * 64 * 1.965e9 / 1e12              # L2 -> SM read path of the whole chip
+L2_TBS = 24.5                                   # L2 read rate at which ncu reports lts__throughput = 100 % (17.9 TB/s at 73 %)
 DATASHEET_BF16_TFLOPS = 2250.0
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 lanes x 2 flop x max SM clock
 
@@ -560,7 +560,7 @@ def main():
                 l2_tbs = 2.0 * alg["flops"] / (f_ms * 1e-3) / 1e12     # every multiply-add gathers 4 bytes of W from L2
                 out["roofline_factors"] = {"bound": "l2", "achieved": l2_tbs, "peak": L2_TBS, "unit": "TB/s",
                                            "frac": l2_tbs / L2_TBS, "kernel": "sc_forward_kernel",
-                                           "peak_source": "148 SMs x 64 B/clk x 1.965 GHz"}
+                                           "peak_source": "ncu: 17.9 TB/s of L2 reads at lts__throughput 73 %"}
             elif path == "f32":
                 out["roofline_factors"] = {"bound": "alu", "achieved": fwd_tflops, "peak": FP32_FMA_TFLOPS,
                                            "unit": "TFLOP/s", "frac": fwd_tflops / FP32_FMA_TFLOPS,

@@ -90,11 +90,18 @@ __global__ void __launch_bounds__(256) sc_forward_kernel(const float* __restrict
     __syncthreads();
     const int n = min(256, row.len - k0);
     if (j < ldt) {
-      for (int e = 0; e < n; ++e) {
-        const float4 w = *reinterpret_cast<const float4*>(Wt + (size_t)s_idx[e] * ldt + j);
-        const float av = s_val[e];
-        acc.x = fmaf(av, w.x, acc.x); acc.y = fmaf(av, w.y, acc.y);
-        acc.z = fmaf(av, w.z, acc.z); acc.w = fmaf(av, w.w, acc.w);
+      // eight gathers in flight per thread before their multiply-adds (entries beyond n hold value 0, atom 0);
+      // the order of the additions stays the order of the entries
+      for (int e0 = 0; e0 < n; e0 += 8) {
+        float4 w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float4*>(Wt + (size_t)s_idx[e0 + q] * ldt + j);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const float av = s_val[e0 + q];
+          acc.x = fmaf(av, w[q].x, acc.x); acc.y = fmaf(av, w[q].y, acc.y);
+          acc.z = fmaf(av, w[q].z, acc.z); acc.w = fmaf(av, w[q].w, acc.w);
+        }
       }
     }
   }
