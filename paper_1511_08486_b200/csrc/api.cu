@@ -28,6 +28,7 @@ struct sfb_ctx {
   bool aux_ok;
   float* f32_part;          // fp32 dense path: partial products [splits][K][ldp] of a split forward reduction
   int ldp, f32_splits;
+  float* f32_nn_ws;         // fp32 dense path: transposed copies of the forward's operands (large shapes only)
   float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
   float* loss_i;            // sfb_loss: per-sample objective [K]
   // sfb_step_host: two sets of device staging buffers for the step's host inputs (allocated on first
@@ -162,8 +163,19 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     const RowMap part = caller_rows(c->f32_part, c->ldp, d.B, 4);
     const long long sstride = (long long)c->K * c->ldp * 4;
     int ks = 1;
-    ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, K, d.J, d.D, u, v, part, sstride,
-                           c->f32_splits, &ks));
+    if (c->f32_nn_ws != nullptr && (Xb == nullptr || v.base != nullptr)) {
+      RowMap src = caller_rows(X, d.D, d.B, 4), copy = v;
+      if (Xb != nullptr) {   // pair differences first (they are the factor v), then contracted from there
+        ACC(launch_diff_rows(c->stream, reinterpret_cast<const float*>(X), Xb, v, K, d.D));
+        src = v;
+        copy = RowMap();
+      }
+      ACC(launch_forward_f32_nn(c->stream, Wf, src, copy, K, d.J, d.D, c->f32_nn_ws, u, part, sstride, c->f32_splits,
+                                &ks));
+    } else {
+      ACC(launch_forward_f32(c->stream, Wf, reinterpret_cast<const float*>(X), Xb, K, d.J, d.D, u, v, part, sstride,
+                             c->f32_splits, &ks));
+    }
     const RowMap zsrc = ks > 1 ? part : u;
     if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, zsrc, u, aux->labels, K, d.J, c->dev_status, ks, sstride));
     else ACC(launch_finish_dml(c->stream, zsrc, u, aux->similar, d.margin, K, d.J, ks, sstride));
@@ -248,6 +260,10 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     c->ldp = (desc->J + 3) & ~3;
     c->f32_splits = ks;
     if (ks > 1) ok = cudaMalloc(&c->f32_part, (size_t)ks * c->K * c->ldp * 4) == cudaSuccess;
+    // shapes with at least a tile of work per dimension take the forward through transposed operand copies
+    const long long nn_floats = forward_f32_nn_workspace_floats(c->K, desc->J, desc->D);
+    if (ok && c->K >= 128 && desc->J >= 64 && desc->D >= 512 && nn_floats * 4 <= (2LL << 30))
+      ok = cudaMalloc(&c->f32_nn_ws, (size_t)nn_floats * 4) == cudaSuccess;
   }
   if (ok) {
     const char* na = getenv("SFB_NO_AUX_STREAM");
@@ -298,6 +314,7 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->a_dense) cudaFree(c->a_dense);
   if (c->csc_ws) cudaFree(c->csc_ws);
   if (c->f32_part) cudaFree(c->f32_part);
+  if (c->f32_nn_ws) cudaFree(c->f32_nn_ws);
   if (c->loss_rows) cudaFree(c->loss_rows);
   if (c->loss_i) cudaFree(c->loss_i);
   for (int k = 0; k < 2; ++k)

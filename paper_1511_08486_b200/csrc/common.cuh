@@ -77,7 +77,15 @@ struct PerDeviceOnce {
 // With a `part` row map (fp32 rows, split_stride bytes between partial buffers) and nsplit_out, a problem
 // with few tiles has its reduction cut into *nsplit_out ranges whose partial products go to `part` instead
 // of `z` (the finishing pass sums them in range order); forward_f32_splits tells how many in advance.
+// v rows = Xa rows - Xb rows, one fp32 subtraction per element, pad columns zero (the DML factor v).
+int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D);
 int forward_f32_splits(int K, int J, int D);
+// The same contraction through transposed copies of both operands (two transposing passes, then the pipelined
+// large-tile kernel).  src: operand rows a_i behind a row map; copy (optional): those rows also written there;
+// ws: forward_f32_nn_workspace_floats(K, J, D) floats.  Needs at least one full 128 x 128 tile of work to pay.
+long long forward_f32_nn_workspace_floats(int K, int J, int D);
+int launch_forward_f32_nn(cudaStream_t s, const float* W, RowMap src, RowMap copy, int K, int J, int D, float* ws,
+                          RowMap z, RowMap part, long long split_stride, int max_splits, int* nsplit_out);
 int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
                        RowMap z, RowMap v, RowMap part = RowMap(), long long split_stride = 0, int max_splits = 1,
                        int* nsplit_out = nullptr);

@@ -229,9 +229,12 @@ __global__ void __launch_bounds__(256, 2) apply_f32_kernel(float* __restrict__ W
     }
 }
 
-// ---- apply, large tiles: the factor rows go to shared memory as they are, so they are fetched with
-// 16-byte asynchronous copies (zero-filled beyond K, J and D) through a ring of PIPE stages: one barrier
-// per reduction step, no staging registers.
+// ---- large tiles with operands whose rows run along the OUTPUT indices: C[m][n] (+)= sum_k A[k][m] * B[k][n].
+// The rows go to shared memory as they are, fetched with 16-byte asynchronous copies (zero-filled beyond the
+// reduction range, M and N) through a ring of PIPE stages: one barrier per reduction step, no staging registers.
+//   OUT 0 (apply):   A = factor rows u_i (k = sample, m = row j of W), B = v_i; W[m][n] -= eta * C[m][n].
+//   OUT 1 (forward): A = X^T (k = feature d, m = sample i), B = W^T (n = class j), both made by a transposing
+//                    pass; the products of reduction range blockIdx.z are stored to z rows (+ range stride).
 constexpr int PIPE = 4;
 constexpr int PIPE_STAGE_FLOATS = 2 * BK * (128 + 4);
 
@@ -243,13 +246,17 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-__global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
-                                                             int D, float eta, const int* __restrict__ dev_status) {
+template <int OUT>
+__global__ void __launch_bounds__(256, 2) sgemm_pipe_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
+                                                         int D, float eta, const int* __restrict__ dev_status,
+                                                         RowMap z, int k_per_range, long long range_stride) {
   constexpr int BM = 128, BN = 128;
   extern __shared__ __align__(16) float ring[];
-  if (dev_status != nullptr && (*dev_status & SFB_DEV_BAD_HEADER)) return;
+  if (OUT == 0 && dev_status != nullptr && (*dev_status & SFB_DEV_BAD_HEADER)) return;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const int j0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
+  const int k_lo = (OUT == 1) ? blockIdx.z * k_per_range : 0;
+  const int k_hi = (OUT == 1) ? min(K, k_lo + k_per_range) : K;
   const int lr = tid >> 5, lc = (tid & 31) * 4;   // loader: factor rows lr and lr + 8 of the step, 4 columns at lc
   // bytes of this thread's 16-byte piece that exist (the rest is zero-filled); a piece with nothing to read
   // still needs a valid aligned address: column 0 of a valid row
@@ -263,7 +270,7 @@ __global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restric
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int r = lr + 8 * h, i = k0 + r;
-      const bool ok = i < K;
+      const bool ok = i < k_hi;
       const int ii = ok ? i : 0;
       cp_async16_zfill(As + r * (BM + 4) + lc, u.row(ii) + u_off, ok ? u_bytes : 0);
       cp_async16_zfill(Bs + r * (BN + 4) + lc, v.row(ii) + v_off, ok ? v_bytes : 0);
@@ -276,23 +283,42 @@ __global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restric
 #pragma unroll
     for (int n = 0; n < 4; ++n) acc[m][n] = make_float2(0.f, 0.f);
 
-  const int nk = (K + BK - 1) / BK;
+  const int nk = (k_hi - k_lo + BK - 1) / BK;
 #pragma unroll
   for (int st = 0; st < PIPE - 1; ++st) {
-    if (st < nk) issue(st, st * BK);
+    if (st < nk) issue(st, k_lo + st * BK);
     cp_async_commit();
   }
   for (int kt = 0; kt < nk; ++kt) {
     cp_async_wait<PIPE - 2>();       // this thread's pieces of step kt have landed
     __syncthreads();                 // ... everybody's have, and everybody is done with step kt - 1
     const int nxt = kt + PIPE - 1;
-    if (nxt < nk) issue(nxt % PIPE, nxt * BK);
+    if (nxt < nk) issue(nxt % PIPE, k_lo + nxt * BK);
     cp_async_commit();
     const float* As = ring + (kt % PIPE) * PIPE_STAGE_FLOATS;
     mma_tile<2, 2, true>(reinterpret_cast<const float(*)[BM + 4]>(As), reinterpret_cast<const float(*)[BN + 4]>(As + BK * (BM + 4)),
                    ty, tx, acc);
   }
   cp_async_wait<0>();
+
+  if (OUT == 1) {   // rows of z: m = sample, n = class; z.ld is a multiple of 4 and columns J .. z.ld - 1 get zeros
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int i = j0 + mi * 64 + ty * 4 + a;
+        if (i >= J) continue;
+        float* zr = reinterpret_cast<float*>(z.row(i) + blockIdx.z * range_stride);
+#pragma unroll
+        for (int ni = 0; ni < 2; ++ni) {
+          const int n = d0 + ni * 64 + tx * 4;
+          if (n < z.ld)
+            *reinterpret_cast<float4*>(zr + n) = make_float4(acc[mi * 4 + a][ni * 2].x, acc[mi * 4 + a][ni * 2].y,
+                                                             acc[mi * 4 + a][ni * 2 + 1].x, acc[mi * 4 + a][ni * 2 + 1].y);
+        }
+      }
+    return;
+  }
 
   const bool vec_ok = (D & 3) == 0;
 #pragma unroll
@@ -321,17 +347,48 @@ __global__ void __launch_bounds__(256, 2) apply_f32_pipe_kernel(float* __restric
     }
 }
 
+// dst[c][r] = src row r, column c (R rows of C values behind a row map; dst rows ldr floats long, columns R .. ldr - 1
+// zero).  `copy` (optional): the same rows also copied there, pad columns zero (the factor v = x of the MLR model).
+__global__ void __launch_bounds__(256) transpose_rows_kernel(RowMap src, float* __restrict__ dst, int R, int C, int ldr,
+                                                             RowMap copy) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+#pragma unroll
+  for (int q = 0; q < 32; q += 8) {
+    const int r = r0 + ty + q, c = c0 + tx;
+    float val = 0.f;
+    if (r < R && c < C) val = reinterpret_cast<const float*>(src.row(r))[c];
+    tile[ty + q][tx] = val;
+    if (copy.base != nullptr && r < R && c < copy.ld) reinterpret_cast<float*>(copy.row(r))[c] = val;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 32; q += 8) {
+    const int c = c0 + ty + q, r = r0 + tx;
+    if (c < C && r < ldr) dst[(size_t)c * ldr + r] = tile[tx][ty + q];
+  }
+}
+
 }  // namespace
 
 // Few 128 x 128 tiles and a long reduction (e.g. 1024 samples x 1000 classes over 20000 features): the
-// reduction is cut into up to 4 ranges so that every SM has two blocks of the large-tile kernel.
+// reduction is cut into ranges so that the blocks fill whole waves of two blocks per SM.  Among 1 .. 12 ranges
+// (each at least 512 reduction steps long) the smallest count whose last wave is at least 94 % full is taken,
+// else the count with the fullest waves.
 int forward_f32_splits(int K, int J, int D) {
-  const long long big_tiles = (long long)((K + 127) / 128) * ((J + 127) / 128);
-  if (big_tiles >= 148) return 1;
-  long long ks = (2 * 148) / big_tiles;
-  if (ks > 4) ks = 4;
-  while (ks > 1 && D / ks < 512) --ks;
-  return (int)ks;
+  const long long tiles = (long long)((K + 127) / 128) * ((J + 127) / 128);
+  const long long slots = 2 * 148;
+  if (tiles >= 148) return 1;
+  int best = 1;
+  double best_fill = 0.0;
+  for (int ks = 1; ks <= 12 && D / ks >= 512; ++ks) {
+    const long long blocks = tiles * ks;
+    const double fill = (double)blocks / (double)(((blocks + slots - 1) / slots) * slots);
+    if (fill >= 0.94) return ks;
+    if (fill > best_fill + 1e-9) { best_fill = fill; best = ks; }
+  }
+  return best;
 }
 
 int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const float* Xb, int K, int J, int D,
@@ -362,14 +419,49 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
     dim3 grid((D + 127) / 128, (J + 127) / 128);
     static PerDeviceOnce attr_once;   // function attributes are per device
     if (attr_once.first()) {
-      cudaFuncSetAttribute(apply_f32_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE * PIPE_STAGE_FLOATS * 4);
+      cudaFuncSetAttribute(sgemm_pipe_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE * PIPE_STAGE_FLOATS * 4);
     }
-    apply_f32_pipe_kernel<<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(W, u, v, K, J, D, eta, dev_status);
+    sgemm_pipe_kernel<0><<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(W, u, v, K, J, D, eta, dev_status, RowMap(), 0, 0);
   } else {
     dim3 grid((D + 63) / 64, (J + 63) / 64);
     apply_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, u, v, K, J, D, eta, dev_status);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+// Forward contraction through transposed copies of its operands (workspace: xt [D][ldk], wt [D][ldj] floats with
+// ldk, ldj = K, J rounded up to 4): two bandwidth-bound transposing passes, then the pipelined kernel above, which
+// runs faster than the kernel that transposes through registers.  src: the operand rows a_i (X rows, or pair
+// differences already written as the factor v); copy: optional second destination of those rows (v = x).
+long long forward_f32_nn_workspace_floats(int K, int J, int D) {
+  return (long long)D * (((K + 3) & ~3) + ((J + 3) & ~3));
+}
+
+int launch_forward_f32_nn(cudaStream_t s, const float* W, RowMap src, RowMap copy, int K, int J, int D, float* ws,
+                          RowMap z, RowMap part, long long split_stride, int max_splits, int* nsplit_out) {
+  const int ldk = (K + 3) & ~3, ldj = (J + 3) & ~3;
+  float* xt = ws;
+  float* wt = ws + (size_t)D * ldk;
+  RowMap wrows;
+  wrows.base = const_cast<char*>(reinterpret_cast<const char*>(W));
+  wrows.worker_stride = 0; wrows.ld = D; wrows.B = J > 0 ? J : 1; wrows.es = 4;
+  transpose_rows_kernel<<<dim3((D + 31) / 32, (ldk + 31) / 32), 256, 0, s>>>(src, xt, K, D, ldk, copy);
+  transpose_rows_kernel<<<dim3((D + 31) / 32, (ldj + 31) / 32), 256, 0, s>>>(wrows, wt, J, D, ldj, RowMap());
+  int ks = (part.base != nullptr && nsplit_out != nullptr) ? forward_f32_splits(K, J, D) : 1;
+  if (ks > max_splits) ks = max_splits;
+  if (nsplit_out != nullptr) *nsplit_out = ks;
+  const int per = ((D + ks - 1) / ks + BK - 1) / BK * BK;
+  RowMap a, b;
+  a.base = reinterpret_cast<char*>(xt); a.worker_stride = 0; a.ld = ldk; a.B = D; a.es = 4;
+  b.base = reinterpret_cast<char*>(wt); b.worker_stride = 0; b.ld = ldj; b.B = D; b.es = 4;
+  static PerDeviceOnce attr_once;   // function attributes are per device
+  if (attr_once.first())
+    cudaFuncSetAttribute(sgemm_pipe_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE * PIPE_STAGE_FLOATS * 4);
+  // rows of the output tile = samples (M = K), columns = classes (N = J), reduction over the D features
+  dim3 grid((J + 127) / 128, (K + 127) / 128, ks);
+  sgemm_pipe_kernel<1><<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(nullptr, a, b, D, K, ldj, 0.f, nullptr,
+                                                                       ks > 1 ? part : z, per, split_stride);
+  return cudaGetLastError() == cudaSuccess ? 3 : SFB_ERR_CUDA;
 }
 
 }  // namespace sfb

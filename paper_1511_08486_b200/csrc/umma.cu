@@ -32,7 +32,6 @@
 namespace sfb {
 
 // extra passes implemented in finish.cu
-int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D);
 int launch_finish_mlr_fused(cudaStream_t s, RowMap u, const float2* stats, int n_parts, int part_cols,
                             const int32_t* labels, int K, int J, int* dev_status);
 
