@@ -544,7 +544,7 @@ def main():
             elif path == "f32":
                 out["roofline"] = {"bound": "alu", "achieved": apply_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
                                    "frac": apply_tflops / FP32_FMA_TFLOPS, "traffic": traffic,
-                                   "kernel": "apply_f32_pipe_kernel", "peak_source": "148 SMs x 128 FMA lanes x 1.965 GHz"}
+                                   "kernel": "sgemm_pipe_kernel<0> (apply)", "peak_source": "148 SMs x 128 FMA lanes x 1.965 GHz"}
             else:
                 scale = 1.0 if path == "bf16" else 0.5          # tf32 nominal rate is half of bf16
                 peak = peaks["bf16_sustained"] * scale
@@ -564,7 +564,7 @@ def main():
             elif path == "f32":
                 out["roofline_factors"] = {"bound": "alu", "achieved": fwd_tflops, "peak": FP32_FMA_TFLOPS,
                                            "unit": "TFLOP/s", "frac": fwd_tflops / FP32_FMA_TFLOPS,
-                                           "kernel": "forward_f32_kernel + finishing pass"}
+                                           "kernel": "fp32 forward kernels + finishing pass"}
             else:
                 scale = 1.0 if path == "bf16" else 0.5
                 out["roofline_factors"] = {"bound": "tensor", "achieved": fwd_tflops, "peak": peaks["bf16_sustained"] * scale,
