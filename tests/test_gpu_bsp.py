@@ -22,6 +22,8 @@ CASES = [
     ("C0", "tf32", {}, 0.1),
     ("C1", "tf32", dict(J=200, D=1024, P=4, B=128), 1e-2),
     ("C1", "f32", dict(J=100, D=260, P=6, B=10), 1e-2),
+    ("C1", "f32", dict(J=200, D=1024, P=4, B=128), 1e-2),          # large enough for the transposed-operand forward
+    ("C2", "f32", dict(J=128, D=1024, P=4, B=64), 1e-3),
     ("C2", "f32", dict(J=40, D=300, P=4, B=6), 1e-3),
     ("C2", "tf32", dict(J=64, D=512, P=4, B=64), 1e-3),
     ("C3", "f32", dict(J=70, D=333, P=4, B=5, density=0.1), 1e-2),
