@@ -121,9 +121,13 @@ def test_bsp_bench_under_a_launcher_runs_the_nccl_exchange():
     import os
     import subprocess
     import sys
+    import socket
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as sock:                      # a port nobody holds right now
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "1", "--master-addr",
-           "127.0.0.1", "--master-port", "29533", "bench.py", "--gpus", "1", "--mode", "bsp", "--config", "C1", "--path",
+           "127.0.0.1", "--master-port", str(port), "bench.py", "--gpus", "1", "--mode", "bsp", "--config", "C1", "--path",
            "tf32", "--J", "200", "--D", "1024", "--P", "4", "--B", "128", "--steps", "3", "--warmup", "3",
            "--no-cpu-baseline"]
     res = subprocess.run(cmd, cwd=root, capture_output=True, text=True, timeout=600)
