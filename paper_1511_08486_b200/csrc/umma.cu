@@ -637,7 +637,9 @@ bool encode_rows_map(CUtensorMap* m, int es, const void* base, long long cols, l
     r = fn(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
-    cuuint64_t dims[4] = {(cuuint64_t)CH, (cuuint64_t)rows, (cuuint64_t)workers, (cuuint64_t)(cols / CH)};
+    // whole chunks; a caller that folds a row length that is no multiple of CH (the u rows of the apply) gets
+    // the tail of the last chunk from the bytes that follow the row, and must discard those output indices
+    cuuint64_t dims[4] = {(cuuint64_t)CH, (cuuint64_t)rows, (cuuint64_t)workers, (cuuint64_t)((cols + CH - 1) / CH)};
     cuuint64_t strides[3] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)worker_stride_bytes, 128};
     cuuint32_t box[4] = {(cuuint32_t)CH, (cuuint32_t)box_rows, (cuuint32_t)box_workers, (cuuint32_t)box_chunks};
     r = fn(m, dt, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
@@ -1012,8 +1014,12 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   memset(&p, 0, sizeof(p));
   p.B = d.B; p.P = workers;
   const int m_units = (d.J + BM - 1) / BM;
-  // folding walks the output indices (J for u, D for v) in 128-byte chunks
-  const Variant v = pick_variant(pl, m_units, d.D, (d.J % CH) == 0 && (d.D % CH) == 0);
+  // Folding walks the output indices (J for u, D for v) in 128-byte chunks.  D must be whole chunks.  J need not
+  // be: the last chunk of a u row then also carries the first bytes of what follows the row inside the worker
+  // stream (the next row, or the stream's V block: always inside the buffer), which only feeds accumulator rows
+  // j >= J, and those are never written.  (The V block of the last stream ends the buffer, hence no such
+  // licence for D.)
+  const Variant v = pick_variant(pl, m_units, d.D, (d.D % CH) == 0);
   const int BK = CH * v.ka;
   if (d.B >= BK) { p.k_bb = BK; p.k_wp = 1; p.k_bpw = (d.B + BK - 1) / BK; p.k_blocks = workers * p.k_bpw; }
   else { p.k_bb = pow2_at_least(d.B); p.k_wp = BK / p.k_bb; p.k_bpw = 1; p.k_blocks = (workers + p.k_wp - 1) / p.k_wp; }
