@@ -126,7 +126,13 @@ __global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, i
   for (int k = threadIdx.x; k < row.len; k += 256) {
     const uint32_t c = row.idx[k];
     if (c >= (uint32_t)D || (k > 0 && row.idx[k - 1] >= c)) atomicOr(dev_status, SFB_DEV_BAD_INDEX);   // entry skipped
-    else dst[c] = row.val[k];
+    else {
+      // the tensor cores drop the low 13 mantissa bits of a tf32 operand: rounding the code value to nearest
+      // here (the dense rows are only ever a tf32 operand; the wire keeps the exact CSR values) halves that error
+      float r;
+      asm("cvt.rna.tf32.f32 %0, %1;" : "=f"(r) : "f"(row.val[k]));
+      dst[c] = r;
+    }
   }
 }
 
