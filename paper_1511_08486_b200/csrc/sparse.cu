@@ -129,9 +129,9 @@ __global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, i
     else {
       // the tensor cores drop the low 13 mantissa bits of a tf32 operand: rounding the code value to nearest
       // here (the dense rows are only ever a tf32 operand; the wire keeps the exact CSR values) halves that error
-      float r;
-      asm("cvt.rna.tf32.f32 %0, %1;" : "=f"(r) : "f"(row.val[k]));
-      dst[c] = r;
+      uint32_t r;
+      asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(row.val[k]));
+      dst[c] = __uint_as_float(r);
     }
   }
 }
