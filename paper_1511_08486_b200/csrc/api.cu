@@ -28,6 +28,10 @@ struct sfb_ctx {
   bool aux_ok;
   float* f32_part;          // fp32 dense path: partial products [splits][K][ldp] of a split forward reduction
   int ldp, f32_splits;
+  // DML, fp32 path: which pairs of the current step contribute (u_i != 0), their ordered list and its length;
+  // the step's apply leaves the others out (bit-identical result, fewer multiply-adds)
+  uint8_t* dml_active;
+  int* dml_idx;             // [K] indices followed by the count
   float* f32_nn_ws;         // fp32 dense path: transposed copies of the forward's operands (large shapes only)
   float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
   float* loss_i;            // sfb_loss: per-sample objective [K]
@@ -178,7 +182,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     }
     const RowMap zsrc = ks > 1 ? part : u;
     if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, zsrc, u, aux->labels, K, d.J, c->dev_status, ks, sstride));
-    else ACC(launch_finish_dml(c->stream, zsrc, u, aux->similar, d.margin, K, d.J, ks, sstride));
+    else ACC(launch_finish_dml(c->stream, zsrc, u, aux->similar, d.margin, K, d.J, ks, sstride, c->dml_active));
     return SFB_OK;
   }
   // tensor-core paths
@@ -260,6 +264,10 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     c->ldp = (desc->J + 3) & ~3;
     c->f32_splits = ks;
     if (ks > 1) ok = cudaMalloc(&c->f32_part, (size_t)ks * c->K * c->ldp * 4) == cudaSuccess;
+    if (ok && desc->model == SFB_DML) {
+      ok = cudaMalloc(&c->dml_active, (size_t)c->K) == cudaSuccess;
+      if (ok) ok = cudaMalloc(&c->dml_idx, ((size_t)c->K + 1) * 4) == cudaSuccess;
+    }
     // shapes with at least a tile of work per dimension take the forward through transposed operand copies
     const long long nn_floats = forward_f32_nn_workspace_floats(c->K, desc->J, desc->D);
     if (ok && c->K >= 128 && desc->J >= 64 && desc->D >= 512 && nn_floats * 4 <= (2LL << 30))
@@ -315,6 +323,8 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->csc_ws) cudaFree(c->csc_ws);
   if (c->f32_part) cudaFree(c->f32_part);
   if (c->f32_nn_ws) cudaFree(c->f32_nn_ws);
+  if (c->dml_active) cudaFree(c->dml_active);
+  if (c->dml_idx) cudaFree(c->dml_idx);
   if (c->loss_rows) cudaFree(c->loss_rows);
   if (c->loss_i) cudaFree(c->loss_i);
   for (int k = 0; k < 2; ++k)
@@ -461,7 +471,9 @@ int sfb_pack(sfb_ctx* c, const void* U, const void* V, const sfb_aux* aux, void*
 }
 
 // csc_built: the atom-major re-sort of this buffer's codes for these K samples is already in the workspace
-static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check, bool csc_built = false) {
+// active_rows: c->dml_active describes the u rows of this buffer (set by the factor stage of the same step)
+static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K, bool check, bool csc_built = false,
+                      bool active_rows = false) {
   const sfb_desc& d = c->d;
   if (check) ACC(launch_check_header(c->stream, sf_buf, d, c->l, c->dev_status));
   if (d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
@@ -477,8 +489,15 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
     if (check) ACC(launch_densify_codes(c->stream, stream_codes(c, sf_buf), dense_codes(c), K, d.D, c->dev_status));
     ACC(umma_apply(c->umma, c->stream, W, nullptr, stream_u(c, sf_buf), dense_codes(c), eta, K, c->dev_status));
   } else if (d.path == SFB_PATH_F32) {
+    const int* idx = nullptr;
+    const int* n_idx = nullptr;
+    if (active_rows && c->dml_active != nullptr) {   // ordered list of the contributing pairs among the first K
+      ACC(launch_compact_active(c->stream, c->dml_active, K, c->dml_idx, c->dml_idx + c->K));
+      idx = c->dml_idx;
+      n_idx = c->dml_idx + c->K;
+    }
     ACC(launch_apply_f32(c->stream, reinterpret_cast<float*>(W), stream_u(c, sf_buf), stream_v(c, sf_buf), K, d.J, d.D,
-                         eta, c->dev_status));
+                         eta, c->dev_status, idx, n_idx));
   } else {
     ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status));
     if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
@@ -562,7 +581,7 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   if (r < 0) return r;
   if (forked && cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess) return SFB_ERR_CUDA;
   if (c->profiling) cudaEventRecord(c->prof_ev[slot][1], c->stream);
-  r = apply_from(c, W, sf_buf, eta, K, false, csc_built);
+  r = apply_from(c, W, sf_buf, eta, K, false, csc_built, d.model == SFB_DML && d.path == SFB_PATH_F32);
   if (c->profiling) {
     cudaEventRecord(c->prof_ev[slot][2], c->stream);
     c->prof_n++;

@@ -92,7 +92,9 @@ int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const flo
 
 // W[j][d] -= eta * sum_{i<K} U[i][j] * V[i][d] on fp32 CUDA cores (fixed summation order).
 int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J, int D, float eta,
-                     const int* dev_status);
+                     const int* dev_status, const int* row_idx = nullptr, const int* n_rows = nullptr);
+// row_idx / n_rows (optional, device): apply only the factor rows row_idx[0 .. *n_rows), in that order, instead of
+// rows 0 .. K-1 (rows that are known to be all zeros can be left out: the result is bit-identical).
 
 // MLR epilogue: u = softmax(z) - onehot(label).  z rows are fp32; u rows fp32 or bf16 (u.es).
 // z may be `nsplit` partial products (split s at z + s * split_stride_bytes), summed in split order.
@@ -100,8 +102,11 @@ int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels,
                       int nsplit = 1, long long split_stride_bytes = 0);
 
 // DML epilogue: u = +z (similar) or -z * [|z|^2 < margin] (dissimilar).
+// active (optional, [K] bytes): 1 where the pair contributes (similar, or dissimilar inside the margin), 0 where u_i = 0.
 int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
-                      int nsplit = 1, long long split_stride_bytes = 0);
+                      int nsplit = 1, long long split_stride_bytes = 0, uint8_t* active = nullptr);
+// idx[0 .. *n_out) = ascending list of the samples i < K with active[i] != 0 (device arrays; one ordered block).
+int launch_compact_active(cudaStream_t s, const uint8_t* active, int K, int* idx, int* n_out);
 
 // Copies K rows of `cols` values from src to dst rows (same value type), zero-filling dst pad columns.
 int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols);

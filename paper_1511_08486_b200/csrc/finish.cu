@@ -142,7 +142,8 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
 }
 
 __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, const uint8_t* __restrict__ similar,
-                                                                 float margin, int K, int J, int cache_floats, int nsplit, long long zstride) {
+                                                                 float margin, int K, int J, int cache_floats, int nsplit, long long zstride,
+                                                                 uint8_t* __restrict__ active) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -165,6 +166,7 @@ __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, co
   n = block_sum(n, red);
   const bool sim = similar[i] != 0;
   const float g = sim ? 1.f : ((n < margin) ? -1.f : 0.f);   // strict hinge: inactive at equality
+  if (active != nullptr && threadIdx.x == 0) active[i] = (g != 0.f) ? 1 : 0;   // u_i is all zeros otherwise
 
   const int ld4 = u.ld >> 2;
   for (int q = threadIdx.x; q < ld4; q += blockDim.x) {
@@ -359,15 +361,50 @@ int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels,
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
+// idx[0 .. n) = the samples i < K with active[i] != 0, in ascending order; *n_out = n.  One block, ordered.
+__global__ void __launch_bounds__(1024) compact_active_kernel(const uint8_t* __restrict__ active, int K, int* __restrict__ idx,
+                                                              int* __restrict__ n_out) {
+  __shared__ int warp_cnt[32];
+  __shared__ int base;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int start = 0; start < K; start += 1024) {
+    const int i = start + threadIdx.x;
+    const bool f = i < K && active[i] != 0;
+    const unsigned m = __ballot_sync(0xffffffffu, f);
+    const int before = __popc(m & ((1u << lane) - 1u));
+    if (lane == 0) warp_cnt[warp] = __popc(m);
+    __syncthreads();
+    int off = 0;
+    for (int w = 0; w < warp; ++w) off += warp_cnt[w];
+    if (f) idx[base + off + before] = i;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int t = 0;
+      for (int w = 0; w < 32; ++w) t += warp_cnt[w];
+      base += t;
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *n_out = base;
+}
+
+int launch_compact_active(cudaStream_t s, const uint8_t* active, int K, int* idx, int* n_out) {
+  compact_active_kernel<<<1, 1024, 0, s>>>(active, K, idx, n_out);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
 int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
-                      int nsplit, long long split_stride_bytes) {
+                      int nsplit, long long split_stride_bytes, uint8_t* active) {
   const int cf = fin_cache_floats(J);
   static PerDeviceOnce attr_once;   // function attributes are per device
   if (attr_once.first()) {
     cudaFuncSetAttribute(finish_mlr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
   }
-  finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf, nsplit, split_stride_bytes / 4);
+  finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf, nsplit, split_stride_bytes / 4,
+                                                              active);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

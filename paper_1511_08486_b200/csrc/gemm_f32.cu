@@ -249,14 +249,16 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 template <int OUT>
 __global__ void __launch_bounds__(256, 2) sgemm_pipe_kernel(float* __restrict__ W, RowMap u, RowMap v, int K, int J,
                                                          int D, float eta, const int* __restrict__ dev_status,
-                                                         RowMap z, int k_per_range, long long range_stride) {
+                                                         RowMap z, int k_per_range, long long range_stride,
+                                                         const int* __restrict__ row_idx, const int* __restrict__ n_rows) {
   constexpr int BM = 128, BN = 128;
   extern __shared__ __align__(16) float ring[];
   if (OUT == 0 && dev_status != nullptr && (*dev_status & SFB_DEV_BAD_HEADER)) return;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const int j0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
   const int k_lo = (OUT == 1) ? blockIdx.z * k_per_range : 0;
-  const int k_hi = (OUT == 1) ? min(K, k_lo + k_per_range) : K;
+  // OUT 0 with a row list: the reduction runs over the listed factor rows only (the others are all zeros)
+  const int k_hi = (OUT == 1) ? min(K, k_lo + k_per_range) : (n_rows != nullptr ? min(K, *n_rows) : K);
   const int lr = tid >> 5, lc = (tid & 31) * 4;   // loader: factor rows lr and lr + 8 of the step, 4 columns at lc
   // bytes of this thread's 16-byte piece that exist (the rest is zero-filled); a piece with nothing to read
   // still needs a valid aligned address: column 0 of a valid row
@@ -271,7 +273,7 @@ __global__ void __launch_bounds__(256, 2) sgemm_pipe_kernel(float* __restrict__ 
     for (int h = 0; h < 2; ++h) {
       const int r = lr + 8 * h, i = k0 + r;
       const bool ok = i < k_hi;
-      const int ii = ok ? i : 0;
+      const int ii = ok ? ((OUT == 0 && row_idx != nullptr) ? row_idx[i] : i) : 0;
       cp_async16_zfill(As + r * (BM + 4) + lc, u.row(ii) + u_off, ok ? u_bytes : 0);
       cp_async16_zfill(Bs + r * (BN + 4) + lc, v.row(ii) + v_off, ok ? v_bytes : 0);
     }
@@ -413,7 +415,7 @@ int launch_forward_f32(cudaStream_t s, const float* W, const float* X, const flo
 }
 
 int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J, int D, float eta,
-                     const int* dev_status) {
+                     const int* dev_status, const int* row_idx, const int* n_rows) {
   const long long big_tiles = (long long)((J + 127) / 128) * ((D + 127) / 128);
   if (big_tiles >= 148) {
     dim3 grid((D + 127) / 128, (J + 127) / 128);
@@ -421,7 +423,8 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
     if (attr_once.first()) {
       cudaFuncSetAttribute(sgemm_pipe_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE * PIPE_STAGE_FLOATS * 4);
     }
-    sgemm_pipe_kernel<0><<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(W, u, v, K, J, D, eta, dev_status, RowMap(), 0, 0);
+    sgemm_pipe_kernel<0><<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(W, u, v, K, J, D, eta, dev_status, RowMap(), 0, 0,
+                                                                         row_idx, n_rows);
   } else {
     dim3 grid((D + 63) / 64, (J + 63) / 64);
     apply_f32_kernel<1, 1><<<grid, 256, 0, s>>>(W, u, v, K, J, D, eta, dev_status);
@@ -460,7 +463,7 @@ int launch_forward_f32_nn(cudaStream_t s, const float* W, RowMap src, RowMap cop
   // rows of the output tile = samples (M = K), columns = classes (N = J), reduction over the D features
   dim3 grid((J + 127) / 128, (K + 127) / 128, ks);
   sgemm_pipe_kernel<1><<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(nullptr, a, b, D, K, ldj, 0.f, nullptr,
-                                                                       ks > 1 ? part : z, per, split_stride);
+                                                                       ks > 1 ? part : z, per, split_stride, nullptr, nullptr);
   return cudaGetLastError() == cudaSuccess ? 3 : SFB_ERR_CUDA;
 }
 

@@ -155,3 +155,38 @@ def test_saturated_softmax(path, over):
         assert orc.rel_fro(U, U_or) <= TOL[path]
     finally:
         wl.close()
+
+
+def test_dml_step_leaves_out_inactive_pairs_bit_identically():
+    """The fp32 DML step applies only the pairs with u != 0 (an ordered index list built on the device); the
+    result must equal, bit for bit, the staged calls that multiply the zero rows through."""
+    cfg = scaled("C2", J=300, D=8192, P=4, B=96)              # 3 x 64 large tiles: the pipelined apply kernel
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        wl.step(0, eta=1e-4)
+        torch.cuda.synchronize()
+        W_step, buf_step = wl.W.clone(), wl.sf_buf.clone()
+        _, U, _ = orc.unpack(buf_step.cpu().numpy())
+        inactive = int((~U.any(axis=1)).sum())
+        assert 0 < inactive < cfg["K"]                        # the case really has pairs beyond the margin
+        wl.reset()
+        wl.sf_buf.zero_()
+        wl.compute_factors(0)
+        wl.pack(0, clock=0)
+        wl.apply(1e-4)
+        assert wl.ctx.status() == 0
+        assert torch.equal(wl.sf_buf, buf_step) and torch.equal(wl.W, W_step)
+        # partial apply inside the step: only the first two workers' streams
+        wl.reset()
+        wl.step(0, eta=1e-4, K=2 * cfg["B"])
+        torch.cuda.synchronize()
+        W_part = wl.W.clone()
+        wl.reset()
+        wl.compute_factors(0)
+        wl.pack(0, clock=0)
+        wl.apply(1e-4, K=2 * cfg["B"])
+        torch.cuda.synchronize()
+        assert torch.equal(wl.W, W_part)
+    finally:
+        wl.close()
