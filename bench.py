@@ -527,8 +527,13 @@ def main():
             "stages_ms": {"factors": f_ms, "apply": a_ms, "steps_recorded": n_rec},
             "clocks": clocks.summary(),
         }
+        applied = wl.ctx.active_pairs()
+        if alg is not None and 0 < applied < K:
+            # the apply left out pairs whose u is zero: its work is counted on the pairs it multiplied through
+            alg["flops_all_pairs"] = alg["flops"]
+            out["pairs_applied_last_step"] = applied
         if alg is not None:
-            apply_tflops = alg["flops"] / (a_ms * 1e-3) / 1e12
+            apply_tflops = alg["flops"] * (applied / K if 0 < applied < K else 1.0) / (a_ms * 1e-3) / 1e12
             fwd_tflops = alg["flops"] / (f_ms * 1e-3) / 1e12
             traffic = NCU_APPLY_TRAFFIC_BYTES.get((args.config, path)) if not over else None
             if alg["sparse"]:

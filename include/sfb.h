@@ -209,6 +209,12 @@ int sfb_prox(sfb_ctx* ctx, void* W);
  * A label outside [0, J) contributes 0 and sets SFB_DEV_BAD_LABEL. */
 int sfb_loss(sfb_ctx* ctx, const void* W, const void* X, const sfb_aux* aux, double* loss);
 
+/* Number of (u, v) pairs the last sfb_step actually multiplied through.  SFB_DML on SFB_PATH_F32 leaves out the
+ * pairs whose u is zero (dissimilar pairs beyond the margin; the update is bit-identical to the sum over all K
+ * slots, Section 6 notes that such sparsity can be used); every other model / path applies all K slots and
+ * reports K.  Synchronises the stream.  *n is 0 before the first step. */
+int sfb_active_pairs(sfb_ctx* ctx, int32_t* n);
+
 /* Tells the context that W was changed by someone else, so a cached bf16 shadow is stale. */
 int sfb_invalidate(sfb_ctx* ctx);
 

@@ -24,7 +24,7 @@ EXPORTS = (
     "sfb_apply", "sfb_step", "sfb_invalidate", "sfb_status", "sfb_launch_count", "sfb_strerror",
     "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
     "sfb_halton_peers", "sfb_ssp_may_proceed", "sfb_prox", "sfb_step_host",
-    "sfb_loss", "sfb_factors_shard", "sfb_commit_header", "sfb_sf_buffer_layout",
+    "sfb_loss", "sfb_factors_shard", "sfb_commit_header", "sfb_sf_buffer_layout", "sfb_active_pairs",
 )
 
 
@@ -78,6 +78,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_step_host.restype = C.c_int
     lib.sfb_prox.argtypes = [vp, vp]
     lib.sfb_prox.restype = C.c_int
+    lib.sfb_active_pairs.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.sfb_active_pairs.restype = C.c_int
     lib.sfb_loss.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp]
     lib.sfb_loss.restype = C.c_int
     lib.sfb_factors_shard.argtypes = [vp, vp, vp, C.POINTER(sfb_aux), vp, C.c_int32, C.c_int32]
@@ -241,6 +243,12 @@ class Context:
 
     def commit_header(self, sf_buf, clock: int = 0):
         self._chk(self._lib.sfb_commit_header(self._h, _ptr(sf_buf), clock), "sfb_commit_header")
+
+    def active_pairs(self) -> int:
+        """Pairs the last step multiplied through (synchronises)."""
+        n = C.c_int32(0)
+        self._chk(self._lib.sfb_active_pairs(self._h, C.byref(n)), "sfb_active_pairs")
+        return int(n.value)
 
     def loss(self, W, X, aux: sfb_aux, out):
         """Minibatch objective at W into `out` (one float64 on the device); asynchronous."""

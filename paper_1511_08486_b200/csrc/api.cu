@@ -32,6 +32,8 @@ struct sfb_ctx {
   // the step's apply leaves the others out (bit-identical result, fewer multiply-adds)
   uint8_t* dml_active;
   int* dml_idx;             // [K] indices followed by the count
+  int last_step_K;          // K of the last sfb_step (0: none yet) and whether its apply walked the list
+  bool last_step_listed;
   float* f32_nn_ws;         // fp32 dense path: transposed copies of the forward's operands (large shapes only)
   float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
   float* loss_i;            // sfb_loss: per-sample objective [K]
@@ -390,6 +392,21 @@ int sfb_loss(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, doubl
   return SFB_OK;
 }
 
+int sfb_active_pairs(sfb_ctx* c, int32_t* n) {
+  if (c == nullptr || n == nullptr) return SFB_ERR_ARG;
+  *n = 0;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  if (c->last_step_K == 0) return SFB_OK;
+  if (c->dml_idx == nullptr || !c->last_step_listed) {
+    *n = c->last_step_K;
+    return SFB_OK;
+  }
+  int32_t h = 0;
+  if (cudaMemcpy(&h, c->dml_idx + c->K, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SFB_ERR_CUDA;
+  *n = h;
+  return SFB_OK;
+}
+
 int sfb_invalidate(sfb_ctx* c) {
   if (c == nullptr) return SFB_ERR_ARG;
   c->shadow_of = nullptr;
@@ -581,7 +598,11 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   if (r < 0) return r;
   if (forked && cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess) return SFB_ERR_CUDA;
   if (c->profiling) cudaEventRecord(c->prof_ev[slot][1], c->stream);
-  r = apply_from(c, W, sf_buf, eta, K, false, csc_built, d.model == SFB_DML && d.path == SFB_PATH_F32);
+  const bool listed = d.model == SFB_DML && d.path == SFB_PATH_F32 && c->dml_active != nullptr &&
+                      (long long)((d.J + 127) / 128) * ((d.D + 127) / 128) >= 148;   // the large-tile apply takes the list
+  r = apply_from(c, W, sf_buf, eta, K, false, csc_built, listed);
+  c->last_step_K = K;
+  c->last_step_listed = listed;
   if (c->profiling) {
     cudaEventRecord(c->prof_ev[slot][2], c->stream);
     c->prof_n++;

@@ -170,6 +170,7 @@ def test_dml_step_leaves_out_inactive_pairs_bit_identically():
         _, U, _ = orc.unpack(buf_step.cpu().numpy())
         inactive = int((~U.any(axis=1)).sum())
         assert 0 < inactive < cfg["K"]                        # the case really has pairs beyond the margin
+        assert wl.ctx.active_pairs() == cfg["K"] - inactive   # what the step's apply multiplied through
         wl.reset()
         wl.sf_buf.zero_()
         wl.compute_factors(0)
