@@ -147,8 +147,12 @@ int sfb_pack(sfb_ctx* ctx, const void* U, const void* V, const sfb_aux* aux, voi
  * multiple of B and at most P*B.  The sum order is fixed, so results are bit-reproducible. */
 int sfb_apply(sfb_ctx* ctx, void* W, const void* sf_buf, float eta, int32_t K);
 
-/* One iteration: factors written straight into the SF buffer (header and directory included, with
- * the given clock), then the apply of the first K slots.  K as in sfb_apply. */
+/* One iteration as Section 3 states it for a worker under BSP (Section 4.1): compute the SF pairs of the
+ * minibatch against the current W, commit them (the broadcast: here, all P simulated workers' streams
+ * written straight into the SF buffer, header and directory included, with the given clock), then apply
+ * the pairs of all workers, W <- W - eta * sum_i u_i v_i^T, over the first K slots.  K as in sfb_apply.
+ * SFB_SC: if a worker's nonzeros exceed cap_p (SFB_DEV_CAPACITY), u is computed from the truncated codes,
+ * the ones that are on the wire and that the apply uses. */
 int sfb_step(sfb_ctx* ctx, void* W, const void* X, const sfb_aux* aux, void* sf_buf, float eta, int32_t K,
              uint32_t clock);
 
@@ -257,14 +261,16 @@ int sfb_ssp_may_proceed(int64_t t_p, const int64_t* tau, int32_t P, int64_t stal
  * problems return SFB_ERR_SCRATCH and launch nothing.  The call itself never allocates or frees.
  *
  * W [J][D] fp32; rowptr [K+1], idx, val: CSR codes (fp32 values, strictly ascending indices);
- * Xdata [K][J] fp32; U out [K][ldu] fp32 with ldu >= J a multiple of 4 (pad columns written as
- * zeros).  dev_status: optional device int that receives the SFB_DEV_* bits (cleared by the call);
- * NULL keeps them in the library's own word.  All pointers are device pointers of the caller.
+ * Xdata [K][J] fp32; U out [K][ldu] fp32 with ldu >= J a multiple of 4 (every pad column up to ldu
+ * is written as zero).  dev_status: optional device int that receives the SFB_DEV_* bits (cleared
+ * by the call).  With NULL the bits go to a word inside the library that no call reads back: pass
+ * a pointer if malformed codes must be noticed.  All pointers are device pointers of the caller.
  *
- * The first call on each device looks up the address of the built-in array; make that first call
- * outside any stream capture.  All calls share the array and it keeps the last call's contents:
- * everything a call depends on is rewritten by that call, but two calls that overlap on the GPU
- * (different streams, or concurrent host threads) race on it, so keep them on one stream. */
+ * The first call on each device looks up the address of the built-in array (host threads that make
+ * it at the same time are serialised); make that first call outside any stream capture.  All calls
+ * share the array and it keeps the last call's contents: everything a call depends on is rewritten
+ * by that call, but two calls whose kernels overlap on the GPU (different streams, or host threads
+ * that enqueue at the same time on different streams) race on it, so keep them on one stream. */
 int sfb_sc_factors_noalloc(const void* W, int32_t J, int32_t D, int32_t K, const uint32_t* rowptr,
                            const uint32_t* idx, const void* val, const void* Xdata, void* U, int32_t ldu,
                            int32_t* dev_status, void* cuda_stream);

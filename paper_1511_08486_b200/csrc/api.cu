@@ -16,8 +16,6 @@ struct sfb_ctx {
   cudaStream_t stream;
   int K;
   int* dev_status;          // sticky device status word
-  float* z_ws;              // fp32 products z = W a, [K][ldz], when u is stored in another type (bf16 path)
-  int ldz;
   float* wt_ws;             // SC, fp32 path: atom-major copy of W for the forward
   float* a_dense;           // SC, tf32 path: dense rows of the codes, [K][ldv]
   void* csc_ws;             // SC, fp32 path: scratch of the atom-major re-sort of the codes (when K fits)
@@ -101,12 +99,13 @@ RowMap stream_v(const sfb_ctx* c, const void* sf_buf) {
   return m;
 }
 RowMap dense_codes(const sfb_ctx* c) { return caller_rows(c->a_dense, c->l.ldv, c->d.B, 4); }
-RowMap z_rows(const sfb_ctx* c) { return caller_rows(c->z_ws, c->ldz, c->d.B, 4); }
 
-CsrView global_codes(const sfb_aux* a, int B) {
+// cap_p > 0: every worker's rows end after its first cap_p nonzeros, as in the stream pack_csr writes
+CsrView global_codes(const sfb_aux* a, int B, int cap_p = 0) {
   CsrView v;
   memset(&v, 0, sizeof(v));
   v.rowptr = a->rowptr; v.idx = a->idx; v.val = reinterpret_cast<const float*>(a->val); v.B = B;
+  v.cap_p = cap_p;
   return v;
 }
 CsrView stream_codes(const sfb_ctx* c, const void* sf_buf) {
@@ -192,7 +191,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     const int r = ensure_shadow(c, W);
     if (r < 0) return r;
   }
-  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, z_rows(c), c->dev_status, workers));
+  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, c->dev_status, workers));
   return SFB_OK;
 }
 
@@ -276,8 +275,7 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
       ok = cudaMalloc(&c->f32_nn_ws, (size_t)nn_floats * 4) == cudaSuccess;
   }
   if (ok) {
-    const char* na = getenv("SFB_NO_AUX_STREAM");
-    if (!(na != nullptr && na[0] == '1') && cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) == cudaSuccess) {
+    if (cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) == cudaSuccess) {
       const bool e1 = cudaEventCreateWithFlags(&c->aux_fork, cudaEventDisableTiming) == cudaSuccess;
       const bool e2 = e1 && cudaEventCreateWithFlags(&c->aux_join, cudaEventDisableTiming) == cudaSuccess;
       c->aux_ok = e2;
@@ -295,7 +293,7 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     return SFB_ERR_ALLOC;
   }
   if (desc->path != SFB_PATH_F32) {
-    const int ur = umma_plan_create(c->d, c->l, c->z_ws, c->ldz, c->w_shadow, &c->umma);
+    const int ur = umma_plan_create(c->d, c->l, &c->umma);
     if (ur != SFB_OK) {
       sfb_destroy(c);
       return ur;
@@ -319,7 +317,6 @@ int sfb_destroy(sfb_ctx* c) {
     for (int i = 0; i < 128; ++i)
       for (int e = 0; e < 3; ++e) cudaEventDestroy(c->prof_ev[i][e]);
   if (c->dev_status) cudaFree(c->dev_status);
-  if (c->z_ws) cudaFree(c->z_ws);
   if (c->wt_ws) cudaFree(c->wt_ws);
   if (c->a_dense) cudaFree(c->a_dense);
   if (c->csc_ws) cudaFree(c->csc_ws);
@@ -495,7 +492,8 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
   if (check) ACC(launch_check_header(c->stream, sf_buf, d, c->l, c->dev_status));
   if (d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
     if (!csc_built)
-      ACC(launch_sc_csc_build(c->stream, stream_codes(c, sf_buf), K, d.D, (long long)d.nnz_capacity, c->csc_ws));
+      ACC(launch_sc_csc_build(c->stream, stream_codes(c, sf_buf), K, d.D, (long long)d.nnz_capacity, c->csc_ws,
+                              c->dev_status));
     ACC(launch_sc_csc_apply(c->stream, reinterpret_cast<float*>(W), stream_u(c, sf_buf), K, d.J, d.D, eta,
                             (long long)d.nnz_capacity, c->csc_ws, c->dev_status));
   } else if (d.v_sparse && d.path == SFB_PATH_F32) {
@@ -582,21 +580,42 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   }
   cudaStream_t hs = forked ? c->aux : c->stream;
   bool csc_built = false;
-  if (d.v_sparse) {
-    ACC(launch_pack_csr(hs, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
-                        c->dev_status));
-    // the forward reads the codes it just committed to the buffer, or, beside the packing, the caller's arrays
-    codes = forked ? global_codes(aux, d.B) : stream_codes(c, sf_buf);
+  // From here on the auxiliary stream may hold work of this call: every exit joins it first (join_aux), so that the
+  // context's stream never runs ahead of it and a stream capture in progress stays well formed.
+  auto aux_side = [&]() -> int {
+    if (d.v_sparse) {
+      ACC(launch_pack_csr(hs, sf_buf, d, c->l, aux->rowptr, aux->idx, reinterpret_cast<const float*>(aux->val),
+                          c->dev_status));
+      // the forward reads the codes it just committed to the buffer, or, beside the packing, the caller's arrays
+      // cut to the same per-worker capacity (so u always belongs to the codes that are on the wire and applied)
+      codes = forked ? global_codes(aux, d.B, c->l.cap_p) : stream_codes(c, sf_buf);
+    }
+    ACC(launch_write_header(hs, sf_buf, d, c->l, clock, d.v_sparse ? aux->rowptr : nullptr));
+    if (forked && d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
+      ACC(launch_sc_csc_build(hs, stream_codes(c, sf_buf), K, d.D, (long long)d.nnz_capacity, c->csc_ws, c->dev_status));
+      csc_built = true;
+    }
+    return SFB_OK;
+  };
+  auto join_aux = [&]() -> int {
+    if (!forked) return SFB_OK;
+    if (cudaEventRecord(c->aux_join, c->aux) != cudaSuccess || cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess)
+      return SFB_ERR_CUDA;
+    return SFB_OK;
+  };
+  r = aux_side();
+  if (r < 0) {
+    join_aux();
+    return r;
   }
-  ACC(launch_write_header(hs, sf_buf, d, c->l, clock, d.v_sparse ? aux->rowptr : nullptr));
-  if (forked && d.v_sparse && d.path == SFB_PATH_F32 && c->csc_ws != nullptr) {
-    ACC(launch_sc_csc_build(hs, stream_codes(c, sf_buf), K, d.D, (long long)d.nnz_capacity, c->csc_ws));
-    csc_built = true;
+  // the join event is recorded before the forward pass is enqueued, so the wait below covers exactly the side work
+  if (forked && cudaEventRecord(c->aux_join, c->aux) != cudaSuccess) {
+    join_aux();
+    return SFB_ERR_CUDA;
   }
-  if (forked && cudaEventRecord(c->aux_join, c->aux) != cudaSuccess) return SFB_ERR_CUDA;
   r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes);
-  if (r < 0) return r;
   if (forked && cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess) return SFB_ERR_CUDA;
+  if (r < 0) return r;
   if (c->profiling) cudaEventRecord(c->prof_ev[slot][1], c->stream);
   const bool listed = d.model == SFB_DML && d.path == SFB_PATH_F32 && c->dml_active != nullptr &&
                       (long long)((d.J + 127) / 128) * ((d.D + 127) / 128) >= 148;   // the large-tile apply takes the list

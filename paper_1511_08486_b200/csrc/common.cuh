@@ -131,6 +131,8 @@ struct CsrView {
   const float* val;
   long long streams_off, stream_stride, v_off, rp_bytes, idx_bytes;  // stream-relative offsets (base != nullptr)
   int B;
+  int cap_p;                 // global arrays only: > 0 cuts every worker's rows off after its first cap_p nonzeros
+                             // (what pack_csr keeps in the stream); 0 = rows as given
 };
 // Wt is a caller-provided workspace of sc_forward_workspace_bytes(J, D) bytes (atom-major copy of W).
 long long sc_forward_workspace_bytes(int J, int D);
@@ -149,7 +151,10 @@ int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K
                         long long nnz_capacity, void* workspace, const int* dev_status_ro);
 // The two halves of launch_sc_apply_csc: the re-sort reads only the codes (it can run beside the forward
 // pass), the update needs u and the workspace the re-sort filled.
-int launch_sc_csc_build(cudaStream_t s, CsrView codes, int K, int D, long long nnz_capacity, void* workspace);
+// dev_status (optional): SFB_DEV_BAD_INDEX is set for entries the re-sort leaves out (atom out of range, row not
+// strictly ascending: the same entries the forward pass skips).
+int launch_sc_csc_build(cudaStream_t s, CsrView codes, int K, int D, long long nnz_capacity, void* workspace,
+                        int* dev_status = nullptr);
 int launch_sc_csc_apply(cudaStream_t s, float* W, RowMap u, int K, int J, int D, float eta, long long nnz_capacity,
                         void* workspace, const int* dev_status_ro);
 

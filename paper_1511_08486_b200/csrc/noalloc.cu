@@ -10,7 +10,9 @@
 // The array below is device memory reserved on every GPU that loads the library, for the life of
 // the process.  In host code its name is only a stand-in for that memory, never a pointer a kernel
 // may be given; the device address is looked up once per device with cudaGetSymbolAddress.
+#include <atomic>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -18,15 +20,16 @@ namespace {
 
 constexpr long long kMaxWtFloats = 4ll << 20;   // 16 MiB: D * roundup(J, 4) may not exceed this
 
-__device__ __align__(256) float g_wt_scratch[kMaxWtFloats];
-__device__ __align__(256) int g_status_scratch[64];
+static __device__ __align__(256) float g_wt_scratch[kMaxWtFloats];
+static __device__ __align__(256) int g_status_scratch[64];
 
 struct DeviceSlots {
-  bool ready;
+  std::atomic<bool> ready;
   float* wt;
   int* status;
 };
 DeviceSlots g_slots[64];
+std::mutex g_setup_mutex;   // two host threads may make the first call on a device at the same time
 
 // Looks the two symbol addresses up for the current device (first call on that device only).
 int setup_current_device(DeviceSlots** out) {
@@ -34,7 +37,12 @@ int setup_current_device(DeviceSlots** out) {
   if (cudaGetDevice(&dev) != cudaSuccess) return SFB_ERR_CUDA;
   if (dev < 0 || dev >= 64) return SFB_ERR_UNSUPPORTED;
   DeviceSlots& s = g_slots[dev];
-  if (!s.ready) {
+  if (!s.ready.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (s.ready.load(std::memory_order_acquire)) {
+      *out = &s;
+      return SFB_OK;
+    }
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SFB_ERR_CUDA;
     if (major != 10) return SFB_ERR_UNSUPPORTED;
@@ -44,7 +52,7 @@ int setup_current_device(DeviceSlots** out) {
     p = nullptr;
     if (cudaGetSymbolAddress(&p, g_status_scratch) != cudaSuccess || p == nullptr) return SFB_ERR_CUDA;
     s.status = static_cast<int*>(p);
-    s.ready = true;
+    s.ready.store(true, std::memory_order_release);
   }
   *out = &s;
   return SFB_OK;

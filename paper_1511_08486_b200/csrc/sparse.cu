@@ -25,7 +25,11 @@ struct CsrRow {
 __device__ __forceinline__ CsrRow csr_row(const CsrView& c, int i) {
   CsrRow r;
   if (c.base == nullptr) {
-    const uint32_t s = c.rowptr[i], e = c.rowptr[i + 1];
+    uint32_t s = c.rowptr[i], e = c.rowptr[i + 1];
+    if (c.cap_p > 0) {   // what the worker's stream can hold: the same truncation as pack_csr
+      const uint32_t lim = c.rowptr[(size_t)(i / c.B) * c.B] + (uint32_t)c.cap_p;
+      s = min(s, lim); e = min(e, lim);
+    }
     r.idx = c.idx + s;
     r.val = c.val + s;
     r.len = (int)(e - s);
@@ -223,7 +227,10 @@ __global__ void __launch_bounds__(SLAB_T) sc_apply_kernel(float* __restrict__ W,
         const int mid = (lo + hi) >> 1;
         if (row.idx[mid] < (uint32_t)d0) lo = mid + 1; else hi = mid;
       }
-      while (lo + cnt < row.len && cnt < SLAB_D && row.idx[lo + cnt] < (uint32_t)(d0 + dn)) ++cnt;
+      // (the lower bound matters only for rows that are not ascending: nothing outside the slab is ever addressed)
+      while (lo + cnt < row.len && cnt < SLAB_D && row.idx[lo + cnt] >= (uint32_t)d0 &&
+             row.idx[lo + cnt] < (uint32_t)(d0 + dn))
+        ++cnt;
     }
     // (2) block-wide exclusive scan of the counts (fixed order)
     int incl = cnt;
@@ -253,7 +260,9 @@ __global__ void __launch_bounds__(SLAB_T) sc_apply_kernel(float* __restrict__ W,
         const int pos = base + e - win;
         if (pos >= 0 && pos < SLAB_CAP) {
           s_key[pos] = i * SLAB_D + ((int)row.idx[lo + e] - d0);
-          s_val[pos] = -eta * row.val[lo + e];
+          // an entry that breaks the ascending order is skipped, as in the forward pass
+          const bool skip = lo + e > 0 && row.idx[lo + e - 1] >= row.idx[lo + e];
+          s_val[pos] = skip ? 0.f : -eta * row.val[lo + e];
         }
       }
       __syncthreads();
@@ -312,7 +321,8 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
   const int ldt = (int)pad_to(J, 4);
   dim3 tg((D + 31) / 32, (ldt + 31) / 32);
   transpose_kernel<<<tg, 256, 0, s>>>(W, Wt, J, D, ldt);
-  dim3 grid(K, (ldt + 1023) / 1024);
+  const int cols = ldt > u.ld ? ldt : u.ld;   // pad columns of a wider u row are written (as zeros) too
+  dim3 grid(K, (cols + 1023) / 1024);
   sc_forward_kernel<<<grid, 256, 0, s>>>(Wt, ldt, codes, Xdata, u, K, J, D, dev_status);
   return cudaGetLastError() == cudaSuccess ? 2 : SFB_ERR_CUDA;
 }

@@ -28,7 +28,11 @@ struct CsrRow2 {
 __device__ __forceinline__ CsrRow2 csr_row2(const CsrView& c, int i) {
   CsrRow2 r;
   if (c.base == nullptr) {
-    const uint32_t s = c.rowptr[i], e = c.rowptr[i + 1];
+    uint32_t s = c.rowptr[i], e = c.rowptr[i + 1];
+    if (c.cap_p > 0) {   // what the worker's stream can hold: the same truncation as pack_csr
+      const uint32_t lim = c.rowptr[(size_t)(i / c.B) * c.B] + (uint32_t)c.cap_p;
+      s = min(s, lim); e = min(e, lim);
+    }
     r.idx = c.idx + s; r.val = c.val + s; r.len = (int)(e - s);
   } else {
     const int p = i / c.B, l = i % c.B;
@@ -42,15 +46,26 @@ __device__ __forceinline__ CsrRow2 csr_row2(const CsrView& c, int i) {
   return r;
 }
 
+// An entry counts only if its atom exists and the row is strictly ascending up to it: the rule of the forward
+// pass (sc_forward_kernel), so that forward and apply agree on malformed rows, and the reason why a
+// (chunk, atom) cell has at most one writer per sample in the fill below (no repeated atom inside a row).
+__device__ __forceinline__ bool entry_ok(const CsrRow2& row, int k, int D) {
+  const uint32_t d = row.idx[k];
+  return d < (uint32_t)D && !(k > 0 && row.idx[k - 1] >= d);
+}
+
 // cnt[chunk][d] += 1 for every nonzero (integer atomics: the final counts do not depend on the order)
-__global__ void __launch_bounds__(256) csc_count_kernel(CsrView codes, int K, int D, int* __restrict__ cnt) {
+__global__ void __launch_bounds__(256) csc_count_kernel(CsrView codes, int K, int D, int* __restrict__ cnt,
+                                                        int* dev_status) {
   const int i = blockIdx.x;
   const CsrRow2 row = csr_row2(codes, i);
   int* c = cnt + (size_t)(i / CSC_CHUNK) * D;
+  bool bad = false;
   for (int k = threadIdx.x; k < row.len; k += 256) {
-    const uint32_t d = row.idx[k];
-    if (d < (uint32_t)D) atomicAdd(c + d, 1);
+    if (entry_ok(row, k, D)) atomicAdd(c + row.idx[k], 1);
+    else bad = true;   // the entry is skipped
   }
+  if (bad && dev_status != nullptr) atomicOr(dev_status, SFB_DEV_BAD_INDEX);
 }
 
 // per atom: counts per chunk -> offsets of each chunk inside the column; column totals
@@ -119,8 +134,8 @@ __global__ void __launch_bounds__(256) csc_fill_kernel(CsrView codes, int K, int
     if (i < K) {
       const CsrRow2 row = csr_row2(codes, i);
       for (int k = threadIdx.x; k < row.len; k += 256) {
-        const uint32_t d = row.idx[k];
-        if (d < (uint32_t)D) {      // indices are unique inside a row: one writer per (chunk, atom) per step
+        if (entry_ok(row, k, D)) {  // indices that pass are unique inside a row: one writer per (chunk, atom) per step
+          const uint32_t d = row.idx[k];
           const int pos = colptr[d] + off[d];
           off[d] += 1;
           ent_i[pos] = i;
@@ -196,7 +211,9 @@ __global__ void __launch_bounds__(512) csc_apply_kernel(float* __restrict__ W, R
         if (beg >= stop && next_beg + lane < nnz) { pre_i = ent_i[next_beg + lane]; pre_a = ent_a[next_beg + lane]; }
         for (int base = beg; base < stop; base += 32) {
           const bool ok = base + lane < stop;
-          strip[lane] = make_int2(ok ? pre_i - i_lo : 0, __float_as_int(ok ? pre_a : 0.f));
+          // the sample index addresses shared memory: keep it inside the slice whatever the entry arrays hold
+          const int li = min(max(pre_i - i_lo, 0), i_n - 1);
+          strip[lane] = make_int2(ok ? li : 0, __float_as_int(ok ? pre_a : 0.f));
           const int nxt = (base + 32 < stop) ? base + 32 : next_beg;
           if (nxt + lane < nnz) { pre_i = ent_i[nxt + lane]; pre_a = ent_a[nxt + lane]; }
           __syncwarp();
@@ -270,11 +287,12 @@ CscScratch csc_scratch(void* workspace, int K, int D, long long nnz_capacity) {
 
 // Atom-major re-sort of the codes into the workspace.  Reads the codes only (not u), so it may run beside
 // the forward pass that produces u.
-int launch_sc_csc_build(cudaStream_t s, CsrView codes, int K, int D, long long nnz_capacity, void* workspace) {
+int launch_sc_csc_build(cudaStream_t s, CsrView codes, int K, int D, long long nnz_capacity, void* workspace,
+                        int* dev_status) {
   const int nchunks = (K + CSC_CHUNK - 1) / CSC_CHUNK;
   const CscScratch w = csc_scratch(workspace, K, D, nnz_capacity);
   if (cudaMemsetAsync(w.cnt, 0, (size_t)nchunks * D * 4, s) != cudaSuccess) return SFB_ERR_CUDA;
-  csc_count_kernel<<<K, 256, 0, s>>>(codes, K, D, w.cnt);
+  csc_count_kernel<<<K, 256, 0, s>>>(codes, K, D, w.cnt, dev_status);
   csc_chunk_offsets_kernel<<<(D + 255) / 256, 256, 0, s>>>(nchunks, D, w.cnt, w.total);
   csc_scan_kernel<<<1, 1024, 0, s>>>(D, w.total, w.colptr);
   csc_fill_kernel<<<nchunks, 256, 0, s>>>(codes, K, D, w.cnt, w.colptr, w.ent_i, w.ent_a);
@@ -307,7 +325,7 @@ int launch_sc_csc_apply(cudaStream_t s, float* W, RowMap u, int K, int J, int D,
 
 int launch_sc_apply_csc(cudaStream_t s, float* W, CsrView codes, RowMap u, int K, int J, int D, float eta,
                         long long nnz_capacity, void* workspace, const int* dev_status_ro) {
-  const int a = launch_sc_csc_build(s, codes, K, D, nnz_capacity, workspace);
+  const int a = launch_sc_csc_build(s, codes, K, D, nnz_capacity, workspace, const_cast<int*>(dev_status_ro));
   if (a < 0) return a;
   const int b2 = launch_sc_csc_apply(s, W, u, K, J, D, eta, nnz_capacity, workspace, dev_status_ro);
   return b2 < 0 ? b2 : a + b2;

@@ -23,12 +23,6 @@
 #include "umma.cuh"
 #include "umma_api.cuh"
 
-// The apply epilogue writes the new fp32 W with TMA bulk stores from its staging blocks (fewer store
-// instructions than per-thread 16-byte stores); -DSFB_LSU_STORE_W switches back to plain stores.
-#ifndef SFB_LSU_STORE_W
-#define SFB_TMA_STORE_W 1
-#endif
-
 namespace sfb {
 
 // extra passes implemented in finish.cu
@@ -146,11 +140,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (p.status_ro != nullptr && (*p.status_ro & SFB_DEV_BAD_HEADER)) return;   // uniform over the grid
-#ifdef SFB_EXP_CLOCKS
-  long long exp_c0 = clock64();
-  unsigned long long exp_t0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(exp_t0));
-#endif
 
   const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;   // 0 = the CTA that issues the MMAs
   const int cluster_id = blockIdx.x / CG, num_clusters = gridDim.x / CG;
@@ -187,9 +176,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int issued = 0;
     bool ok = true;
     const uint64_t pol_a = ptx::l2_policy(p.a_policy), pol_b = ptx::l2_policy(p.b_policy);
-#ifdef SFB_EXP_CLOCKS
-    long long exp_wait_empty = 0;
-#endif
     for (int work = cluster_id; work < total_work && ok; work += num_clusters) {
       const int tile = work / p.k_splits, split = work - tile * p.k_splits;
       const int kb_begin = split * p.k_per_split, kb_end = min(kb_begin + p.k_per_split, p.k_blocks);
@@ -204,13 +190,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       int row0 = 0, kp0 = 0;           // apply: first row / worker of the current reduction block
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-#ifdef SFB_EXP_CLOCKS
-        long long w0 = clock64();
-#endif
         ok = wait_or_abort(&ctl->empty[s], ph ^ 1u, ctl, p.status);
-#ifdef SFB_EXP_CLOCKS
-        exp_wait_empty += clock64() - w0;
-#endif
         if (!ok) break;
         if (lane == 0) {
           uint8_t* a_dst = tiles + s * STAGE_BYTES;
@@ -277,9 +257,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
-#ifdef SFB_EXP_CLOCKS
-    if (blockIdx.x == 0 && lane == 0) printf("EXPW apply=%d producer_wait_empty=%lld\n", (int)APPLY, exp_wait_empty);
-#endif
     if ((!ok || ctl->abort) && rank == 0) {
       // let copies already in flight land before the CTA goes away (bounded)
       int n = issued < STAGES ? issued : STAGES;
@@ -296,36 +273,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint32_t ph = 0;
     int it = 0;
     bool ok = (rank == 0);
-#ifdef SFB_EXP_CLOCKS
-    long long exp_wait_full = 0, exp_wait_tmem = 0;
-#endif
     for (int work = cluster_id; work < total_work && ok; work += num_clusters, ++it) {
       const int split = work % p.k_splits;
       const int kb_begin = split * p.k_per_split, kb_end = min(kb_begin + p.k_per_split, p.k_blocks);
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
-#ifdef SFB_EXP_CLOCKS
-      long long w1 = clock64();
-#endif
       ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
-#ifdef SFB_EXP_CLOCKS
-      exp_wait_tmem += clock64() - w1;
-#endif
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * BN;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-#ifdef SFB_EXP_CLOCKS
-        long long w2 = clock64();
-#endif
         ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
-#ifdef SFB_EXP_CLOCKS
-        exp_wait_full += clock64() - w2;
-#endif
         if (!ok) break;
-#ifndef SFB_EXP_NO_KLOOP_FENCE
         ptx::tc_fence_after();
-#endif
         if (lane == 0) {
           const uint32_t a_addr = ptx::smem_u32(tiles + s * STAGE_BYTES);
           const uint32_t b_addr = a_addr + A_STAGE_BYTES;
@@ -372,10 +332,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
-#ifdef SFB_EXP_CLOCKS
-    if (blockIdx.x == 0 && lane == 0)
-      printf("EXPW apply=%d mma_wait_full=%lld mma_wait_tmem_empty=%lld\n", (int)APPLY, exp_wait_full, exp_wait_tmem);
-#endif
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9, every CTA)
     // A warp may only read the TMEM lanes of its quarter (warp index mod 4).  Two warps share each
@@ -420,11 +376,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       float4 wv[8];
 #pragma unroll
       for (int g = 0; g < 8; ++g) wv[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-#ifdef SFB_EXP_SKIP_EPILOGUE_LOADS
-      if (APPLY && p.eta == 123.456f) {
-#else
       if (APPLY) {
-#endif
 #pragma unroll
         for (int g = 0; g < 8; ++g)
           if (rowp[g] != nullptr && cbase < ncols) wv[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + cbase));
@@ -509,11 +461,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float4 wn[8];   // next block of W, in flight while this block is combined and stored
 #pragma unroll
         for (int g = 0; g < 8; ++g) wn[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-#ifdef SFB_EXP_SKIP_EPILOGUE_LOADS
-        if (APPLY && cc + 1 < BN / 64 && p.eta == 123.456f) {
-#else
         if (APPLY && cc + 1 < BN / 64) {
-#endif
 #pragma unroll
           for (int g = 0; g < 8; ++g)
             if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
@@ -528,25 +476,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int g = 0; g < 8; ++g) {
           const int lr = 4 * g + lrow;
           const float4 a = *reinterpret_cast<const float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2));
-#ifdef SFB_EXP_SKIP_EPILOGUE_STORES
-          if (a.x == 123.456f && rowp[g] != nullptr && c < ncols) {
-#else
           if (rowp[g] != nullptr && c < ncols) {
-#endif
             if (APPLY) {
               float4 w = wv[g];
               w.x = fmaf(-p.eta, a.x, w.x); w.y = fmaf(-p.eta, a.y, w.y);
               w.z = fmaf(-p.eta, a.z, w.z); w.w = fmaf(-p.eta, a.w, w.w);
-#ifdef SFB_TMA_STORE_W
-              *reinterpret_cast<float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2)) = w;   // goes out by TMA below
-#elif !defined(SFB_EXP_SKIP_W_STORE)
-              __stcs(reinterpret_cast<float4*>(rowp[g] + c), w);   // streamed: keep L2 for the factors
-#endif
-#ifdef SFB_EXP_SKIP_SHADOW_STORE
-              if (p.shadow != nullptr && w.x == 123.456f) {
-#else
+              // the new fp32 W goes out by a TMA bulk store of the whole staging block (below): fewer store
+              // instructions than per-thread 16-byte stores
+              *reinterpret_cast<float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2)) = w;
               if (p.shadow != nullptr) {
-#endif
                 __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
                 uint2 pk;
                 pk.x = *reinterpret_cast<uint32_t*>(&lo);
@@ -560,7 +498,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
 #pragma unroll
         for (int g = 0; g < 8; ++g) wv[g] = wn[g];
-#ifdef SFB_TMA_STORE_W
         if (APPLY) {   // the 32 x 32 block of new W sits in the staging block, swizzled as the tensor map expects
           ptx::fence_proxy_async();
           __syncwarp();
@@ -570,7 +507,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ptx::tma_store_wait_read();   // the block is rewritten by the next pass
           }
         }
-#endif
         __syncwarp();
       }
       ptx::tc_fence_before();
@@ -582,17 +518,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   }
 
-#ifdef SFB_EXP_CLOCKS
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    unsigned long long exp_t1;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(exp_t1));
-    printf("EXPCLK apply=%d cycles=%lld ns=%llu MHz=%.0f\n", (int)APPLY, clock64() - exp_c0, exp_t1 - exp_t0,
-           1e3 * (double)(clock64() - exp_c0) / (double)(exp_t1 - exp_t0));
-  }
-#endif
-#ifdef SFB_TMA_STORE_W
   if (APPLY && warp >= 2 && lane == 0) ptx::tma_store_wait_all();
-#endif
   ptx::tc_fence_before();
   __syncthreads();
   if (CG == 2) ptx::cluster_sync();   // nobody leaves while its pair may still signal it or read its tiles
@@ -738,48 +664,38 @@ constexpr int MAX_SPLITS = 8;   // ranges a forward reduction may be cut into (p
 struct UmmaPlan {
   sfb_desc d;
   Layout l;
-  float* z_ws;
-  int ldz;
   int num_sms;
   int es;
-  bool pair_ok;   // CTA-pair kernels allowed (off with SFB_NO_CTA_PAIRS=1, for A/B measurements)
-  bool fold_ok;   // folded operand loads allowed (off with SFB_NO_FOLD=1)
-  int fold_ka;    // 128-byte atoms of the reduction index per stage in the folded kernels (SFB_FOLD_KA, default 2)
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
-  int fwd_group, apply_group;   // tile-order group widths (SFB_FWD_GROUP / SFB_APPLY_GROUP override the defaults)
   float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
   int ldp;
   // MLR: the factor v is a copy of x that nothing in the factor stage reads, so it runs on a side stream
-  // next to the forward GEMM (fork / join by events; SFB_NO_SIDE_COPY=1 keeps it on the main stream)
+  // next to the forward GEMM (fork / join by events)
   cudaStream_t side;
   cudaEvent_t fork, join;
   bool side_ok;
-  // SFB_TEST_LOSE_SIGNAL=1 at plan creation: the first GEMM launched through this plan loses one pipeline
-  // signal in its first CTA (pair), which must end in SFB_DEV_TIMEOUT after the bounded wait, not in a hang
+  // Test hook.  SFB_TEST_LOSE_SIGNAL=1 in the environment at plan creation: the first GEMM launched through this
+  // plan loses one pipeline signal in its first CTA (pair), which must end in SFB_DEV_TIMEOUT after the bounded
+  // wait, not in a hang.  The only environment variable the library reads.
   int lose_signal;
 };
 
-int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* /*w_shadow*/,
-                     UmmaPlan** out) {
+// Tile order: tiles of the fast dimension walked before the slow one advances.  Eight 256-wide column tiles keep
+// the slab of the smaller factor matrix (64 MB of V at 32768 x 8192, K = 4096, bf16) in L2 while the other streams.
+constexpr int FWD_GROUP = 8, APPLY_GROUP = 8;
+// 128-byte atoms of the reduction index per pipeline stage wherever three such stages fit in shared memory.
+constexpr int STAGE_ATOMS = 2;
+
+int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   if (get_encode() == nullptr) return SFB_ERR_CUDA;
   UmmaPlan* p = new UmmaPlan();
-  p->d = d; p->l = l; p->z_ws = z_ws; p->ldz = ldz;
+  p->d = d; p->l = l;
   p->es = (d.path == SFB_PATH_BF16) ? 2 : 4;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev);
-  const char* no_pairs = getenv("SFB_NO_CTA_PAIRS");
-  p->pair_ok = !(no_pairs != nullptr && no_pairs[0] == '1');
-  const char* no_fold = getenv("SFB_NO_FOLD");
-  p->fold_ok = !(no_fold != nullptr && no_fold[0] == '1');
-  const char* ka = getenv("SFB_FOLD_KA");
-  p->fold_ka = (ka != nullptr && ka[0] == '1') ? 1 : 2;
   const char* ls = getenv("SFB_TEST_LOSE_SIGNAL");
   p->lose_signal = (ls != nullptr && ls[0] == '1') ? 1 : 0;
-  const char* fg = getenv("SFB_FWD_GROUP");
-  const char* ag = getenv("SFB_APPLY_GROUP");
-  p->fwd_group = fg != nullptr ? atoi(fg) : 8;
-  p->apply_group = ag != nullptr ? atoi(ag) : 8;
   p->part_ws = nullptr;
   p->ldp = (int)pad_to(d.J, 4);
   {   // forward GEMMs whose 128 x 128 tiles do not fill the SMs may split their reduction
@@ -793,8 +709,7 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, _
   }
   p->side_ok = false;
   {
-    const char* ns = getenv("SFB_NO_SIDE_COPY");
-    if (d.model == SFB_MLR && !(ns != nullptr && ns[0] == '1')) {
+    if (d.model == SFB_MLR) {
       p->side_ok = cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking) == cudaSuccess;
       if (p->side_ok) {
         const bool e1 = cudaEventCreateWithFlags(&p->fork, cudaEventDisableTiming) == cudaSuccess;
@@ -844,9 +759,9 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
   if (splits != nullptr) *splits = 1;
   v.bn = (N > 128 && (long long)m_units * ((N + 255) / 256) >= pl->num_sms) ? 256 : 128;
   // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
-  v.cg = (v.bn == 256 && pl->pair_ok && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
+  v.cg = (v.bn == 256 && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
   if (v.cg == 1 && k_atoms > 0) {
-    const int k_blocks = (k_atoms + pl->fold_ka - 1) / pl->fold_ka;
+    const int k_blocks = (k_atoms + STAGE_ATOMS - 1) / STAGE_ATOMS;
     auto ranges = [&](long long tiles, int slots) {
       long long ks = slots / (tiles > 0 ? tiles : 1);
       if (ks > max_splits) ks = max_splits;
@@ -859,7 +774,7 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
     const int ks_one = ranges(t_one, pl->num_sms);
     // pairs that fill three quarters of the machine beat single tiles that fill all of it: the single
     // 128 x 128 tiles are bound by the operand feed (about 50 % tensor-pipe activity with fp32 operands)
-    if (pl->pair_ok && N > 128 && m_units >= 2 && 4 * t_pair * ks_pair >= 3 * (pl->num_sms / 2)) {
+    if (N > 128 && m_units >= 2 && 4 * t_pair * ks_pair >= 3 * (pl->num_sms / 2)) {
       v.bn = 256; v.cg = 2;
       if (splits != nullptr) *splits = ks_pair;
     } else if (t_one < pl->num_sms && splits != nullptr && max_splits > 1) {
@@ -867,10 +782,10 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
       *splits = ks_one;
     }
   }
-  v.fold = v.cg == 2 && pl->fold_ok && dims_chunk_aligned;
+  v.fold = v.cg == 2 && dims_chunk_aligned;
   // two 128-byte atoms of reduction per stage wherever three such stages fit in shared memory: the
   // per-stage barrier round trip, not the number of TMA instructions, is what costs
-  v.ka = (v.cg == 2 || v.bn == 128) ? pl->fold_ka : 1;
+  v.ka = (v.cg == 2 || v.bn == 128) ? STAGE_ATOMS : 1;
   return v;
 }
 
@@ -906,7 +821,7 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.m_fastest = ((long long)d.J * d.D > (long long)P * d.B * d.D) ? 1 : 0;
   p.a_policy = p.m_fastest ? 2 : 0;   // the operand whose slab changes every tile is re-read all along: keep it
   p.b_policy = p.m_fastest ? 0 : 2;
-  p.group = pl->fwd_group;
+  p.group = FWD_GROUP;
   p.z = z;
   p.status = dev_status;
   p.lose_signal = pl->lose_signal;
@@ -928,7 +843,7 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
-                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status, int workers) {
+                 const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers) {
   const sfb_desc& d = pl->d;
   const int K = (workers > 0 ? workers : d.P) * d.B;
   int launches = 0, r;
@@ -942,45 +857,57 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     if (v.base != nullptr && pl->side_ok) {   // v = x on the side stream, joined before this call returns its work
       if (cudaEventRecord(pl->fork, s) != cudaSuccess || cudaStreamWaitEvent(pl->side, pl->fork, 0) != cudaSuccess)
         return SFB_ERR_CUDA;
-      if ((r = launch_copy_rows(pl->side, x_rows, v, K, d.D)) < 0) return r;
-      launches += r;
-      if (cudaEventRecord(pl->join, pl->side) != cudaSuccess) return SFB_ERR_CUDA;
       forked = true;
     }
-    auto finish_v = [&]() -> int {
-      if (forked) return cudaStreamWaitEvent(s, pl->join, 0) == cudaSuccess ? 0 : SFB_ERR_CUDA;
-      if (v.base == nullptr) return 0;
-      return launch_copy_rows(s, x_rows, v, K, d.D);
+    // Once forked, every exit (errors included) makes `s` wait for the side stream, so the caller's stream
+    // never runs ahead of the copy and a stream capture in progress stays well formed.
+    auto join_side = [&]() -> int {
+      if (!forked) return 0;
+      if (cudaEventRecord(pl->join, pl->side) != cudaSuccess || cudaStreamWaitEvent(s, pl->join, 0) != cudaSuccess)
+        return SFB_ERR_CUDA;
+      return 0;
     };
-    RowMap zz = bf16 ? z : u;   // fp32 products: workspace when u is bf16, else u itself (finished in place)
-    // the GEMM epilogue leaves exp(z - local max) in u and (max, sum) per half tile; the finishing
-    // pass rescales to the softmax and subtracts the one-hot label, in place
-    if (pl->part_ws != nullptr) {
-      // few tiles: split reduction into the partial buffers, then the plain softmax pass sums them
-      RowMap pz;
-      pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
-      pz.worker_stride = (long long)d.B * pl->ldp * 4;
-      const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
-      int ks = 1;
-      if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr, nullptr,
-                                 &ks, MAX_SPLITS, sstride, workers)) < 0)
-        return r;
-      launches += r;
-      if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
-      launches += r;
-      if ((r = finish_v()) < 0) return r;
-      return launches + r;
-    }
-    int n_parts = 0, part_cols = 0;
-    (void)zz;
-    if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
-                               &part_cols, nullptr, 1, 0, workers)) < 0)
-      return r;
-    launches += r;
-    if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status)) < 0) return r;
-    launches += r;
-    if ((r = finish_v()) < 0) return r;
-    return launches + r;
+    auto body = [&]() -> int {
+      if (forked) {
+        if ((r = launch_copy_rows(pl->side, x_rows, v, K, d.D)) < 0) return r;
+        launches += r;
+      }
+      // the GEMM epilogue leaves exp(z - local max) in u and (max, sum) per half tile; the finishing
+      // pass rescales to the softmax and subtracts the one-hot label, in place
+      if (pl->part_ws != nullptr) {
+        // few tiles: split reduction into the partial buffers, then the plain softmax pass sums them
+        RowMap pz;
+        pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
+        pz.worker_stride = (long long)d.B * pl->ldp * 4;
+        const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
+        int ks = 1;
+        if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr,
+                                   nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
+          return r;
+        launches += r;
+        if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
+        launches += r;
+      } else {
+        int n_parts = 0, part_cols = 0;
+        if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
+                                   &part_cols, nullptr, 1, 0, workers)) < 0)
+          return r;
+        launches += r;
+        if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status)) < 0)
+          return r;
+        launches += r;
+      }
+      if (!forked && v.base != nullptr) {
+        if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
+        launches += r;
+      }
+      return 0;
+    };
+    const int rb = body();
+    const int rj = join_side();
+    if (rb < 0) return rb;
+    if (rj < 0) return rj;
+    return launches;
   }
   // DML (TF32): the pair differences are the factor v and the GEMM operand
   if (v.base == nullptr) return SFB_ERR_ARG;
@@ -1030,7 +957,7 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
   p.a_policy = p.m_fastest ? 2 : 0;
   p.b_policy = p.m_fastest ? 0 : 2;
-  p.group = pl->apply_group;
+  p.group = APPLY_GROUP;
   p.W = reinterpret_cast<float*>(W);
   p.shadow = (d.path == SFB_PATH_BF16) ? w_shadow : nullptr;
   p.ldw = d.D;

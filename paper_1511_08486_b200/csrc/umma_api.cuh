@@ -7,15 +7,14 @@ namespace sfb {
 
 struct UmmaPlan;   // tensor maps and launch geometry for one descriptor
 
-// Builds the plan for a TF32 or BF16 descriptor.  z_ws: fp32 [K][ldz] product workspace;
-// w_shadow: bf16 copy of W (BF16 path) or nullptr.
-int umma_plan_create(const sfb_desc& d, const Layout& l, float* z_ws, int ldz, __nv_bfloat16* w_shadow, UmmaPlan** out);
+// Builds the plan for a TF32 or BF16 descriptor.
+int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out);
 void umma_plan_destroy(UmmaPlan* p);
 
 // z = W a on the tensor cores followed by the model epilogue; factors go through u / v row maps.
 // workers > 0: only that many workers' samples (X, aux, u, v start at the first of them).
 int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
-                 const sfb_aux* aux, RowMap u, RowMap v, RowMap z, int* dev_status, int workers = 0);
+                 const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers = 0);
 
 // Z rows (fp32) = A rows (the path's value type) times Wop^T on the tensor cores; no epilogue beyond the store.
 int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,

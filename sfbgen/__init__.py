@@ -14,6 +14,7 @@ alone and in any order.
 from .configs import CONFIGS, scaled, get_config
 from .generate import (
     make_inputs,
+    batch_of,
     bf16_round_bits,
     bf16_bits_to_f32,
     philox,
@@ -24,6 +25,7 @@ __all__ = [
     "scaled",
     "get_config",
     "make_inputs",
+    "batch_of",
     "bf16_round_bits",
     "bf16_bits_to_f32",
     "philox",

@@ -149,3 +149,13 @@ def make_inputs(cfg: dict) -> dict:
     if model == "sc":
         return _make_sc(cfg)
     raise ValueError(f"unknown model {model!r}")
+
+
+def batch_of(inputs: dict, cfg: dict, b: int = 0) -> dict:
+    """Minibatch b of `inputs` as the keyword arrays one step consumes (views of the generated tensors, no arithmetic)."""
+    m = cfg["model"]
+    if m == "mlr":
+        return dict(X=inputs["X"][b], labels=inputs["labels"][b])
+    if m == "dml":
+        return dict(Xa=inputs["Xa"][b], Xb=inputs["Xb"][b], similar=inputs["similar"])
+    return dict(rowptr=inputs["rowptr"][b], idx=inputs["idx"][b], val=inputs["val"][b], Xdata=inputs["Xdata"][b])

@@ -191,3 +191,37 @@ def test_dml_step_leaves_out_inactive_pairs_bit_identically():
         assert torch.equal(wl.W, W_part)
     finally:
         wl.close()
+
+
+def test_bf16_two_classes_step_size_and_the_rounding_contract():
+    """MLR with J = 2, D = 760, K = 260 on the bf16 path, the one shape a randomised sweep found above 1e-2
+    (1.1e-2 after two steps with eta = 0.3, i.e. eta * |x|^2 = 228: the first step throws the logits of the
+    second to +-300).  The cause is the path's contract, not its kernels: W enters the forward pass rounded to
+    bf16 and u goes on the wire in bf16, and a softmax at |z| ~ 300 amplifies those roundings.  Checked both ways:
+    (a) with a step ten times smaller the same shape is inside the stated tolerance against the plain oracle;
+    (b) at eta = 0.3 the GPU agrees to 1e-3 with the oracle run on operands rounded the way the contract says
+        (bf16 W for the forward, bf16 u for the update, fp32 storage of W between steps)."""
+    from sfbgen import bf16_bits_to_f32, bf16_round_bits
+    cfg = scaled("C4", J=2, D=760, P=2, B=130, pool=1, labels="uniform")
+    cfg["path"] = "bf16"
+    check_config(cfg, "bf16", eta=0.03, steps=2)
+    inputs = make_inputs(cfg)
+    X, y = bf16_bits_to_f32(inputs["X_bits"][0]), inputs["labels"][0]
+    rb = lambda a: bf16_bits_to_f32(bf16_round_bits(np.ascontiguousarray(a, dtype=np.float32)))
+    eta = 0.3
+    W = inputs["W"].astype(np.float32)
+    for _ in range(2):
+        U, V = orc.mlr_factors(rb(W), X, y)
+        W = orc.apply_dense(W, rb(U.astype(np.float32)), V, eta).astype(np.float32)
+    wl = _workload(cfg, inputs, "bf16")
+    try:
+        for t in range(2):
+            wl.step(t, eta=eta)
+        torch.cuda.synchronize()
+        assert wl.ctx.status() == 0
+        W0 = inputs["W"].astype(np.float64)
+        got, want = to_f64(wl.W) - W0, W.astype(np.float64) - W0
+        err = np.linalg.norm(got - want) / np.linalg.norm(want)
+        assert err <= 1e-3, f"{err:.3e} against the oracle on contract-rounded operands"
+    finally:
+        wl.close()

@@ -10,7 +10,8 @@ import torch
 
 from oracle import sfb_oracle as orc
 from sfbgen import get_config, make_inputs, scaled
-from tests.util import MODEL_ID, TOL, batch_of, dml_accept_gate, oracle_apply, oracle_factors, to_f64
+from tests.util import (MAX_STORAGE_OVER_TOL, MODEL_ID, TOL, assert_lines, batch_of, dml_accept_gate, oracle_apply,
+                        oracle_factors, to_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -48,6 +49,7 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
         U_ref = dml_accept_gate(cfg, U_gpu, U_or, extra, path) if cfg["model"] == "dml" else U_or
         e_u = orc.rel_fro(U_gpu, U_ref)
         assert e_u <= tol, f"E_U = {e_u:.3e} > {tol}"
+        assert_lines(U_gpu, U_ref, tol, "U")                 # no single sample's u, no single class, is far off
         if cfg["model"] != "sc":
             V_gpu = to_f64(wl.V)
             assert not V_gpu[:, D:].any(), "pad columns of V must be zero"
@@ -72,6 +74,7 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
             dW_or = orc.delta_w(U_gpu, V_or)
         e_dw = orc.rel_fro(dW_gpu, dW_or)
         assert e_dw <= tol, f"E_dW = {e_dw:.3e} > {tol}"
+        assert_lines(dW_gpu, dW_or, tol, "U^T V")            # no row, no column of the update is far off
         # partial apply: only the first worker's stream
         if cfg["P"] > 1:
             wl.W.zero_()
@@ -85,6 +88,7 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
             else:
                 ref1 = orc.delta_w(U_gpu[:Bn], V_or[:Bn])
             assert orc.rel_fro(to_f64(wl.W), ref1) <= tol
+            assert_lines(to_f64(wl.W), ref1, tol, "U^T V of the first worker")
         # ---- steps: W_T - W_0 against the oracle's trajectory ----------------------------------------
         W_or = W0.astype(np.float64)
         for t in range(steps):
@@ -118,15 +122,26 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
                 ref_move = -eta * orc.delta_w(U_fix, V_o)
                 got_move = wl.W.cpu().numpy().astype(np.float64) - W_t.astype(np.float64)
                 storage = 2.0 ** -24 * np.linalg.norm(W_t) / np.linalg.norm(ref_move)
+                assert storage <= MAX_STORAGE_OVER_TOL * tol, f"storage term {storage:.1e} swamps the tolerance: raise eta"
                 e_t = np.linalg.norm(got_move - ref_move) / np.linalg.norm(ref_move)
                 assert e_t <= tol + storage, f"step {t}: E_step = {e_t:.3e} > {tol} + {storage:.1e}"
+                W_t64 = W_t.astype(np.float64)
+                assert_lines(got_move, ref_move, tol, f"step {t}: W' - W",
+                             extra_rows=2.0 ** -24 * np.linalg.norm(W_t64, axis=1),
+                             extra_cols=2.0 ** -24 * np.linalg.norm(W_t64, axis=0))
                 e_step = max(e_step, e_t)
         else:
             moved = np.linalg.norm(W_or - W0)
             e_step = np.linalg.norm((W_gpu - W0) - (W_or - W0)) / moved
-            # W is stored in fp32: its storage rounding (2^-24 per element, relative) is not the kernel's error
-            storage = steps * 2.0 ** -24 * np.linalg.norm(W0) / moved
+            # W is stored in fp32: every step rounds it once (at most 2^-24 relative per element, independent from
+            # step to step, so T roundings add up like sqrt(T)); that is not the kernel's error
+            storage = np.sqrt(steps) * 2.0 ** -24 * np.linalg.norm(W0) / moved
+            assert storage <= MAX_STORAGE_OVER_TOL * tol, f"storage term {storage:.1e} swamps the tolerance: raise eta"
             assert e_step <= tol + storage, f"E_step = {e_step:.3e} > {tol} + {storage:.1e}"
+            W064 = W0.astype(np.float64)
+            assert_lines(W_gpu - W064, W_or - W064, tol, "W_T - W_0",
+                         extra_rows=np.sqrt(steps) * 2.0 ** -24 * np.linalg.norm(W064, axis=1),
+                         extra_cols=np.sqrt(steps) * 2.0 ** -24 * np.linalg.norm(W064, axis=0))
         # the buffer left by the last step is a valid serialisation with the step's clock
         h, U_last, _ = orc.unpack(runs[0][1])
         assert h["clock"] == steps - 1 and h["P"] == cfg["P"] and h["J"] == J
@@ -258,6 +273,95 @@ def test_sparse_bad_index_sets_status():
         wl.batches[0]["idx"][0] = 1000
         wl.compute_factors(0)
         assert wl.ctx.status() & B.SFB_DEV_BAD_INDEX
+    finally:
+        wl.close()
+
+
+def test_sparse_repeated_and_unsorted_indices_are_skipped_everywhere():
+    """A CSR row that repeats an atom or is not ascending: the offending entries are skipped by the forward pass,
+    by the atom-major re-sort and by the scatter apply alike (status bit set, nothing out of range is touched),
+    so the step equals the oracle's step on the codes with those entries removed."""
+    from paper_1511_08486_b200 import binding as B
+    cfg = scaled("C3", J=96, D=120, P=2, B=8, density=0.15)
+    inputs = make_inputs(cfg)
+    rp = inputs["rowptr"][0].astype(np.int64)
+    ix, vl = inputs["idx"][0].copy(), inputs["val"][0].copy()
+    # sample 3: repeat an atom (entry 2 takes the index of entry 1); sample 9: an entry out of order (smaller than its
+    # predecessor); sample 12: an atom that does not exist (which also puts its successor out of order)
+    for i, k, new in ((3, 2, None), (9, 4, 0), (12, 1, 100000)):
+        s0 = rp[i]
+        assert rp[i + 1] - s0 > 6
+        ix[s0 + k] = ix[s0 + k - 1] if new is None else new
+    # the documented rule: an entry is dropped if its atom is out of range or not above its predecessor in the row
+    keep = np.ones(ix.size, bool)
+    for i in range(cfg["K"]):
+        for k in range(rp[i], rp[i + 1]):
+            if ix[k] >= cfg["D"] or (k > rp[i] and ix[k - 1] >= ix[k]):
+                keep[k] = False
+    assert (~keep).sum() == 4
+    inputs["idx"][0] = ix
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        eta = 1e-2
+        wl.step(0, eta=eta)
+        status = wl.ctx.status()
+        assert status & B.SFB_DEV_BAD_INDEX
+        W1 = wl.W.cpu().numpy().astype(np.float64)
+        assert np.isfinite(W1).all()
+        counts = np.array([keep[rp[i]:rp[i + 1]].sum() for i in range(cfg["K"])])
+        rp_ok = np.concatenate([[0], np.cumsum(counts)]).astype(np.uint32)
+        W_or, U_or, _ = orc.step(orc.MODEL_SC, inputs["W"], dict(rowptr=rp_ok, idx=ix[keep], val=vl[keep],
+                                                                  Xdata=inputs["Xdata"][0]), eta)
+        W0 = inputs["W"].astype(np.float64)
+        err = np.linalg.norm((W1 - W0) - (W_or - W0)) / np.linalg.norm(W_or - W0)
+        assert err <= 1e-5 + 2.0 ** -24 * np.linalg.norm(W0) / np.linalg.norm(W_or - W0), f"{err:.3e}"
+        _, U_wire, _ = orc.unpack(wl.sf_buf.cpu().numpy())
+        assert orc.rel_fro(U_wire, U_or) <= 1e-5
+        # the staged calls (factors, pack, apply: the re-sort then reads the buffer's streams) agree bit for bit
+        wl.reset()
+        wl.compute_factors(0)
+        wl.pack(0, clock=0)
+        wl.apply(eta)
+        assert wl.ctx.status() & B.SFB_DEV_BAD_INDEX
+        assert np.array_equal(wl.W.cpu().numpy().astype(np.float64), W1)
+    finally:
+        wl.close()
+
+
+def test_sparse_capacity_overflow_keeps_factors_and_wire_consistent():
+    """Codes beyond a worker's capacity are cut off (status bit): the u the step computes, the codes on the wire and
+    the codes the apply uses are the same truncated ones, so the step equals the oracle's step on them."""
+    from paper_1511_08486_b200 import binding as B
+    cfg = scaled("C3", J=64, D=200, P=2, B=4, density=0.2)
+    inputs = make_inputs(cfg)
+    cap_p = 96
+    inputs["nnz_capacity"] = cap_p * cfg["P"]
+    rp = inputs["rowptr"][0].astype(np.int64)
+    ix, vl = inputs["idx"][0], inputs["val"][0]
+    assert rp[cfg["B"]] - rp[0] > cap_p                     # worker 0 overflows
+    wl = _workload(cfg, inputs, "f32")
+    try:
+        eta = 1e-2
+        wl.step(0, eta=eta)
+        assert wl.ctx.status() & B.SFB_DEV_CAPACITY
+        keep = np.zeros(ix.size, bool)
+        counts = np.zeros(cfg["K"], np.int64)
+        for p in range(cfg["P"]):
+            base = rp[p * cfg["B"]]
+            for i in range(p * cfg["B"], (p + 1) * cfg["B"]):
+                s0, e0 = min(rp[i], base + cap_p), min(rp[i + 1], base + cap_p)
+                keep[s0:e0] = True
+                counts[i] = e0 - s0
+        rp_t = np.concatenate([[0], np.cumsum(counts)]).astype(np.uint32)
+        W_or, U_or, _ = orc.step(orc.MODEL_SC, inputs["W"], dict(rowptr=rp_t, idx=ix[keep], val=vl[keep],
+                                                                  Xdata=inputs["Xdata"][0]), eta)
+        W0 = inputs["W"].astype(np.float64)
+        W1 = wl.W.cpu().numpy().astype(np.float64)
+        err = np.linalg.norm((W1 - W0) - (W_or - W0)) / np.linalg.norm(W_or - W0)
+        assert err <= 1e-5 + 2.0 ** -24 * np.linalg.norm(W0) / np.linalg.norm(W_or - W0), f"{err:.3e}"
+        _, U_wire, (rp_w, ix_w, _) = orc.unpack(wl.sf_buf.cpu().numpy())
+        assert np.array_equal(rp_w, rp_t) and np.array_equal(ix_w, ix[keep])
+        assert orc.rel_fro(U_wire, U_or) <= 1e-5
     finally:
         wl.close()
 

@@ -104,3 +104,11 @@ def test_many_workers_and_long_reductions():
     update), and 256 workers x 64 pairs on the tf32 path (reduction blocks that span two workers)."""
     check_config(_cfg("C4", "bf16", J=256, D=256, P=256, B=256, pool=1, labels="uniform"), "bf16", eta=1e-3, steps=1)
     check_config(_cfg("C2", "tf32", J=128, D=256, P=256, B=64), "tf32", eta=1e-6, steps=1)
+
+
+def test_bf16_c4_full_fifty_steps():
+    """The workload's own schedule at full size: 50 steps over the pool of 4 minibatches (32768 x 8192, K = 4096,
+    Zipf labels), free-running against the oracle's fp64 trajectory; the error is taken on W_50 - W_0, whole
+    matrix, every row and every column.  (The oracle needs a few seconds per step.)"""
+    cfg = get_config("C4")
+    check_config(cfg, "bf16", eta=cfg["eta"], steps=cfg["steps"])

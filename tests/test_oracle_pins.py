@@ -413,3 +413,24 @@ def test_losses_closed_forms():
     Xd = (A @ W.T.astype(np.float64)).astype(np.float32)
     assert orc.sc_loss(W, rowptr, idx, val, Xd) == 0.0
     assert abs(orc.sc_loss(np.zeros_like(W), rowptr, idx, val, Xd) - 0.5 * float((Xd.astype(np.float64) ** 2).sum())) <= 1e-9
+
+
+# ----------------------------------------------------------------------------- parity metric
+def test_rel_fro_hand_values():
+    """The metric every GPU tolerance rests on: ||a - b||_F / ||b||_F with b the reference, by hand."""
+    # a - b = (3, -1): norm sqrt(10); ||b|| = 5
+    assert orc.rel_fro([3.0, 4.0], [0.0, 5.0]) == pytest.approx(math.sqrt(10.0) / 5.0, rel=1e-15)
+    # not symmetric: the denominator is the SECOND argument's norm
+    assert orc.rel_fro([1.0, 0.0], [0.0, 2.0]) == pytest.approx(math.sqrt(5.0) / 2.0, rel=1e-15)
+    assert orc.rel_fro([0.0, 2.0], [1.0, 0.0]) == pytest.approx(math.sqrt(5.0), rel=1e-15)
+    # a square root is taken (not the ratio of squared norms), and the norm runs over all entries of a matrix
+    a = [[1.0, 2.0], [3.0, 4.0]]
+    b = [[1.0, 2.0], [3.0, 0.0]]
+    assert orc.rel_fro(a, b) == pytest.approx(4.0 / math.sqrt(14.0), rel=1e-15)
+    # scale invariance and the 1e-k reading used by the tolerances
+    assert orc.rel_fro([1.0 + 1e-5, 1.0], [1.0, 1.0]) == pytest.approx(1e-5 / math.sqrt(2.0), rel=1e-9)
+    # zero reference: the absolute norm of the difference
+    assert orc.rel_fro([3.0, 4.0], [0.0, 0.0]) == 5.0
+    assert orc.rel_fro([0.0, 0.0], [0.0, 0.0]) == 0.0
+    # float32 inputs are promoted, not compared in fp32
+    assert orc.rel_fro(np.float32([1.0]), np.float64([1.0 + 1e-12])) == pytest.approx(1e-12, rel=1e-3)
