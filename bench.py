@@ -236,8 +236,9 @@ def whole_job_throughput(units_per_rank_step, steps, ms, world):
 
 
 def workload_name(cfg, path):
+    dens = f" density={cfg['density']}" if cfg["model"] == "sc" else ""
     return (f"{cfg['name']} {cfg['model'].upper()} J={cfg['J']} D={cfg['D']} P={cfg['P']} B={cfg['B']} "
-            f"K={cfg['K']} path={path}")
+            f"K={cfg['K']}{dens} path={path}")
 
 
 def run_bsp(args, cfg, inputs, wl, path, rank, world, local_rank, barrier):
@@ -375,6 +376,8 @@ def main():
                          "over the ranks with an all-gather of the worker streams per step (sufficient factor broadcasting)")
     for dim in ("J", "D", "P", "B"):
         ap.add_argument(f"--{dim}", type=int, default=None, help=f"override {dim} (smaller cases for profiler captures)")
+    ap.add_argument("--density", type=float, default=None,
+                    help="sparse coding: fraction of nonzeros in the codes (default: the configuration's 5 %%)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -384,6 +387,8 @@ def main():
     from sfbgen import get_config, make_inputs
     cfg = get_config(args.config)
     over = {k: getattr(args, k) for k in ("J", "D", "P", "B") if getattr(args, k) is not None}
+    if args.density is not None:
+        over["density"] = args.density
     if over:
         from sfbgen import scaled
         cfg = scaled(args.config, **over)

@@ -226,16 +226,55 @@ def sf_layout(model, dtype, J, D, P, B, v_sparse=False, nnz_capacity=0):
                 total_bytes=streams_off + P * stream_stride)
 
 
-def pack(model, dtype, J, D, P, B, U, V=None, csr=None, clock=0, nnz_capacity=0):
+FLAG_V_SPARSE, FLAG_COMPACT = 1, 2
+
+
+def _wire_round(mat, dtype):
+    """Values as they sit on the wire (fp32, or bf16 round-to-nearest-even), returned as fp32."""
+    m32 = np.asarray(mat, dtype=np.float64).astype(np.float32)
+    if dtype == DTYPE_F32:
+        return m32
+    return (_bf16_bits(m32).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def compact_pairs(U, V, P, B):
+    """Inactive-pair compaction (Section 6.1: the sufficient factors are sparse and that is used).
+
+    A pair whose u is all zeros (a dissimilar DML pair beyond the margin) contributes u v^T = 0, so a worker need
+    not send it.  Per worker, the pairs with a nonzero u move to the front of the worker's B slots in their original
+    order; the slots behind them are zero.  Returns (U_c, V_c, n_sf) with n_sf[p] the number of pairs kept.
+    """
+    U, V = np.asarray(U), np.asarray(V)
+    Uc, Vc = np.zeros_like(U), np.zeros_like(V)
+    n_sf = []
+    for p in range(P):
+        rows = [i for i in range(p * B, (p + 1) * B) if np.any(U[i] != 0)]
+        for k, i in enumerate(rows):
+            Uc[p * B + k] = U[i]
+            Vc[p * B + k] = V[i]
+        n_sf.append(len(rows))
+    return Uc, Vc, n_sf
+
+
+def pack(model, dtype, J, D, P, B, U, V=None, csr=None, clock=0, nnz_capacity=0, compact=False):
     """Serialise K = P*B (u, v) pairs as P worker streams.  Returns a uint8 array.
 
     U: [K][J] values (rounded here to the wire dtype, round to nearest even).
     V: [K][D] values for dense v; csr = (rowptr[K+1], idx, val) for sparse v.
+    compact (dense v only): pairs whose wire u is all zeros are left out as `compact_pairs` describes; the
+    directory then carries each worker's own pair count and header flag bit 1 is set.  The slot layout (offsets,
+    strides) is unchanged, so a receiver reads the first n_sf rows of a worker's U and V blocks.
     """
     v_sparse = csr is not None
     lay = sf_layout(model, dtype, J, D, P, B, v_sparse, nnz_capacity)
     buf = np.zeros(lay["total_bytes"], dtype=np.uint8)
-    flags = 1 if v_sparse else 0
+    flags = FLAG_V_SPARSE if v_sparse else 0
+    n_sf = [B] * P
+    if compact:
+        if v_sparse:
+            raise ValueError("compaction is defined for dense v")
+        U, V, n_sf = compact_pairs(_wire_round(U, dtype), _wire_round(V, dtype), P, B)
+        flags |= FLAG_COMPACT
     hdr = struct.pack("<IHBBIIIIIIIIQQQI", MAGIC, VERSION, model, dtype, flags, P, B, J, D, clock,
                       lay["ldu"], lay["ldv"], lay["stream_stride"], lay["total_bytes"],
                       lay["streams_off"], lay["cap_p"])
@@ -270,7 +309,7 @@ def pack(model, dtype, J, D, P, B, U, V=None, csr=None, clock=0, nnz_capacity=0)
             buf[vo:vo + vb.size * lay["es"]] = vb.view(np.uint8)
         else:
             put_vals(v_off, B, lay["ldv"], np.asarray(V)[p * B:(p + 1) * B])
-        ent = struct.pack("<IIIIQQ", p, B, clock, nnz_p, u_off, v_off)
+        ent = struct.pack("<IIIIQQ", p, n_sf[p], clock, nnz_p, u_off, v_off)
         d_off = HEADER_BYTES + p * DIR_ENTRY_BYTES
         buf[d_off:d_off + DIR_ENTRY_BYTES] = np.frombuffer(ent, dtype=np.uint8)
     return buf
@@ -283,9 +322,31 @@ def parse_header(buf):
     return dict(zip(names, f))
 
 
-def unpack(buf):
-    """Inverse of `pack`: returns header dict, U [K][J] fp32, and V [K][D] fp32 or CSR (rowptr, idx, val)."""
+def wire_bytes(buf):
+    """Bytes a broadcast of this buffer carries (Section 5.1 counts these per worker pair): header, directory, and
+    per worker its first n_sf rows of U and of dense V, or all B rows of U plus row pointers and nnz (index, value)
+    pairs for sparse v.  Padding is not sent."""
     h = parse_header(buf)
+    P, B, J, D = h["P"], h["B"], h["J"], h["D"]
+    es = 4 if h["dtype"] == DTYPE_F32 else 2
+    total = HEADER_BYTES + P * DIR_ENTRY_BYTES
+    for p in range(P):
+        _, n_sf, _, nnz_p, _, _ = struct.unpack_from(
+            "<IIIIQQ", bytes(buf[HEADER_BYTES + p * DIR_ENTRY_BYTES:HEADER_BYTES + (p + 1) * DIR_ENTRY_BYTES]))
+        if h["flags"] & FLAG_V_SPARSE:
+            total += n_sf * J * es + (B + 1) * 4 + nnz_p * (4 + es)
+        else:
+            total += n_sf * (J + D) * es
+    return total
+
+
+def unpack(buf):
+    """Inverse of `pack`: returns header dict, U [K][J] fp32, and V [K][D] fp32 or CSR (rowptr, idx, val).
+
+    The header dict also carries "n_sf", the per-worker pair counts of the directory (all B unless the buffer is
+    compacted; the rows behind a worker's n_sf are returned as stored, i.e. zeros)."""
+    h = parse_header(buf)
+    h["n_sf"] = []
     P, B, J, D = h["P"], h["B"], h["J"], h["D"]
     lay = sf_layout(h["model"], h["dtype"], J, D, P, B, bool(h["flags"] & 1), h["cap_p"] * P)
     es = lay["es"]
@@ -304,6 +365,7 @@ def unpack(buf):
     for p in range(P):
         wid, n_sf, clk, nnz_p, u_off, v_off = struct.unpack_from(
             "<IIIIQQ", bytes(buf[HEADER_BYTES + p * DIR_ENTRY_BYTES:HEADER_BYTES + (p + 1) * DIR_ENTRY_BYTES]))
+        h["n_sf"].append(n_sf)
         U[p * B:(p + 1) * B] = get_vals(u_off, B, lay["ldu"], J)
         if V is not None:
             V[p * B:(p + 1) * B] = get_vals(v_off, B, lay["ldv"], D)

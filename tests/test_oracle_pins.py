@@ -434,3 +434,63 @@ def test_rel_fro_hand_values():
     assert orc.rel_fro([0.0, 0.0], [0.0, 0.0]) == 0.0
     # float32 inputs are promoted, not compared in fp32
     assert orc.rel_fro(np.float32([1.0]), np.float64([1.0 + 1e-12])) == pytest.approx(1e-12, rel=1e-3)
+
+
+# ----------------------------------------------------------------------------- inactive-pair compaction
+def test_compact_pack_hand_example_bytes():
+    """Two workers x three slots, J = 2, D = 3, fp32.  Pairs 1, 3 and 4 have u = 0 and are left out: worker 0 keeps
+    pairs (0, 2), worker 1 keeps pair 5.  Every offset below is computed by hand from the wire format: header 128 B,
+    directory 2 x 32 B padded to 128, so streams start at 256; ldu = 4, ldv = 4 (rows padded to 16 bytes); U block
+    3 x 4 x 4 = 48 -> 128 B, V block likewise, stream stride 256."""
+    U = np.array([[1, 2], [0, 0], [3, 4], [0, 0], [0, 0], [5, 6]], dtype=np.float64)
+    V = np.arange(18, dtype=np.float64).reshape(6, 3) + 1.0
+    buf = orc.pack(orc.MODEL_DML, orc.DTYPE_F32, 2, 3, 2, 3, U, V, clock=9, compact=True)
+    assert buf.size == 256 + 2 * 256
+    assert int(buf[8:12].view(np.uint32)[0]) == 2                       # flags: bit 1 = compacted, bit 0 (sparse v) clear
+    assert int(buf[128 + 4:128 + 8].view(np.uint32)[0]) == 2            # worker 0: two pairs kept
+    assert int(buf[160 + 4:160 + 8].view(np.uint32)[0]) == 1            # worker 1: one pair kept
+    f = lambda off, n: buf[off:off + 4 * n].view(np.float32).tolist()
+    assert f(256, 12) == [1, 2, 0, 0, 3, 4, 0, 0, 0, 0, 0, 0]           # worker 0, U block: u_0, u_2, empty slot
+    assert f(256 + 128, 12) == [1, 2, 3, 0, 7, 8, 9, 0, 0, 0, 0, 0]     # worker 0, V block: v_0, v_2, empty slot
+    assert f(512, 12) == [5, 6, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0]           # worker 1, U block: u_5 only
+    assert f(512 + 128, 12) == [16, 17, 18, 0, 0, 0, 0, 0, 0, 0, 0, 0]  # worker 1, V block: v_5 only
+    # what a broadcast carries: header + directory entries + three pairs of (2 + 3) fp32 values
+    assert orc.wire_bytes(buf) == 128 + 2 * 32 + 3 * 5 * 4
+    full = orc.pack(orc.MODEL_DML, orc.DTYPE_F32, 2, 3, 2, 3, U, V, clock=9)
+    assert orc.wire_bytes(full) == 128 + 2 * 32 + 6 * 5 * 4
+
+
+def test_compaction_leaves_the_update_unchanged_and_round_trips():
+    """Dropping pairs with u = 0 changes nothing in W' = W - eta sum u v^T; pairs keep their order inside a worker;
+    with every pair active the buffer differs from the plain one in the flag bit only."""
+    rng = np.random.default_rng(21)
+    J, D, P, B = 5, 7, 3, 4
+    K = P * B
+    L = (0.3 * rng.standard_normal((J, D))).astype(np.float32)
+    Xa, Xb = rng.standard_normal((K, D)).astype(np.float32), rng.standard_normal((K, D)).astype(np.float32)
+    sim = (np.arange(K) % 2 == 0).astype(np.uint8)
+    U, V, n, active = orc.dml_factors(L, Xa, Xb, sim, 1.0)
+    assert 0 < (~active).sum() < K                                       # the case has pairs beyond the margin
+    buf = orc.pack(orc.MODEL_DML, orc.DTYPE_F32, J, D, P, B, U, V, compact=True)
+    h, Uc, Vc = orc.unpack(buf)
+    assert h["flags"] == orc.FLAG_COMPACT
+    U32 = U.astype(np.float32)
+    for p in range(P):
+        kept = [i for i in range(p * B, (p + 1) * B) if U32[i].any()]
+        assert h["n_sf"][p] == len(kept)
+        assert np.array_equal(Uc[p * B:p * B + len(kept)], U32[kept])    # original order inside the worker
+        assert np.array_equal(Vc[p * B:p * B + len(kept)], V.astype(np.float32)[kept])
+        assert not Uc[p * B + len(kept):(p + 1) * B].any() and not Vc[p * B + len(kept):(p + 1) * B].any()
+    W_full = orc.apply_dense(L, U32, V.astype(np.float32), 0.1)
+    W_comp = orc.apply_dense(L, Uc, Vc, 0.1)
+    assert np.abs(W_full - W_comp).max() <= 1e-15 * np.abs(W_full).max()
+    assert sum(h["n_sf"]) == int(active.sum())
+    # all pairs active: same bytes except the flag word
+    Ua = U.copy()
+    Ua[~active] = 1.0
+    a, b = (orc.pack(orc.MODEL_DML, orc.DTYPE_F32, J, D, P, B, Ua, V, compact=c) for c in (False, True))
+    diff = np.nonzero(a != b)[0]
+    assert diff.tolist() == [8]
+    with pytest.raises(ValueError):
+        orc.pack(orc.MODEL_SC, orc.DTYPE_F32, J, D, P, B, U, csr=(np.zeros(K + 1, np.uint32), np.zeros(0, np.uint32),
+                                                                   np.zeros(0, np.float32)), nnz_capacity=32 * P, compact=True)
