@@ -376,6 +376,8 @@ def main():
                          "over the ranks with an all-gather of the worker streams per step (sufficient factor broadcasting)")
     for dim in ("J", "D", "P", "B"):
         ap.add_argument(f"--{dim}", type=int, default=None, help=f"override {dim} (smaller cases for profiler captures)")
+    ap.add_argument("--compact", action="store_true",
+                    help="leave pairs whose u is zero out of the SF buffer (DML: dissimilar pairs beyond the margin)")
     ap.add_argument("--density", type=float, default=None,
                     help="sparse coding: fraction of nonzeros in the codes (default: the configuration's 5 %%)")
     args = ap.parse_args()
@@ -393,6 +395,8 @@ def main():
         from sfbgen import scaled
         cfg = scaled(args.config, **over)
     path = args.path or cfg["path"]
+    if args.compact:
+        cfg["compact"] = 1
 
     if args.impl == "reference":
         if rank == 0:
@@ -552,7 +556,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": workload_name(cfg, path), "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "per-step footprint larger than L2" if flush is None else "L2 flushed between steps",
-                       "eta": eta, "pool": cfg["pool"], "cuda_graph": graphs_used},
+                       "eta": eta, "pool": cfg["pool"], "cuda_graph": graphs_used, "compact": bool(cfg.get("compact", 0))},
             "e2e": {"value": whole_job_throughput(K, args.steps, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "last_clock_read_back": clock_of_last,
                     "returned": "the 128-byte header the step committed (clock, shapes); W (the worker's local copy of "
@@ -563,6 +567,14 @@ def main():
                           "pass": "the timed region of `value`" if stages_same_pass else "a second pass after it"},
             "clocks": clocks.summary(),
         }
+        # the message of the last step: what a full broadcast (every worker to P - 1 peers) would put on the wire,
+        # next to what synchronising the full matrix through a server would (push + pull of J x D per worker)
+        P_ = cfg["P"]
+        sent = wl.ctx.wire_bytes(wl.sf_buf)
+        es_ = 2 if path == "bf16" else 4
+        out["wire"] = {"sf_buffer_bytes_sent": sent, "compacted": bool(cfg.get("compact", 0)),
+                       "full_broadcast_bytes": (P_ - 1) * sent,
+                       "full_matrix_sync_bytes": 2 * P_ * cfg["J"] * cfg["D"] * es_}
         applied = wl.ctx.active_pairs()
         if alg is not None and 0 < applied < K:
             # the apply left out pairs whose u is zero: its work is counted on the pairs it multiplied through

@@ -58,6 +58,15 @@
  *               u32 idx[cap_p], value val[cap_p], each padded to 128 B, unused tail zero.
  *   ldu (ldv) is J (D) rounded up so that a row is a whole number of 16-byte units.
  *   cap_p = nnz_capacity / P.  bf16 values are fp32 rounded to nearest even.
+ *
+ * Compacted buffers (sfb_desc.compact = 1; Section 6.1: the sufficient factors are sparse and that is used)
+ *   A pair whose u is all zeros (a dissimilar DML pair beyond the margin, a sample with a bad label) adds nothing
+ *   to the update and is not sent.  Per worker the remaining pairs sit in the first n_sf slots of the U and V
+ *   blocks, in their original order; the slots behind them are zero; the directory's n_sf is the worker's own
+ *   count and flags bit 1 is set.  Offsets and strides are those of the full buffer: a sender transmits the
+ *   first n_sf rows of each block (sfb_wire_bytes counts them), a receiver reads them in place.  sfb_pack and
+ *   sfb_step compact, sfb_apply leaves out the reduction blocks that hold only empty slots; W' is the same
+ *   sum (bit-identical on SFB_PATH_F32).  Not available with sparse v or sfb_factors_shard.
  */
 #ifndef SFB_H_
 #define SFB_H_
@@ -102,6 +111,7 @@ typedef struct sfb_desc {
   int32_t v_sparse;      /* 1: v is CSR (required for SFB_SC), 0: dense */
   float margin;          /* DML hinge margin on the squared distance */
   uint64_t nnz_capacity; /* total CSR capacity (a multiple of 32*P) when v_sparse */
+  int32_t compact;       /* 1: pairs whose u is all zeros are left out of the SF buffer (dense v only), see below */
 } sfb_desc;
 
 /* Per-model side inputs of the factor computation (device pointers; unused ones NULL). */
@@ -215,9 +225,15 @@ int sfb_loss(sfb_ctx* ctx, const void* W, const void* X, const sfb_aux* aux, dou
 
 /* Number of (u, v) pairs the last sfb_step actually multiplied through.  SFB_DML on SFB_PATH_F32 leaves out the
  * pairs whose u is zero (dissimilar pairs beyond the margin; the update is bit-identical to the sum over all K
- * slots, Section 6 notes that such sparsity can be used); every other model / path applies all K slots and
- * reports K.  Synchronises the stream.  *n is 0 before the first step. */
+ * slots, Section 6 notes that such sparsity can be used), and so does every context with compact = 1 (the count
+ * is then the number of pairs the compaction kept); every other model / path applies all K slots and reports K.  Synchronises the stream.  *n is 0 before the first step. */
 int sfb_active_pairs(sfb_ctx* ctx, int32_t* n);
+
+/* Bytes a broadcast of this committed buffer would carry (Section 5.1 counts them per pair of workers: every
+ * worker sends its K pairs of J + D values to P - 1 peers): header, directory entries, and per worker its first
+ * n_sf rows of U and of dense V (sparse v: its B rows of U, B + 1 row pointers and nnz (index, value) pairs);
+ * padding is not counted.  Synchronises the stream (reads the directory back). */
+int sfb_wire_bytes(sfb_ctx* ctx, const void* sf_buf, uint64_t* bytes);
 
 /* Tells the context that W was changed by someone else, so a cached bf16 shadow is stale. */
 int sfb_invalidate(sfb_ctx* ctx);

@@ -25,13 +25,14 @@ EXPORTS = (
     "sfb_profile", "sfb_stage_ms", "sfb_sc_factors_noalloc", "sfb_noalloc_max_scratch_floats",
     "sfb_halton_peers", "sfb_ssp_may_proceed", "sfb_prox", "sfb_step_host",
     "sfb_loss", "sfb_factors_shard", "sfb_commit_header", "sfb_sf_buffer_layout", "sfb_active_pairs",
+    "sfb_wire_bytes",
 )
 
 
 class sfb_desc(C.Structure):
     _fields_ = [("model", C.c_int32), ("path", C.c_int32), ("J", C.c_int32), ("D", C.c_int32),
                 ("P", C.c_int32), ("B", C.c_int32), ("v_sparse", C.c_int32), ("margin", C.c_float),
-                ("nnz_capacity", C.c_uint64)]
+                ("nnz_capacity", C.c_uint64), ("compact", C.c_int32)]
 
 
 class sfb_aux(C.Structure):
@@ -88,6 +89,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.sfb_commit_header.restype = C.c_int
     lib.sfb_sf_buffer_layout.argtypes = [C.POINTER(sfb_desc), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.sfb_sf_buffer_layout.restype = C.c_int
+    lib.sfb_wire_bytes.argtypes = [vp, vp, C.POINTER(C.c_uint64)]
+    lib.sfb_wire_bytes.restype = C.c_int
     lib.sfb_invalidate.argtypes = [vp]
     lib.sfb_invalidate.restype = C.c_int
     lib.sfb_status.argtypes = [vp, C.POINTER(C.c_int32)]
@@ -117,9 +120,9 @@ def strerror(code: int) -> str:
     return load_library().sfb_strerror(code).decode()
 
 
-def make_desc(model, path, J, D, P, B, v_sparse=0, margin=1.0, nnz_capacity=0) -> sfb_desc:
+def make_desc(model, path, J, D, P, B, v_sparse=0, margin=1.0, nnz_capacity=0, compact=0) -> sfb_desc:
     return sfb_desc(MODELS.get(model, model), PATHS.get(path, path), J, D, P, B, int(v_sparse), float(margin),
-                    int(nnz_capacity))
+                    int(nnz_capacity), int(compact))
 
 
 def _ptr(t) -> int | None:
@@ -253,6 +256,12 @@ class Context:
     def loss(self, W, X, aux: sfb_aux, out):
         """Minibatch objective at W into `out` (one float64 on the device); asynchronous."""
         self._chk(self._lib.sfb_loss(self._h, _ptr(W), _ptr(X), C.byref(aux), _ptr(out)), "sfb_loss")
+
+    def wire_bytes(self, sf_buf) -> int:
+        """Bytes a broadcast of the committed buffer would carry (synchronises)."""
+        n = C.c_uint64(0)
+        self._chk(self._lib.sfb_wire_bytes(self._h, _ptr(sf_buf), C.byref(n)), "sfb_wire_bytes")
+        return int(n.value)
 
     def invalidate(self):
         self._chk(self._lib.sfb_invalidate(self._h), "sfb_invalidate")

@@ -32,6 +32,8 @@ struct sfb_ctx {
   int* dml_idx;             // [K] indices followed by the count
   int last_step_K;          // K of the last sfb_step (0: none yet) and whether its apply walked the list
   bool last_step_listed;
+  void* compact_ws;         // compact = 1: flags, new slots and per-worker counts of the pair compaction
+  int* kept_idx;            // compact = 1, fp32 path: ordered list of the kept pairs' slots, followed by its length
   float* f32_nn_ws;         // fp32 dense path: transposed copies of the forward's operands (large shapes only)
   float* loss_rows;         // sfb_loss: fp32 products [K][ldl], allocated by the first call
   float* loss_i;            // sfb_loss: per-sample objective [K]
@@ -75,6 +77,8 @@ int check_desc(const sfb_desc* d) {
   if (d->path == SFB_PATH_BF16 && (d->D % 8) != 0) return SFB_ERR_SHAPE;   // 16-byte rows of bf16 X and W shadow
   if (d->path == SFB_PATH_TF32 && (d->D % 4) != 0) return SFB_ERR_SHAPE;   // 16-byte rows of fp32 X and W
   if (d->model == SFB_DML && !(d->margin > 0.f)) return SFB_ERR_ARG;
+  if (d->compact != 0 && d->compact != 1) return SFB_ERR_ARG;
+  if (d->compact && d->v_sparse) return SFB_ERR_UNSUPPORTED;   // pair compaction is defined for dense v
   return SFB_OK;
 }
 
@@ -287,6 +291,10 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     }
   }
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
+  if (ok && desc->compact) {
+    ok = cudaMalloc(&c->compact_ws, (size_t)compact_workspace_bytes(c->K, desc->P)) == cudaSuccess;
+    if (ok && desc->path == SFB_PATH_F32) ok = cudaMalloc(&c->kept_idx, ((size_t)c->K + 1) * 4) == cudaSuccess;
+  }
   if (!ok) {
     cudaGetLastError();
     sfb_destroy(c);
@@ -322,6 +330,8 @@ int sfb_destroy(sfb_ctx* c) {
   if (c->csc_ws) cudaFree(c->csc_ws);
   if (c->f32_part) cudaFree(c->f32_part);
   if (c->f32_nn_ws) cudaFree(c->f32_nn_ws);
+  if (c->compact_ws) cudaFree(c->compact_ws);
+  if (c->kept_idx) cudaFree(c->kept_idx);
   if (c->dml_active) cudaFree(c->dml_active);
   if (c->dml_idx) cudaFree(c->dml_idx);
   if (c->loss_rows) cudaFree(c->loss_rows);
@@ -394,6 +404,16 @@ int sfb_active_pairs(sfb_ctx* c, int32_t* n) {
   *n = 0;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SFB_ERR_CUDA;
   if (c->last_step_K == 0) return SFB_OK;
+  if (c->d.compact) {   // the pair counts the compaction left in its workspace, over the workers the step applied
+    const int workers = c->last_step_K / c->d.B;
+    int32_t* h = new (std::nothrow) int32_t[workers];
+    if (h == nullptr) return SFB_ERR_ALLOC;
+    const char* counts = reinterpret_cast<const char*>(c->compact_ws) + pad_to(c->K, 256) + pad_to((long long)c->K * 4, 256);
+    const bool ok = cudaMemcpy(h, counts, (size_t)workers * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    for (int p = 0; ok && p < workers; ++p) *n += h[p];
+    delete[] h;
+    return ok ? SFB_OK : SFB_ERR_CUDA;
+  }
   if (c->dml_idx == nullptr || !c->last_step_listed) {
     *n = c->last_step_K;
     return SFB_OK;
@@ -401,6 +421,27 @@ int sfb_active_pairs(sfb_ctx* c, int32_t* n) {
   int32_t h = 0;
   if (cudaMemcpy(&h, c->dml_idx + c->K, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SFB_ERR_CUDA;
   *n = h;
+  return SFB_OK;
+}
+
+int sfb_wire_bytes(sfb_ctx* c, const void* sf_buf, uint64_t* bytes) {
+  if (c == nullptr || sf_buf == nullptr || bytes == nullptr) return SFB_ERR_ARG;
+  *bytes = 0;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SFB_ERR_CUDA;
+  const sfb_desc& d = c->d;
+  uint32_t* dir = new (std::nothrow) uint32_t[(size_t)d.P * 8];
+  if (dir == nullptr) return SFB_ERR_ALLOC;
+  const bool ok = cudaMemcpy(dir, reinterpret_cast<const char*>(sf_buf) + 128, (size_t)d.P * 32, cudaMemcpyDeviceToHost) ==
+                  cudaSuccess;
+  uint64_t total = 128 + (uint64_t)d.P * 32;
+  for (int p = 0; ok && p < d.P; ++p) {
+    const uint64_t n_sf = dir[p * 8 + 1] < (uint32_t)d.B ? dir[p * 8 + 1] : (uint32_t)d.B, nnz = dir[p * 8 + 3];
+    if (d.v_sparse) total += n_sf * d.J * c->l.es + ((uint64_t)d.B + 1) * 4 + nnz * (4 + (uint64_t)c->l.es);
+    else total += n_sf * ((uint64_t)d.J + d.D) * c->l.es;
+  }
+  delete[] dir;
+  if (!ok) return SFB_ERR_CUDA;
+  *bytes = total;
   return SFB_OK;
 }
 
@@ -481,6 +522,7 @@ int sfb_pack(sfb_ctx* c, const void* U, const void* V, const sfb_aux* aux, void*
   else
     ACC(launch_copy_rows(c->stream, caller_rows(V, c->l.ldv, d.B, c->l.es), stream_v(c, sf_buf), c->K, d.D));
   ACC(launch_write_header(c->stream, sf_buf, d, c->l, clock, rowptr));
+  if (d.compact) ACC(launch_compact(c->stream, sf_buf, d, c->l, c->compact_ws));
   return SFB_OK;
 }
 
@@ -506,7 +548,11 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
   } else if (d.path == SFB_PATH_F32) {
     const int* idx = nullptr;
     const int* n_idx = nullptr;
-    if (active_rows && c->dml_active != nullptr) {   // ordered list of the contributing pairs among the first K
+    if (d.compact) {   // compacted buffer: the kept pairs sit in the first n_sf slots of every worker (directory)
+      ACC(launch_kept_rows(c->stream, sf_buf, d.B, K / d.B, c->kept_idx, c->kept_idx + c->K));
+      idx = c->kept_idx;
+      n_idx = c->kept_idx + c->K;
+    } else if (active_rows && c->dml_active != nullptr) {   // ordered list of the contributing pairs among the first K
       ACC(launch_compact_active(c->stream, c->dml_active, K, c->dml_idx, c->dml_idx + c->K));
       idx = c->dml_idx;
       n_idx = c->dml_idx + c->K;
@@ -514,7 +560,8 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
     ACC(launch_apply_f32(c->stream, reinterpret_cast<float*>(W), stream_u(c, sf_buf), stream_v(c, sf_buf), K, d.J, d.D,
                          eta, c->dev_status, idx, n_idx));
   } else {
-    ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status));
+    ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status,
+                   d.compact ? reinterpret_cast<const char*>(sf_buf) + 128 : nullptr));
     if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
   }
   return SFB_OK;
@@ -525,6 +572,7 @@ int sfb_factors_shard(sfb_ctx* c, const void* W, const void* X, const sfb_aux* a
   if (c == nullptr || W == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
   if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
   const sfb_desc& d = c->d;
+  if (d.compact) return SFB_ERR_UNSUPPORTED;   // the sharded step keeps every slot
   if (first_worker < 0 || n_workers <= 0 || first_worker > d.P - n_workers) return SFB_ERR_ARG;
   int r = check_aux(c, aux);
   if (r != SFB_OK) return r;
@@ -616,8 +664,10 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
   r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes);
   if (forked && cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess) return SFB_ERR_CUDA;
   if (r < 0) return r;
+  // pairs whose u came out as zero are dropped from the message before it is "sent" (and applied)
+  if (d.compact) ACC(launch_compact(c->stream, sf_buf, d, c->l, c->compact_ws));
   if (c->profiling) cudaEventRecord(c->prof_ev[slot][1], c->stream);
-  const bool listed = d.model == SFB_DML && d.path == SFB_PATH_F32 && c->dml_active != nullptr &&
+  const bool listed = !d.compact && d.model == SFB_DML && d.path == SFB_PATH_F32 && c->dml_active != nullptr &&
                       (long long)((d.J + 127) / 128) * ((d.D + 127) / 128) >= 148;   // the large-tile apply takes the list
   r = apply_from(c, W, sf_buf, eta, K, false, csc_built, listed);
   c->last_step_K = K;

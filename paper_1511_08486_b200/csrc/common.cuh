@@ -119,6 +119,14 @@ int launch_write_header(cudaStream_t s, void* sf_buf, const sfb_desc& d, const L
 int launch_pack_csr(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, const uint32_t* rowptr,
                     const uint32_t* idx, const float* val, int* dev_status);
 
+// Inactive-pair compaction of a committed dense-v buffer, in place: per worker the pairs with a nonzero u move to
+// the front (same order), the slots behind them are cleared, the directory gets the pair counts and the header
+// its "compacted" flag.  workspace: compact_workspace_bytes(K, P) bytes.  launch_kept_rows lists the slots
+// p * B + r, r < count of worker p, of the first `workers` workers (idx [K], n_out one int; device arrays).
+long long compact_workspace_bytes(int K, int P);
+int launch_compact(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace);
+int launch_kept_rows(cudaStream_t s, const void* sf_buf, int B, int workers, int* idx, int* n_out);
+
 // Sets SFB_DEV_BAD_HEADER in *dev_status unless the buffer's header matches the descriptor.
 int launch_check_header(cudaStream_t s, const void* sf_buf, const sfb_desc& d, const Layout& l, int* dev_status);
 

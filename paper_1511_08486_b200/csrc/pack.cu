@@ -73,6 +73,7 @@ __global__ void check_header_kernel(const char* buf, HeaderImage h, int* dev_sta
   const int t = threadIdx.x;   // 32 threads
   bool ok = true;
   if (t < 17 && t != 7) ok = (w[t] == ref[t]);   // word 7 is the clock: any value is accepted
+  if (t == 2) ok = ((w[t] & ~2u) == ref[t]);      // flag bit 1 (compacted) may be set or not
   if (!__all_sync(0xffffffffu, ok) && t == 0) atomicOr(dev_status, SFB_DEV_BAD_HEADER);
 }
 

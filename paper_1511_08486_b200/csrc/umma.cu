@@ -36,6 +36,7 @@ constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
 constexpr int RING_BYTES = 192 * 1024;   // shared memory given to the operand ring
 constexpr int MAX_STAGES = 8;
+constexpr int MAX_DIR_WORKERS = 256;      // workers whose pair counts the apply can take from the directory
 constexpr uint32_t WAIT_LIMIT = 1u << 20;   // polls of a bounded wait: a failed poll suspends about 1.4 us, so about 1.4 s
 
 struct GemmParams {
@@ -56,6 +57,9 @@ struct GemmParams {
   RowMap z;                 // forward: output rows (fp32 products, or exps in the factor's storage type)
   float2* stats;            // forward, EPI 1: (max, sum of exps) per (sample, half tile), [K][n_parts]
   int n_parts;
+  // apply: directory of the SF buffer (32-byte entries, word 1 = the worker's pair count) when the rows behind a
+  // worker's count are known to be zero and whole reduction blocks of them can be left out; nullptr = all B rows
+  const uint32_t* dir;
   const int* status_ro;
   int* status;
   int lose_signal;          // test hook: the first pair / CTA drops its first "stage free" signal (see UmmaPlan)
@@ -65,6 +69,8 @@ struct SharedCtl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   volatile int abort;
+  int k_total;                 // apply: reduction blocks per tile (sum of nb[] when a directory is given)
+  uint16_t nb[MAX_DIR_WORKERS];   // apply with a directory: reduction blocks of each worker
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int* status) {
@@ -154,6 +160,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&ctl->tmem_empty[b], 8 * CG);   // one arrival per epilogue warp of every CTA of the pair
     }
     ctl->abort = 0;
+    if (APPLY) {
+      int tot = p.k_blocks;
+      if (p.dir != nullptr) {   // only with B >= BK and at most MAX_DIR_WORKERS workers (the host checks)
+        tot = 0;
+        for (int w = 0; w < p.P; ++w) {
+          const int n = min((int)p.dir[w * 8 + 1], p.B);
+          const int nbw = (n + BK - 1) / BK;
+          ctl->nb[w] = (uint16_t)nbw;
+          tot += nbw;
+        }
+      }
+      ctl->k_total = tot;
+    }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmA);
     ptx::prefetch_tmap(&tmB);
@@ -167,7 +186,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (CG == 2) ptx::cluster_sync();   // the peer's barriers exist before anything is signalled remotely
   ptx::tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
-  const int total_work = p.m_tiles * p.n_tiles * p.k_splits;
+  // apply: every worker contributes its own number of reduction blocks; none at all = nothing to add to W
+  const int k_blocks = APPLY ? ctl->k_total : p.k_blocks;
+  const int k_per_split = APPLY ? k_blocks : p.k_per_split;
+  const bool by_dir = APPLY && p.dir != nullptr;
+  const int total_work = (APPLY && k_blocks == 0) ? 0 : p.m_tiles * p.n_tiles * p.k_splits;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (every CTA)
@@ -178,7 +201,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint64_t pol_a = ptx::l2_policy(p.a_policy), pol_b = ptx::l2_policy(p.b_policy);
     for (int work = cluster_id; work < total_work && ok; work += num_clusters) {
       const int tile = work / p.k_splits, split = work - tile * p.k_splits;
-      const int kb_begin = split * p.k_per_split, kb_end = min(kb_begin + p.k_per_split, p.k_blocks);
+      const int kb_begin = split * k_per_split, kb_end = min(kb_begin + k_per_split, k_blocks);
       int mt, nt;
       tile_coords(p, tile, mt, nt);
       mt = mt * CG + (int)rank;                           // 128-row unit of this CTA
@@ -189,6 +212,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         else { mp0 = mt * p.m_wp; }
       }
       int row0 = 0, kp0 = 0;           // apply: first row / worker of the current reduction block
+      if (by_dir)
+        while (kp0 < p.P && ctl->nb[kp0] == 0) ++kp0;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
         ok = wait_or_abort(&ctl->empty[s], ph ^ 1u, ctl, p.status);
         if (!ok) break;
@@ -247,7 +272,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (APPLY) {   // next reduction block: next BK rows of this worker, or the next group of workers
           if (p.B >= BK) {
             row0 += BK;
-            if (row0 >= p.B) { row0 = 0; ++kp0; }
+            if (row0 >= (by_dir ? (int)ctl->nb[kp0] * BK : p.B)) {
+              row0 = 0;
+              ++kp0;
+              if (by_dir)
+                while (kp0 < p.P && ctl->nb[kp0] == 0) ++kp0;
+            }
           } else {
             kp0 += p.k_wp;
           }
@@ -275,7 +305,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     bool ok = (rank == 0);
     for (int work = cluster_id; work < total_work && ok; work += num_clusters, ++it) {
       const int split = work % p.k_splits;
-      const int kb_begin = split * p.k_per_split, kb_end = min(kb_begin + p.k_per_split, p.k_blocks);
+      const int kb_begin = split * k_per_split, kb_end = min(kb_begin + k_per_split, k_blocks);
       const int buf = it & 1;
       const uint32_t acc_ph = (it >> 1) & 1u;
       ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
@@ -933,7 +963,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
 }
 
 int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
-               int K, const int* dev_status) {
+               int K, const int* dev_status, const void* directory) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   const int workers = K / d.B;
@@ -953,6 +983,9 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
   p.n_tiles = (d.D + v.bn - 1) / v.bn;
   p.k_splits = 1; p.k_per_split = p.k_blocks;
+  // pair counts from the directory: whole reduction blocks behind a worker's last pair are left out
+  p.dir = (directory != nullptr && d.B >= BK && workers <= MAX_DIR_WORKERS) ? reinterpret_cast<const uint32_t*>(directory)
+                                                                            : nullptr;
   p.Mvalid = d.J; p.Nvalid = d.D;
   p.m_fastest = (d.D > d.J) ? 1 : 0;   // U is K x J, V is K x D: share the slab of the larger factor matrix
   p.a_policy = p.m_fastest ? 2 : 0;

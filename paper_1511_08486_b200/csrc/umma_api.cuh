@@ -23,7 +23,9 @@ int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, Ro
 
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
 // u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).
+// directory (optional): the SF buffer's directory (sf_buf + 128) of a compacted buffer, whose rows behind each
+// worker's pair count are zeros: reduction blocks that hold only such rows are skipped.
 int umma_apply(UmmaPlan* p, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
-               int K, const int* dev_status);
+               int K, const int* dev_status, const void* directory = nullptr);
 
 }  // namespace sfb

@@ -55,7 +55,7 @@ class DeviceWorkload:
         self.pool = cfg["pool"]
         sparse = model == "sc"
         self.desc = B.make_desc(model, self.path, J, D, P, Bsz, v_sparse=int(sparse), margin=cfg.get("margin", 1.0),
-                                nnz_capacity=inputs.get("nnz_capacity", 0))
+                                nnz_capacity=inputs.get("nnz_capacity", 0), compact=int(cfg.get("compact", 0)))
         self.ctx = B.Context(self.desc, stream)
         self.ldu, self.ldv = self.ctx.ldu, self.ctx.ldv
         dev = self.device
