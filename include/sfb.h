@@ -43,6 +43,14 @@
  *   SFB_PATH_BF16  tensor cores (tcgen05, kind::f16 with bf16 inputs), fp32 accumulate; X, U, V
  *                  bf16 in memory; W stays an fp32 master and the context keeps a bf16 shadow of
  *                  it that the apply refreshes.
+ *   SFB_PATH_TF32X3  tensor cores with error compensation, for fp32-grade results (the tolerance class of
+ *                  SFB_PATH_F32): every fp32 operand is split, inside the kernel, into the part the tensor core
+ *                  sees (its top 10 mantissa bits) and the exact remainder, and each product is formed from
+ *                  three tensor-core multiplications (a b ~ hi hi + lo hi + hi lo); X, U, V fp32 in memory,
+ *                  same wire format as SFB_PATH_TF32.  The tensor core's fp32 accumulator rounds toward zero
+ *                  once per instruction of 8 reduction steps, which costs about 1.6e-8 of a sum per
+ *                  instruction: forward reductions are cut into ranges that are added in fp32 afterwards, and
+ *                  the stated tolerance holds for updates of up to about 4096 pairs per sfb_apply.
  *
  * SF buffer wire format (little-endian; every offset a multiple of 128 bytes)
  *   header, 128 bytes:
@@ -81,7 +89,7 @@ extern "C" {
 typedef struct sfb_ctx sfb_ctx; /* opaque: workspace, cached tensor maps, device status word */
 
 enum { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2 };
-enum { SFB_PATH_F32 = 0, SFB_PATH_TF32 = 1, SFB_PATH_BF16 = 2 };
+enum { SFB_PATH_F32 = 0, SFB_PATH_TF32 = 1, SFB_PATH_BF16 = 2, SFB_PATH_TF32X3 = 3 };
 
 enum {
   SFB_OK = 0,

@@ -11,12 +11,12 @@ import os
 from .build import LIB_PATH
 
 SFB_MLR, SFB_DML, SFB_SC = 0, 1, 2
-SFB_PATH_F32, SFB_PATH_TF32, SFB_PATH_BF16 = 0, 1, 2
+SFB_PATH_F32, SFB_PATH_TF32, SFB_PATH_BF16, SFB_PATH_TF32X3 = 0, 1, 2, 3
 SFB_OK = 0
 SFB_DEV_BAD_LABEL, SFB_DEV_BAD_INDEX, SFB_DEV_BAD_HEADER, SFB_DEV_CAPACITY, SFB_DEV_TIMEOUT = 1, 2, 4, 8, 16
 
 MODELS = {"mlr": SFB_MLR, "dml": SFB_DML, "sc": SFB_SC}
-PATHS = {"f32": SFB_PATH_F32, "tf32": SFB_PATH_TF32, "bf16": SFB_PATH_BF16}
+PATHS = {"f32": SFB_PATH_F32, "tf32": SFB_PATH_TF32, "bf16": SFB_PATH_BF16, "tf32x3": SFB_PATH_TF32X3}
 
 # Every entry point include/sfb.h declares (checked by the CPU test-suite against the built library).
 EXPORTS = (

@@ -62,7 +62,7 @@ bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p
 int check_desc(const sfb_desc* d) {
   if (d == nullptr) return SFB_ERR_ARG;
   if (d->model < SFB_MLR || d->model > SFB_SC) return SFB_ERR_ARG;
-  if (d->path < SFB_PATH_F32 || d->path > SFB_PATH_BF16) return SFB_ERR_ARG;
+  if (d->path < SFB_PATH_F32 || d->path > SFB_PATH_TF32X3) return SFB_ERR_ARG;
   if (d->J <= 0 || d->D <= 0 || d->P <= 0 || d->B <= 0) return SFB_ERR_SHAPE;
   if ((long long)d->P * d->B > (1 << 24)) return SFB_ERR_SHAPE;
   if (d->model == SFB_SC) {
@@ -75,7 +75,8 @@ int check_desc(const sfb_desc* d) {
   }
   if (d->path == SFB_PATH_BF16 && d->model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
   if (d->path == SFB_PATH_BF16 && (d->D % 8) != 0) return SFB_ERR_SHAPE;   // 16-byte rows of bf16 X and W shadow
-  if (d->path == SFB_PATH_TF32 && (d->D % 4) != 0) return SFB_ERR_SHAPE;   // 16-byte rows of fp32 X and W
+  if ((d->path == SFB_PATH_TF32 || d->path == SFB_PATH_TF32X3) && (d->D % 4) != 0)
+    return SFB_ERR_SHAPE;   // 16-byte rows of fp32 X and W
   if (d->model == SFB_DML && !(d->margin > 0.f)) return SFB_ERR_ARG;
   if (d->compact != 0 && d->compact != 1) return SFB_ERR_ARG;
   if (d->compact && d->v_sparse) return SFB_ERR_UNSUPPORTED;   // pair compaction is defined for dense v
@@ -161,9 +162,10 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
   }
   if (d.model == SFB_SC) {   // dense alternative: the codes as dense tf32 rows through the tensor-core GEMM
     const RowMap a = dense_codes(c);
-    ACC(launch_densify_codes(c->stream, codes, a, K, d.D, c->dev_status));
-    ACC(umma_forward_rows(c->umma, c->stream, W, a, u, c->dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers));
-    ACC(launch_finish_sc(c->stream, u, u, reinterpret_cast<const float*>(aux->Xdata), K, d.J));
+    // plain tf32: the code values are rounded to nearest tf32 as they are densified; the compensated path keeps
+    // them exact (its kernels split every operand into what the tensor core sees and the rest)
+    ACC(launch_densify_codes(c->stream, codes, a, K, d.D, c->dev_status, d.path == SFB_PATH_TF32));
+    ACC(umma_forward_sc(c->umma, c->stream, W, a, u, reinterpret_cast<const float*>(aux->Xdata), c->dev_status, workers));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {
@@ -262,7 +264,7 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     ok = cudaMalloc(&c->wt_ws, (size_t)sc_forward_workspace_bytes(desc->J, desc->D)) == cudaSuccess;
   if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_F32 && sc_csc_supported(c->K))
     ok = cudaMalloc(&c->csc_ws, (size_t)sc_csc_workspace_bytes(c->K, desc->D, (long long)desc->nnz_capacity)) == cudaSuccess;
-  if (ok && desc->model == SFB_SC && desc->path == SFB_PATH_TF32)
+  if (ok && desc->model == SFB_SC && (desc->path == SFB_PATH_TF32 || desc->path == SFB_PATH_TF32X3))
     ok = cudaMalloc(&c->a_dense, (size_t)c->K * c->l.ldv * 4) == cudaSuccess;
   if (ok && desc->model != SFB_SC && desc->path == SFB_PATH_F32) {
     const int ks = forward_f32_splits(c->K, desc->J, desc->D);
@@ -543,7 +545,9 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
                         d.D, eta, c->dev_status, c->dev_status));
   } else if (d.v_sparse) {
     // dense alternative: rebuild the dense code rows from the buffer's CSR streams unless this step just made them
-    if (check) ACC(launch_densify_codes(c->stream, stream_codes(c, sf_buf), dense_codes(c), K, d.D, c->dev_status));
+    if (check)
+      ACC(launch_densify_codes(c->stream, stream_codes(c, sf_buf), dense_codes(c), K, d.D, c->dev_status,
+                               d.path == SFB_PATH_TF32));
     ACC(umma_apply(c->umma, c->stream, W, nullptr, stream_u(c, sf_buf), dense_codes(c), eta, K, c->dev_status));
   } else if (d.path == SFB_PATH_F32) {
     const int* idx = nullptr;

@@ -121,7 +121,8 @@ __global__ void __launch_bounds__(256) sc_forward_kernel(const float* __restrict
 }
 
 // One block per sample: zero the dense row, then scatter the sample's nonzeros into it.
-__global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, int K, int D, int* dev_status) {
+__global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, int K, int D, int* dev_status,
+                                                      bool round_tf32) {
   const int i = blockIdx.x;
   float* dst = reinterpret_cast<float*>(a.row(i));
   for (int q = threadIdx.x; q < (a.ld >> 2); q += 256) reinterpret_cast<float4*>(dst)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -133,8 +134,8 @@ __global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, i
     else {
       // the tensor cores drop the low 13 mantissa bits of a tf32 operand: rounding the code value to nearest
       // here (the dense rows are only ever a tf32 operand; the wire keeps the exact CSR values) halves that error
-      uint32_t r;
-      asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(row.val[k]));
+      uint32_t r = __float_as_uint(row.val[k]);
+      if (round_tf32) asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(row.val[k]));
       dst[c] = __uint_as_float(r);
     }
   }
@@ -327,8 +328,8 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
   return cudaGetLastError() == cudaSuccess ? 2 : SFB_ERR_CUDA;
 }
 
-int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status) {
-  densify_kernel<<<K, 256, 0, s>>>(codes, a, K, D, dev_status);
+int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status, bool round_tf32) {
+  densify_kernel<<<K, 256, 0, s>>>(codes, a, K, D, dev_status, round_tf32);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

@@ -33,6 +33,7 @@ namespace {
 
 constexpr int BM = 128;          // rows per CTA tile = TMEM lanes
 constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
+constexpr int SPLIT_THREADS = 128;       // error-compensated kernels: 4 more warps that split the operand stages
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
 constexpr int RING_BYTES = 192 * 1024;   // shared memory given to the operand ring
 constexpr int MAX_STAGES = 8;
@@ -67,15 +68,17 @@ struct GemmParams {
 
 struct SharedCtl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+  uint64_t ready[MAX_STAGES];   // error-compensated kernels: the stage's residual tiles are written (both CTAs of a pair)
   uint32_t tmem_base;
   volatile int abort;
   int k_total;                 // apply: reduction blocks per tile (sum of nb[] when a directory is given)
   uint16_t nb[MAX_DIR_WORKERS];   // apply with a directory: reduction blocks of each worker
 };
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int* status) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int* status,
+                                              bool cluster_scope = false) {
   for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (cluster_scope ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && ctl->abort) return false;
   }
   ctl->abort = 1;
@@ -124,8 +127,16 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 //   FOLD   operands come through 4-D tensor maps whose extra dimension walks the 128-byte chunks, so
 //          one TMA instruction fills a whole operand stage (needs J, D multiples of CH); otherwise
 //          one 3-D TMA per chunk, with zero fill on every ragged edge.
-template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+//   SPLIT  error-compensated tf32 (ES = 4): the tensor core drops the low 13 mantissa bits of an fp32 operand, so
+//          x = hi + lo with hi = what the tensor core sees of x and lo = x - hi (exact in fp32).  Four extra
+//          warps compute the lo tiles of every operand stage in shared memory, and every reduction step
+//          issues three MMAs: a * b into the main accumulator, lo(a) * b and a * lo(b) into a second one
+//          (lo * lo, about 2^-22 of the product, is dropped).  The accumulators are added in the epilogue.
+//          Two accumulators because the tensor core's fp32 accumulation rounds toward zero once per
+//          instruction (measured: a sum of n instructions comes out short by about n * 2^-26): the small
+//          corrections must not cost the large sum two more roundings per step.
+template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI, bool SPLIT>
+__global__ void __launch_bounds__(NUM_THREADS + (SPLIT ? SPLIT_THREADS : 0), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
   constexpr int CH = 128 / ES;                 // values per 128-byte chunk
@@ -134,7 +145,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   constexpr int BNC = BN / CG;                 // B columns this CTA loads
   constexpr int A_STAGE_BYTES = BM * 128 * KA;
   constexpr int B_STAGE_BYTES = BNC * 128 * KA;
-  constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  constexpr int RAW_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;     // what TMA brings per stage
+  constexpr int STAGE_BYTES = RAW_BYTES * (SPLIT ? 2 : 1);     // SPLIT: the lo tiles follow, same layout
+  constexpr int NACC = SPLIT ? 2 : 1;                          // accumulators per tile (main, corrections)
+  constexpr int ACC_COLS = BN * NACC;
+  static_assert(!SPLIT || (ES == 4 && EPI == 0), "error compensation is for fp32 operands and plain stores");
+  // whose "full" barrier a CTA's loads are credited to: its own (single CTAs; and SPLIT pairs, where each CTA's
+  // splitter warps wait for their own CTA's bytes), or the even CTA's (plain pairs: one barrier for the MMA issuer)
+  constexpr bool OWN = (CG == 1) || SPLIT;
   constexpr int STAGES = (RING_BYTES / STAGE_BYTES) < MAX_STAGES ? (RING_BYTES / STAGE_BYTES) : MAX_STAGES;
   constexpr uint32_t IDESC = ptx::instr_desc(ES == 2 ? 1u : 2u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM * CG, BN);
   static_assert(STAGES >= 2, "ring too shallow");
@@ -154,6 +172,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&ctl->full[s], 1);
       ptx::mbar_init(&ctl->empty[s], 1);
+      ptx::mbar_init(&ctl->ready[s], (SPLIT_THREADS / 32) * CG);   // one arrival per splitter warp of every CTA
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->tmem_full[b], 1);
@@ -178,7 +197,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::prefetch_tmap(&tmB);
   }
   if (warp == 1) {
-    ptx::tmem_alloc<CG>(&ctl->tmem_base, 2 * BN);
+    ptx::tmem_alloc<CG>(&ctl->tmem_base, 2 * ACC_COLS);
     ptx::tmem_relinquish<CG>();
   }
   ptx::tc_fence_before();
@@ -223,10 +242,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           uint64_t* bar = &ctl->full[s];
           uint32_t full_addr = ptx::smem_u32(bar);
           if (CG == 2) full_addr = ptx::map_to_cta(full_addr, 0);
-          if (rank == 0) ptx::mbar_expect_tx(bar, CG * STAGE_BYTES);
+          if (OWN) ptx::mbar_expect_tx(bar, RAW_BYTES);
+          else if (rank == 0) ptx::mbar_expect_tx(bar, CG * STAGE_BYTES);
           if (!APPLY) {
             if (FOLD) {   // dims (value-in-atom, row, worker, atom): one box = KA atoms of 128 rows
-              if (CG == 1) {
+              if (OWN) {
                 ptx::tma_load_4d_hint(a_dst, &tmA, bar, 0, slot0, mp0, kb * KA, pol_a);
                 ptx::tma_load_4d_hint(b_dst, &tmB, bar, 0, ncol0, 0, kb * KA, pol_b);
               } else {
@@ -237,7 +257,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
               for (int a = 0; a < KA; ++a) {
                 const int k0 = (kb * KA + a) * CH;
-                if (CG == 1) {
+                if (OWN) {
                   ptx::tma_load_3d_hint(a_dst + a * (BM * 128), &tmA, bar, k0, slot0, mp0, pol_a);
                   ptx::tma_load_3d_hint(b_dst + a * (BNC * 128), &tmB, bar, k0, ncol0, 0, pol_b);
                 } else {
@@ -248,7 +268,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           } else {
             if (FOLD) {   // dims (value-in-chunk, row, worker, chunk): one box = all chunks x BK rows
-              if (CG == 1) {
+              if (OWN) {
                 ptx::tma_load_4d_hint(a_dst, &tmA, bar, 0, row0, kp0, (mt * BM) / CH, pol_a);
                 ptx::tma_load_4d_hint(b_dst, &tmB, bar, 0, row0, kp0, ncol0 / CH, pol_b);
               } else {
@@ -258,12 +278,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             } else {
 #pragma unroll
               for (int c = 0; c < BM / CH; ++c) {
-                if (CG == 1) ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, bar, mt * BM + c * CH, row0, kp0, pol_a);
+                if (OWN) ptx::tma_load_3d_hint(a_dst + c * (BK * 128), &tmA, bar, mt * BM + c * CH, row0, kp0, pol_a);
                 else ptx::tma_load_3d_hint_pair(a_dst + c * (BK * 128), &tmA, full_addr, mt * BM + c * CH, row0, kp0, pol_a);
               }
 #pragma unroll
               for (int c = 0; c < BNC / CH; ++c) {
-                if (CG == 1) ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, bar, ncol0 + c * CH, row0, kp0, pol_b);
+                if (OWN) ptx::tma_load_3d_hint(b_dst + c * (BK * 128), &tmB, bar, ncol0 + c * CH, row0, kp0, pol_b);
                 else ptx::tma_load_3d_hint_pair(b_dst + c * (BK * 128), &tmB, full_addr, ncol0 + c * CH, row0, kp0, pol_b);
               }
             }
@@ -287,7 +307,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
-    if ((!ok || ctl->abort) && rank == 0) {
+    if ((!ok || ctl->abort) && (rank == 0 || OWN)) {
       // let copies already in flight land before the CTA goes away (bounded)
       int n = issued < STAGES ? issued : STAGES;
       for (int q = 0; q < n; ++q) {
@@ -311,9 +331,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
       if (!ok) break;
       ptx::tc_fence_after();
-      const uint32_t d_tmem = tmem_base + buf * BN;
+      const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
+      const uint32_t d_lo = d_tmem + BN;              // SPLIT: accumulator of the correction products
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
+        ok = wait_or_abort(SPLIT ? &ctl->ready[s] : &ctl->full[s], ph, ctl, p.status, SPLIT && CG == 2);
         if (!ok) break;
         ptx::tc_fence_after();
         if (lane == 0) {
@@ -331,6 +352,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const uint32_t acc = (kb > kb_begin || a > 0 || k > 0) ? 1u : 0u;
                 if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
                 else ptx::mma_tf32<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
+                if (SPLIT) {   // lo(a) * b + a * lo(b): the lo tiles sit RAW_BYTES behind the raw ones
+                  ptx::mma_tf32<CG>(d_lo, a_desc + (RAW_BYTES >> 4) + k * 2, b_desc + k * 2, IDESC, acc);
+                  ptx::mma_tf32<CG>(d_lo, a_desc + k * 2, b_desc + (RAW_BYTES >> 4) + k * 2, IDESC, 1u);
+                }
               }
             }
           } else {
@@ -345,6 +370,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               const uint32_t acc = (kb > kb_begin || k > 0) ? 1u : 0u;
               if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
               else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
+              if (SPLIT) {
+                ptx::mma_tf32<CG>(d_lo, a_desc + (RAW_BYTES >> 4) + k * STEP, b_desc + k * STEP, IDESC, acc);
+                ptx::mma_tf32<CG>(d_lo, a_desc + k * STEP, b_desc + (RAW_BYTES >> 4) + k * STEP, IDESC, 1u);
+              }
             }
           }
           // (test hook: one lost signal, so that the producer's bounded wait runs out and the abort path is taken)
@@ -359,6 +388,43 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           }
         }
         __syncwarp();
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (SPLIT && warp >= NUM_THREADS / 32) {
+    // ------------------------------------------------------------------ operand splitter (warps 10..13, every CTA)
+    // For every stage that has landed: lo = x - (x with the low 13 mantissa bits cleared), element by element, into
+    // the second half of the stage (the swizzled layout is the same, so the tiles are walked as flat memory).
+    const int t = threadIdx.x - NUM_THREADS;
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    uint32_t ready_addr = ptx::smem_u32(&ctl->ready[0]);
+    if (CG == 2) ready_addr = ptx::map_to_cta(ready_addr, 0);
+    for (int work = cluster_id; work < total_work && ok; work += num_clusters) {
+      const int split = work % p.k_splits;
+      const int kb_begin = split * k_per_split, kb_end = min(kb_begin + k_per_split, k_blocks);
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
+        if (!ok) break;
+        uint4* raw = reinterpret_cast<uint4*>(tiles + s * STAGE_BYTES);
+#pragma unroll 4
+        for (int q = t; q < RAW_BYTES / 16; q += SPLIT_THREADS) {
+          const uint4 x = raw[q];
+          uint4 lo;
+          lo.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(x.x & 0xFFFFE000u));
+          lo.y = __float_as_uint(__uint_as_float(x.y) - __uint_as_float(x.y & 0xFFFFE000u));
+          lo.z = __float_as_uint(__uint_as_float(x.z) - __uint_as_float(x.z & 0xFFFFE000u));
+          lo.w = __float_as_uint(__uint_as_float(x.w) - __uint_as_float(x.w & 0xFFFFE000u));
+          raw[q + RAW_BYTES / 16] = lo;
+        }
+        ptx::fence_proxy_async();   // the tensor core reads these tiles through the async proxy
+        __syncwarp();
+        if (lane == 0) {
+          const uint32_t bar = ready_addr + (uint32_t)(s * sizeof(uint64_t));
+          if (CG == 1) ptx::mbar_arrive(&ctl->ready[s]);
+          else ptx::mbar_arrive_cluster(bar);
+        }
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
@@ -421,7 +487,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ok = wait_or_abort(&ctl->tmem_full[buf], acc_ph, ctl, p.status);
       if (!ok) break;
       ptx::tc_fence_after();
-      const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
+      const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
       if (!APPLY && EPI == 1) {
         // ---- multiclass-logistic epilogue: thread = sample row while the values sit in registers
         const float kLog2e = 1.4426950408889634f;
@@ -491,12 +557,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float4 wn[8];   // next block of W, in flight while this block is combined and stored
 #pragma unroll
         for (int g = 0; g < 8; ++g) wn[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (APPLY && cc + 1 < BN / 64) {
+        // (the compensated kernels have registers for one block of W only: they fetch the next one afterwards;
+        // their reduction loop is three times as long, so the epilogue has the time)
+        if (APPLY && !SPLIT && cc + 1 < BN / 64) {
 #pragma unroll
           for (int g = 0; g < 8; ++g)
             if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
         }
         ptx::tmem_ld_wait();
+        if (SPLIT) {   // main accumulator + correction accumulator, one fp32 addition (round to nearest) per value
+          uint32_t lo[32];
+          ptx::tmem_ld32(taddr + BN + col_in_tile, lo);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 32; ++q) v[q] = __float_as_uint(__uint_as_float(v[q]) + __uint_as_float(lo[q]));
+        }
 #pragma unroll
         for (int q = 0; q < 8; ++q)
           *reinterpret_cast<uint4*>(stage + lane * 32 + ((q ^ (lane & 7)) << 2)) =
@@ -526,6 +601,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
         }
+        if (APPLY && SPLIT && cc + 1 < BN / 64) {
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
+        }
 #pragma unroll
         for (int g = 0; g < 8; ++g) wv[g] = wn[g];
         if (APPLY) {   // the 32 x 32 block of new W sits in the staging block, swizzled as the tensor map expects
@@ -554,7 +634,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (CG == 2) ptx::cluster_sync();   // nobody leaves while its pair may still signal it or read its tiles
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc<CG>(tmem_base, 2 * BN);
+    ptx::tmem_dealloc<CG>(tmem_base, 2 * ACC_COLS);
   }
 }
 
@@ -610,13 +690,14 @@ int pow2_at_least(int n) {
   return p;
 }
 
-template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI>
+template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI, bool SPLIT = false>
 int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w, const GemmParams& p,
                 int num_sms) {
-  constexpr int stage_bytes = (BM + BN / CG) * 128 * KA;
+  constexpr int stage_bytes = (BM + BN / CG) * 128 * KA * (SPLIT ? 2 : 1);
+  constexpr int threads = NUM_THREADS + (SPLIT ? SPLIT_THREADS : 0);
   constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
   constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
-  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD, EPI>;
+  auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD, EPI, SPLIT>;
   static PerDeviceOnce attr_once;   // function attributes are per device
   static int max_clusters = 0;
   if (attr_once.first()) {
@@ -629,7 +710,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
       qa[0].id = cudaLaunchAttributeClusterDimension;
       qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
       q.gridDim = dim3(num_sms & ~1, 1, 1);
-      q.blockDim = dim3(NUM_THREADS, 1, 1);
+      q.blockDim = dim3(threads, 1, 1);
       q.dynamicSmemBytes = smem;
       q.attrs = qa; q.numAttrs = 1;
       if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &q) != cudaSuccess || max_clusters < 1) {
@@ -641,7 +722,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
   const int tiles = p.m_tiles * p.n_tiles * p.k_splits;
   if (CG == 1) {
     const int grid = tiles < num_sms ? tiles : num_sms;
-    kernel<<<grid, NUM_THREADS, smem, s>>>(a, b, w, p);
+    kernel<<<grid, threads, smem, s>>>(a, b, w, p);
   } else {
     const int clusters = tiles < max_clusters ? tiles : max_clusters;
     cudaLaunchConfig_t cfg;
@@ -650,7 +731,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.gridDim = dim3(2 * clusters, 1, 1);
-    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cfg.attrs = at; cfg.numAttrs = 1;
@@ -664,11 +745,20 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
 struct Variant {
   int bn, cg, ka;
   bool fold;
+  bool split;   // error-compensated tf32: 128-column tiles, one atom per stage, lo tiles made in shared memory
 };
 
 template <int ES, bool APPLY, int EPI>
 int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w,
                 const GemmParams& p, int num_sms) {
+  if (v.split) {
+    if (ES == 4 && EPI == 0) {   // the only instantiations: fp32 operands, plain stores / W write-back
+      if (v.cg == 2 && v.fold) return launch_gemm<4, APPLY, 128, 2, 1, true, 0, true>(s, a, b, w, p, num_sms);
+      if (v.cg == 2) return launch_gemm<4, APPLY, 128, 2, 1, false, 0, true>(s, a, b, w, p, num_sms);
+      return launch_gemm<4, APPLY, 128, 1, 1, false, 0, true>(s, a, b, w, p, num_sms);
+    }
+    return SFB_ERR_UNSUPPORTED;
+  }
   if (v.cg == 2) {
     if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, w, p, num_sms);
     if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, w, p, num_sms);
@@ -696,6 +786,7 @@ struct UmmaPlan {
   Layout l;
   int num_sms;
   int es;
+  bool x3;        // error-compensated tf32 (SFB_PATH_TF32X3): the SPLIT kernels, forward always through partial buffers
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
   float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
   int ldp;
@@ -715,12 +806,16 @@ struct UmmaPlan {
 constexpr int FWD_GROUP = 8, APPLY_GROUP = 8;
 // 128-byte atoms of the reduction index per pipeline stage wherever three such stages fit in shared memory.
 constexpr int STAGE_ATOMS = 2;
+// Compensated kernels: 128-byte atoms (32 fp32 reduction steps = 4 MMA instructions) one accumulator may take
+// before its range ends: 40 atoms = 160 roundings toward zero, about 2.6e-6 of the sum.
+constexpr int X3_ATOMS_PER_RANGE = 40;
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   if (get_encode() == nullptr) return SFB_ERR_CUDA;
   UmmaPlan* p = new UmmaPlan();
   p->d = d; p->l = l;
   p->es = (d.path == SFB_PATH_BF16) ? 2 : 4;
+  p->x3 = d.path == SFB_PATH_TF32X3;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev);
@@ -731,7 +826,7 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   {   // forward GEMMs whose 128 x 128 tiles do not fill the SMs may split their reduction
     const long long K_ = (long long)d.P * d.B;
     const long long tiles = ((K_ + 127) / 128) * ((d.J + 127) / 128);
-    if (tiles < p->num_sms && cudaMalloc(&p->part_ws, (size_t)MAX_SPLITS * K_ * p->ldp * 4) != cudaSuccess) {
+    if ((tiles < p->num_sms || p->x3) && cudaMalloc(&p->part_ws, (size_t)MAX_SPLITS * K_ * p->ldp * 4) != cudaSuccess) {
       cudaGetLastError();
       delete p;
       return SFB_ERR_ALLOC;
@@ -786,7 +881,28 @@ void umma_plan_destroy(UmmaPlan* p) {
 static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_chunk_aligned, int k_atoms = 0,
                             int max_splits = 1, int* splits = nullptr) {
   Variant v;
+  v.split = false;
   if (splits != nullptr) *splits = 1;
+  if (pl->x3) {
+    // Compensated kernels: 256 x 128 pair tiles (128 x 128 for a single row unit), one atom per stage.
+    v.split = true;
+    v.bn = 128; v.ka = 1;
+    v.cg = m_units >= 2 ? 2 : 1;
+    v.fold = v.cg == 2 && dims_chunk_aligned;
+    if (splits != nullptr && k_atoms > 0 && max_splits > 1) {
+      // Ranges of the reduction, added in fp32 by the finishing pass: enough of them that one accumulator takes
+      // at most X3_ATOMS_PER_RANGE atoms (4 instructions each; every instruction rounds the sum toward zero,
+      // about 1.6e-8 of it), and enough to give every SM work.
+      const long long tiles = (long long)((m_units + v.cg - 1) / v.cg) * ((N + 127) / 128);
+      const long long slots = pl->num_sms / v.cg;
+      long long ks = (k_atoms + X3_ATOMS_PER_RANGE - 1) / X3_ATOMS_PER_RANGE;
+      if (tiles * ks < slots) ks = (slots + tiles - 1) / tiles;
+      if (ks > max_splits) ks = max_splits;
+      while (ks > 1 && k_atoms < 4 * ks) --ks;
+      *splits = (int)(ks < 1 ? 1 : ks);
+    }
+    return v;
+  }
   v.bn = (N > 128 && (long long)m_units * ((N + 255) / 256) >= pl->num_sms) ? 256 : 128;
   // CTA pairs (256-row tiles) once there is enough work to fill the machine with them
   v.cg = (v.bn == 256 && (long long)((m_units + 1) / 2) * ((N + 255) / 256) >= pl->num_sms / 2) ? 2 : 1;
@@ -870,6 +986,30 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
     return SFB_ERR_CUDA;
   return stats != nullptr ? dispatch_gemm<false, 1>(s, es, v, ta, tb, ta, p, pl->num_sms)
                           : dispatch_gemm<false, 0>(s, es, v, ta, tb, ta, p, pl->num_sms);
+}
+
+// Sparse coding on the tensor cores: u rows = dense code rows `a` times W^T, minus the data rows.
+int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
+                    int workers) {
+  const sfb_desc& d = pl->d;
+  const int K = (workers > 0 ? workers : d.P) * d.B;
+  int r, launches = 0;
+  if (pl->part_ws != nullptr) {   // reduction in ranges (few tiles, or the compensated path): summed by the finishing pass
+    RowMap pz;
+    pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
+    pz.worker_stride = (long long)d.B * pl->ldp * 4;
+    const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
+    int ks = 1;
+    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
+      return r;
+    launches += r;
+    if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride)) < 0) return r;
+    return launches + r;
+  }
+  if ((r = umma_forward_rows(pl, s, W, a, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers)) < 0) return r;
+  launches += r;
+  if ((r = launch_finish_sc(s, u, u, Xdata, K, d.J)) < 0) return r;
+  return launches + r;
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,

@@ -21,6 +21,10 @@ int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, Ro
                       float2* stats = nullptr, int* n_parts_out = nullptr, int* part_cols_out = nullptr,
                       int* k_splits_out = nullptr, int max_splits = 1, long long split_stride = 0, int workers = 0);
 
+// Sparse coding: u rows = dense code rows `a` (fp32) times W^T minus the data rows Xdata [K][J].
+int umma_forward_sc(UmmaPlan* p, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
+                    int workers = 0);
+
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
 // u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).
 // directory (optional): the SF buffer's directory (sf_buf + 128) of a compacted buffer, whose rows behind each
