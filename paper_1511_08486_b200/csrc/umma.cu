@@ -172,7 +172,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&ctl->full[s], 1);
       ptx::mbar_init(&ctl->empty[s], 1);
-      ptx::mbar_init(&ctl->ready[s], (SPLIT_THREADS / 32) * CG);   // one arrival per splitter warp of every CTA
+      ptx::mbar_init(&ctl->ready[s], CG);   // one arrival per CTA: the splitter warp that took the stage
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->tmem_full[b], 1);
@@ -395,21 +395,29 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ------------------------------------------------------------------ operand splitter (warps 10..13, every CTA)
     // For every stage that has landed: lo = x - (x with the low 13 mantissa bits cleared), element by element, into
     // the second half of the stage (the swizzled layout is the same, so the tiles are walked as flat memory).
-    const int t = threadIdx.x - NUM_THREADS;
-    int s = 0;
-    uint32_t ph = 0;
+    // Each of the four warps takes its own stages of the ring and splits them alone, so up to four stages are in the works at a
+    // time: the chain "wait for the bytes, read, subtract, write, fence, signal" of one stage is longer than the
+    // tensor core needs for the stage's MMAs, but four of them overlap.
+    constexpr int NSPLIT = SPLIT_THREADS / 32;
+    const int sw = warp - NUM_THREADS / 32;
+    long long n_stage = 0;     // running count of reduction blocks over all of this CTA's tiles
     bool ok = true;
     uint32_t ready_addr = ptx::smem_u32(&ctl->ready[0]);
     if (CG == 2) ready_addr = ptx::map_to_cta(ready_addr, 0);
     for (int work = cluster_id; work < total_work && ok; work += num_clusters) {
       const int split = work % p.k_splits;
       const int kb_begin = split * k_per_split, kb_end = min(kb_begin + k_per_split, k_blocks);
-      for (int kb = kb_begin; kb < kb_end; ++kb) {
+      for (int kb = kb_begin; kb < kb_end; ++kb, ++n_stage) {
+        // a warp owns whole stages of the ring (stage s belongs to warp s mod 4), so it meets every phase of its
+        // stages' barriers in order; parity waits cannot tell phases two apart
+        const int s = (int)(n_stage % STAGES);
+        if (s % NSPLIT != sw) continue;
+        const uint32_t ph = (uint32_t)((n_stage / STAGES) & 1);
         ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
         if (!ok) break;
         uint4* raw = reinterpret_cast<uint4*>(tiles + s * STAGE_BYTES);
-#pragma unroll 4
-        for (int q = t; q < RAW_BYTES / 16; q += SPLIT_THREADS) {
+#pragma unroll 8
+        for (int q = lane; q < RAW_BYTES / 16; q += 32) {
           const uint4 x = raw[q];
           uint4 lo;
           lo.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(x.x & 0xFFFFE000u));
@@ -421,11 +429,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::fence_proxy_async();   // the tensor core reads these tiles through the async proxy
         __syncwarp();
         if (lane == 0) {
-          const uint32_t bar = ready_addr + (uint32_t)(s * sizeof(uint64_t));
           if (CG == 1) ptx::mbar_arrive(&ctl->ready[s]);
-          else ptx::mbar_arrive_cluster(bar);
+          else ptx::mbar_arrive_cluster(ready_addr + (uint32_t)(s * sizeof(uint64_t)));
         }
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
   } else {
