@@ -892,6 +892,11 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
   if (pl->x3) {
     // Compensated kernels: 256 x 128 pair tiles (128 x 128 for a single row unit), one atom per stage.
     v.split = true;
+    // 128 columns: main and correction accumulators of two tiles fill the 512 columns of tensor memory, so the
+    // epilogue of a tile overlaps the MMAs of the next (256-column tiles with a single set and an exposed epilogue
+    // were measured 6 % slower at 4096 x 10000, K = 1024, in spite of a third less shared-memory traffic per flop;
+    // two warps per stage instead of one stage per warp in the splitter changed nothing either: what bounds these
+    // kernels, at 43 % tensor-pipe activity, is the shared-memory read path of three MMAs per fp32 operand pair)
     v.bn = 128; v.ka = 1;
     v.cg = m_units >= 2 ? 2 : 1;
     v.fold = v.cg == 2 && dims_chunk_aligned;
