@@ -8,15 +8,15 @@
 // bit 1 is set.  Offsets and strides of the buffer do not change.
 //
 // In place and deterministic: a row only ever moves to a lower slot of its own worker, and every block of the
-// move kernel owns one (worker, 1 KB column slice) and walks the rows in waves of 32: a wave is read whole into
+// move kernel owns one (worker, 256-byte column slice) and walks the rows in waves of 64: a wave is read whole into
 // shared memory before any of its rows is written, and the slots it writes were all read by then.
 #include "common.cuh"
 
 namespace sfb {
 namespace {
 
-constexpr int WAVE = 32;          // rows per wave of the move
-constexpr int SLICE_UNITS = 64;   // 16-byte units per column slice (1 KB)
+constexpr int WAVE = 64;          // rows per wave of the move
+constexpr int SLICE_UNITS = 16;   // 16-byte units per column slice (256 B): many small blocks hide the latency
 
 // flags[i] = 1 if the wire values of u row i are not all zero (-0 counts as zero).  One warp per row.
 __global__ void __launch_bounds__(256) row_nonzero_kernel(RowMap u, int K, int J, uint8_t* __restrict__ flags) {
@@ -67,12 +67,12 @@ __global__ void __launch_bounds__(256) compact_scan_kernel(const uint8_t* __rest
   }
 }
 
-// grid = (P, slices of the U rows + slices of the V rows).  Moves this block's 1 KB column slice of every kept
+// grid = (P, slices of the U rows + slices of the V rows).  Moves this block's 256-byte column slice of every kept
 // row of worker p to its new slot and clears the slice in the slots behind the last kept row.
 __global__ void __launch_bounds__(256) compact_move_kernel(char* streams, long long stream_stride, long long v_off, int B,
                                                            int u_units, int v_units, int u_slices,
                                                            const int* __restrict__ dest, const int* __restrict__ counts) {
-  __shared__ uint4 wave[WAVE * SLICE_UNITS];   // 32 KB
+  __shared__ uint4 wave[WAVE * SLICE_UNITS];   // 16 KB
   __shared__ int s_dest[WAVE];
   const int p = blockIdx.x;
   const bool is_v = (int)blockIdx.y >= u_slices;
