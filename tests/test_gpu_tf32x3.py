@@ -50,3 +50,39 @@ def test_x3_c2_full():
 
 def test_x3_c3_full():
     check_config(_cfg("C3"), "tf32x3", eta=1e-4, steps=1)
+
+
+@pytest.mark.parametrize("path,P", [("bf16", 16), ("bf16", 64), ("tf32", 16), ("tf32", 64)])
+def test_tensor_core_accumulation_rounds_toward_zero(path, P):
+    """The measurement the design of the compensated kernels rests on.  With exact products (bf16 operands, or
+    fp32 operands with the low 13 mantissa bits already cleared) the only error of an apply to zero is the tensor
+    core's fp32 accumulation: it comes out SHORT of the exact sum by about n x 2^-26, n = MMA instructions per
+    output (16 bf16 or 8 tf32 reduction steps each), i.e. one rounding toward zero per instruction."""
+    import numpy as np
+    import torch
+    from oracle import sfb_oracle as orc
+    from sfbgen import make_inputs
+    from tests.test_gpu_parity import _workload
+    from tests.util import to_f64
+    cfg = scaled("C4" if path == "bf16" else "C1", J=256, D=256, P=P, B=256, pool=1, labels="uniform")
+    cfg["path"] = path
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, path)
+    try:
+        wl.compute_factors(0)
+        wl.pack(0)
+        wl.W.zero_()
+        wl.ctx.invalidate()
+        wl.apply(-1.0)
+        torch.cuda.synchronize()
+        U, V = to_f64(wl.U)[:, :256], to_f64(wl.V)[:, :256]
+        if path == "tf32":
+            cut = lambda a: (a.astype(np.float32).view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32).astype(np.float64)
+            U, V = cut(U), cut(V)
+        ref, got = orc.delta_w(U, V), to_f64(wl.W)
+        shortfall = -float(((got - ref) * ref).sum() / (ref * ref).sum())
+        n = cfg["K"] // (16 if path == "bf16" else 8)
+        print(f"{path} K={cfg['K']}: rel_fro {orc.rel_fro(got, ref):.3e}, short by {shortfall:.3e}, n x 2^-26 = {n * 2.0 ** -26:.3e}")
+        assert 0.5 * n * 2.0 ** -26 <= shortfall <= 2.0 * n * 2.0 ** -26
+    finally:
+        wl.close()
