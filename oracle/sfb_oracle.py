@@ -31,7 +31,8 @@ Parity pins (tests/test_oracle_pins.py): brute-force full-matrix gradients by a
 route that never forms u, central finite differences of the losses, sum_j u_ij
 = 0 for MLR, rank(Delta W) <= K by SVD, closed forms (W = 0, J = 2 logistic
 regression, one-hot codes, fixed points), additivity / eta-linearity /
-worker-split invariance of the apply, and byte-level checks of the packer.
+worker-split invariance of the apply, byte-level checks of the packer (plain and
+compacted), and hand values for the parity metric rel_fro and for wire_bytes.
 Multi-step trajectories have no closed form: parity unpinned beyond "the step is
 the composition of the pinned pieces" (guarded by loss decrease).
 """
