@@ -31,6 +31,33 @@ def _oracle_pack_of(cfg, path, U, V, batch, inputs, clock):
                     clock=clock, nnz_capacity=inputs.get("nnz_capacity", 0))
 
 
+_ORACLE_MEMO = {}
+
+
+def _memo(cfg, tag, fn):
+    """Oracle results that several tests of one session ask for again (the same workload on another arithmetic
+    path): computed once.  Keyed by everything that determines the synthetic inputs and the request."""
+    key = (tag,) + tuple(sorted((k, repr(v)) for k, v in cfg.items() if k not in ("path", "compact")))
+    if key not in _ORACLE_MEMO:
+        if len(_ORACLE_MEMO) > 4:
+            _ORACLE_MEMO.clear()
+        _ORACLE_MEMO[key] = fn()
+    return _ORACLE_MEMO[key]
+
+
+def _sc_update_from_zero(cfg, U, batch, n_rows=None):
+    """U^T A for sparse codes A: the oracle's sparse apply to W = 0 with eta = -1, or, for workloads whose K outer
+    products would take its Python loop minutes, the dense product of the same codes (the same sum; the two routes
+    are pinned equal on the CPU)."""
+    J, D = cfg["J"], cfg["D"]
+    n = cfg["K"] if n_rows is None else n_rows
+    rp = batch["rowptr"][:n + 1]
+    if int(rp[-1]) < 100000:
+        return orc.apply_sparse(np.zeros((J, D)), U[:n], rp, batch["idx"], batch["val"], -1.0)
+    A = _memo(cfg, "dense codes", lambda: orc.csr_to_dense(batch["rowptr"], batch["idx"], batch["val"], D))
+    return orc.delta_w(U[:n], A[:n])
+
+
 def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
     inputs = make_inputs(cfg)
     wl = _workload(cfg, inputs, path)
@@ -41,7 +68,7 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
     batch = batch_of(inputs, cfg, 0)
     try:
         # ---- factors -----------------------------------------------------------------------------
-        U_or, V_or, extra = oracle_factors(cfg, W0, batch)
+        U_or, V_or, extra = _memo(cfg, "factors at W0", lambda: oracle_factors(cfg, W0, batch))
         wl.compute_factors(0)
         torch.cuda.synchronize()
         U_gpu = to_f64(wl.U)[:, :J]
@@ -69,7 +96,7 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
         torch.cuda.synchronize()
         dW_gpu = to_f64(wl.W)
         if cfg["model"] == "sc":
-            dW_or = orc.apply_sparse(np.zeros((J, D)), U_gpu, batch["rowptr"], batch["idx"], batch["val"], -1.0)
+            dW_or = _sc_update_from_zero(cfg, U_gpu, batch)
         else:
             dW_or = orc.delta_w(U_gpu, V_or)
         e_dw = orc.rel_fro(dW_gpu, dW_or)
@@ -83,18 +110,21 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
             torch.cuda.synchronize()
             Bn = cfg["B"]
             if cfg["model"] == "sc":
-                rp = batch["rowptr"][:Bn + 1]
-                ref1 = orc.apply_sparse(np.zeros((J, D)), U_gpu[:Bn], rp, batch["idx"], batch["val"], -1.0)
+                ref1 = _sc_update_from_zero(cfg, U_gpu, batch, Bn)
             else:
                 ref1 = orc.delta_w(U_gpu[:Bn], V_or[:Bn])
             assert orc.rel_fro(to_f64(wl.W), ref1) <= tol
             assert_lines(to_f64(wl.W), ref1, tol, "U^T V of the first worker")
         # ---- steps: W_T - W_0 against the oracle's trajectory ----------------------------------------
-        W_or = W0.astype(np.float64)
-        for t in range(steps):
-            bt = batch_of(inputs, cfg, t % cfg["pool"])
-            U_t, V_t, _ = oracle_factors(cfg, W_or, bt)
-            W_or = oracle_apply(cfg, W_or, U_t, V_t, bt, eta)
+        def trajectory():
+            W_t = W0.astype(np.float64)
+            for t in range(steps):
+                bt = batch_of(inputs, cfg, t % cfg["pool"])
+                U_t, V_t, _ = oracle_factors(cfg, W_t, bt)
+                W_t = oracle_apply(cfg, W_t, U_t, V_t, bt, eta)
+            return W_t
+        # (DML is checked step by step from the GPU's own state below: no free-running trajectory)
+        W_or = None if cfg["model"] == "dml" else _memo(cfg, ("trajectory", float(eta), steps), trajectory)
         runs = []
         for rep in range(2):
             wl.reset()
