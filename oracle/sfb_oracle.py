@@ -21,6 +21,10 @@ What each function follows:
   else 0); v_i = a_i.
 * SC (Section 2, Figure 3): f_i = 1/2 ||W a_i - x_i||^2, u_i = W a_i - x_i,
   v_i = a_i (sparse code, an input here).
+* SDCA for L2-regularised MLR (Section 2.1): the update of the auxiliary matrix is
+  also rank one, (du_i, a_i); the paper gives no closed form for du_i, so
+  sdca_mlr_factors follows a stated reading: PARITY UNPINNED by the paper, pinned
+  by the fixed point, the primal-dual link and convergence to the primal optimum.
 
 All arithmetic is fp64 on inputs promoted exactly from their stored fp32 (or
 bf16-valued fp32) bytes.  One exception fixed by the wire format: the DML pair
@@ -78,6 +82,25 @@ def mlr_loss(W, X, labels):
     m = Z.max(axis=1)
     lse = m + np.log(np.exp(Z - m[:, None]).sum(axis=1))
     return float((lse - Z[np.arange(Z.shape[0]), np.asarray(labels, dtype=np.int64)]).sum())
+
+
+def sdca_mlr_factors(W, X, labels, dual, step):
+    """Mini-batch SDCA step for L2-regularised MLR (Section 2.1, "Stochastic DCA"; the L2-MLR workload of Section 6).
+
+    Primal: min_W (1/N) sum_i f_i(W x_i) + (lam/2) ||W||^2, f_i the multiclass logistic loss; dual variables u_i in
+    R^J, auxiliary matrix Z = (1/N) sum_i u_i x_i^T, W = grad h*(Z) = Z / lam.  At the optimum u_i = -grad f_i(W x_i).
+    The paper updates u_i <- u_i - du_i, Z <- Z - du_i x_i^T (with the 1/N of Z's definition) and leaves du_i to
+    "minimising (D) over u_i", which has no closed form for this loss.  READING (parity unpinned by the paper): the
+    damped step toward the coordinate's optimality condition,
+        du_i = step * (u_i + g_i),   g_i = softmax(W x_i) - onehot(y_i)   (the SGD factor of the same sample),
+    0 < step <= 1, all K samples of the mini-batch from the same W.  The update of W is then the same rank-K apply as
+    for SGD, W <- W - eta * sum_i du_i x_i^T with eta = 1 / (lam * N): the sufficient factors are (du_i, x_i).
+
+    dual: [K][J] current dual variables of the mini-batch's samples.  Returns (dU [K][J], V [K][D], new dual [K][J]).
+    """
+    G, V = mlr_factors(W, X, labels)
+    dU = float(step) * (_f64(dual) + G)
+    return dU, V, _f64(dual) - dU
 
 
 def dml_difference(Xa, Xb):

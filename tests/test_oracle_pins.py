@@ -494,3 +494,47 @@ def test_compaction_leaves_the_update_unchanged_and_round_trips():
     with pytest.raises(ValueError):
         orc.pack(orc.MODEL_SC, orc.DTYPE_F32, J, D, P, B, U, csr=(np.zeros(K + 1, np.uint32), np.zeros(0, np.uint32),
                                                                    np.zeros(0, np.float32)), nnz_capacity=32 * P, compact=True)
+
+
+# ----------------------------------------------------------------------------- SDCA for L2-regularised MLR
+def test_sdca_fixed_point_link_and_convergence():
+    """The SDCA factor rule is a reading (the paper gives no closed form), so it is pinned by what any correct dual
+    coordinate method must satisfy: (1) at u_i = -grad f_i the step is zero; (2) W = (1 / (lam N)) sum_i u_i x_i^T
+    holds after every step when W is updated by the rank-K apply with eta = 1 / (lam N); (3) the iterates converge to
+    the primal optimum, checked through the primal optimality condition written with independent loops:
+    (1/N) sum_i (softmax(W x_i) - e_{y_i}) x_i^T + lam W = 0."""
+    rng = np.random.default_rng(5)
+    N, J, D, K, lam, step = 12, 4, 6, 3, 0.1, 0.5
+    X = rng.standard_normal((N, D)).astype(np.float32)
+    y = rng.integers(0, J, N).astype(np.int32)
+    W = np.zeros((J, D))
+    dual = np.zeros((N, J))
+    # (1) fixed point
+    G, _ = orc.mlr_factors(W, X[:K], y[:K])
+    dU, V, new = orc.sdca_mlr_factors(W, X[:K], y[:K], -G, step)
+    assert np.abs(dU).max() == 0.0 and np.array_equal(new, -G) and np.array_equal(V, X[:K].astype(np.float64))
+    # first step from zero duals is a damped gradient step: du = step * g
+    dU, _, new = orc.sdca_mlr_factors(W, X[:K], y[:K], np.zeros((K, J)), step)
+    assert np.allclose(dU, step * G, rtol=0, atol=1e-16) and np.allclose(new, -step * G, rtol=0, atol=1e-16)
+    eta = 1.0 / (lam * N)
+    for epoch in range(400):
+        for b in range(0, N, K):
+            sl = slice(b, b + K)
+            dU, V, dual[sl] = orc.sdca_mlr_factors(W, X[sl], y[sl], dual[sl], step)
+            W = orc.apply_dense(W, dU, V, eta)
+        if epoch % 100 == 0:   # (2) primal-dual link
+            link = (dual.T @ X.astype(np.float64)) / (lam * N)
+            assert np.abs(W - link).max() <= 1e-13
+    # (3) primal optimality by loops
+    grad = [[lam * W[j][d] for d in range(D)] for j in range(J)]
+    for i in range(N):
+        p = loop_softmax(loop_matvec(W.tolist(), X[i].astype(np.float64).tolist()))
+        for j in range(J):
+            g = p[j] - (1.0 if j == y[i] else 0.0)
+            for d in range(D):
+                grad[j][d] += g * float(X[i][d]) / N
+    assert max(abs(v) for row in grad for v in row) <= 1e-9
+    assert np.abs(W).max() > 0.05          # a non-trivial optimum
+    # at the optimum the duals are minus the gradients of the losses
+    G, _ = orc.mlr_factors(W, X, y)
+    assert np.abs(dual + G).max() <= 1e-7
