@@ -131,6 +131,9 @@ typedef struct sfb_aux {
   const uint32_t* idx;    /* SC: atom index of each nonzero, strictly ascending within a row */
   const void* val;        /* SC: value of each nonzero (fp32) */
   const void* Xdata;      /* SC: data vectors x_i, [K][J] fp32 */
+  void* dual;             /* MLR, optional: SDCA dual variables of the K samples (see below), DEVICE memory also for
+                             sfb_step_host, [K][J rounded up to 4] fp32, updated in place; NULL = SGD factors */
+  float sdca_step;        /* MLR with dual: damping of the dual step, in (0, 1] */
 } sfb_aux;
 
 /* Creates a context for one (model, path, shape).  `cuda_stream` is a cudaStream_t (NULL = the
@@ -152,7 +155,16 @@ int sfb_ld(const sfb_desc* desc, int32_t* ldu, int32_t* ldv);
  *   DML  d = x - xb, z = W d, u = +z (similar) | -z*[|z|^2 < margin] (dissimilar), v = d
  *   SC   z = W a (a = CSR code), u = z - xdata,                          v = a (not copied here)
  * W [J][D] fp32; X [K][D] (fp32, or bf16 on SFB_PATH_BF16); U out [K][ldu]; V out [K][ldv]
- * (V may be NULL for SC and is ignored).  Pad columns of U and V are written as zeros. */
+ * (V may be NULL for SC and is ignored).  Pad columns of U and V are written as zeros.
+ *
+ * SDCA for L2-regularised MLR (Section 2.1, "Stochastic DCA": dual variables u_i, auxiliary matrix
+ * Z = (1/N) sum_i u_i a_i^T, W = Z / lambda, and the update of Z is again an outer product (du_i, a_i)).  With
+ * aux->dual set the factors are the dual steps of the K samples, all from the same W,
+ *   du_i = sdca_step * (dual_i + softmax(W x_i) - onehot(y_i)),   dual_i <- dual_i - du_i,   v_i = x_i
+ * (the paper leaves du_i to "minimising the dual over u_i", which has no closed form for this loss: this damped
+ * step toward the coordinate's optimality condition dual_i = -grad f_i is this library's reading), and the caller
+ * applies them with eta = 1 / (lambda N): W <- W - eta sum_i du_i x_i^T keeps W = (1 / (lambda N)) sum_i dual_i x_i^T.
+ * A sample with a label outside [0, J) takes no step. */
 int sfb_compute_factors(sfb_ctx* ctx, const void* W, const void* X, const sfb_aux* aux, void* U, void* V);
 
 /* Lays K (u, v) pairs out as P worker streams with header and directory: what the workers would

@@ -37,7 +37,8 @@ class sfb_desc(C.Structure):
 
 class sfb_aux(C.Structure):
     _fields_ = [("labels", C.c_void_p), ("Xb", C.c_void_p), ("similar", C.c_void_p), ("rowptr", C.c_void_p),
-                ("idx", C.c_void_p), ("val", C.c_void_p), ("Xdata", C.c_void_p)]
+                ("idx", C.c_void_p), ("val", C.c_void_p), ("Xdata", C.c_void_p), ("dual", C.c_void_p),
+                ("sdca_step", C.c_float)]
 
 
 class SfbError(RuntimeError):
@@ -134,8 +135,10 @@ def _ptr(t) -> int | None:
     return t.data_ptr()
 
 
-def make_aux(labels=None, Xb=None, similar=None, rowptr=None, idx=None, val=None, Xdata=None) -> sfb_aux:
-    return sfb_aux(_ptr(labels), _ptr(Xb), _ptr(similar), _ptr(rowptr), _ptr(idx), _ptr(val), _ptr(Xdata))
+def make_aux(labels=None, Xb=None, similar=None, rowptr=None, idx=None, val=None, Xdata=None, dual=None,
+             sdca_step=0.0) -> sfb_aux:
+    return sfb_aux(_ptr(labels), _ptr(Xb), _ptr(similar), _ptr(rowptr), _ptr(idx), _ptr(val), _ptr(Xdata), _ptr(dual),
+                   float(sdca_step))
 
 
 def sfb_sf_buffer_bytes(desc: sfb_desc) -> int:

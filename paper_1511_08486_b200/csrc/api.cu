@@ -125,7 +125,10 @@ CsrView stream_codes(const sfb_ctx* c, const void* sf_buf) {
 int check_aux(const sfb_ctx* c, const sfb_aux* a) {
   if (a == nullptr) return SFB_ERR_ARG;
   switch (c->d.model) {
-    case SFB_MLR: return (a->labels != nullptr && aligned(a->labels, 4)) ? SFB_OK : SFB_ERR_ARG;
+    case SFB_MLR:
+      if (a->labels == nullptr || !aligned(a->labels, 4)) return SFB_ERR_ARG;
+      if (a->dual != nullptr && (!aligned(a->dual, 16) || !(a->sdca_step > 0.f && a->sdca_step <= 1.f))) return SFB_ERR_ARG;
+      return SFB_OK;
     case SFB_DML: return (a->Xb != nullptr && a->similar != nullptr && aligned(a->Xb, 16)) ? SFB_OK : SFB_ERR_ARG;
     default:
       return (a->rowptr && a->idx && a->val && a->Xdata && aligned(a->rowptr, 4) && aligned(a->idx, 4) &&
@@ -188,7 +191,9 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
                              c->f32_splits, &ks));
     }
     const RowMap zsrc = ks > 1 ? part : u;
-    if (d.model == SFB_MLR) ACC(launch_finish_mlr(c->stream, zsrc, u, aux->labels, K, d.J, c->dev_status, ks, sstride));
+    if (d.model == SFB_MLR)
+      ACC(launch_finish_mlr(c->stream, zsrc, u, aux->labels, K, d.J, c->dev_status, ks, sstride,
+                            reinterpret_cast<float*>(aux->dual), aux->sdca_step));
     else ACC(launch_finish_dml(c->stream, zsrc, u, aux->similar, d.margin, K, d.J, ks, sstride, c->dml_active));
     return SFB_OK;
   }
@@ -734,6 +739,8 @@ int sfb_step_host(sfb_ctx* c, void* W, const void* X_host, const sfb_aux* aux_ho
     if (aux_host->labels == nullptr) return SFB_ERR_ARG;
     if ((r = stage_in(c, set, 1, aux_host->labels, Kt * 4, &p)) != SFB_OK) return r;
     dev_aux.labels = static_cast<const int32_t*>(p);
+    dev_aux.dual = aux_host->dual;          // SDCA state lives on the device
+    dev_aux.sdca_step = aux_host->sdca_step;
   } else if (d.model == SFB_DML) {
     if (aux_host->Xb == nullptr || aux_host->similar == nullptr) return SFB_ERR_ARG;
     if ((r = stage_in(c, set, 1, aux_host->Xb, Kt * d.D * es, &p)) != SFB_OK) return r;

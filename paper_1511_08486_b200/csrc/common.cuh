@@ -98,8 +98,10 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
 
 // MLR epilogue: u = softmax(z) - onehot(label).  z rows are fp32; u rows fp32 or bf16 (u.es).
 // z may be `nsplit` partial products (split s at z + s * split_stride_bytes), summed in split order.
+// dual (optional, SDCA): fp32 dual variables of the K samples, [K][J rounded up to 4], updated in place; the factor
+// written to u is then the dual step sdca_step * (dual + softmax - onehot).
 int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
-                      int nsplit = 1, long long split_stride_bytes = 0);
+                      int nsplit = 1, long long split_stride_bytes = 0, float* dual = nullptr, float sdca_step = 0.f);
 
 // DML epilogue: u = +z (similar) or -z * [|z|^2 < margin] (dissimilar).
 // active (optional, [K] bytes): 1 where the pair contributes (similar, or dissimilar inside the margin), 0 where u_i = 0.

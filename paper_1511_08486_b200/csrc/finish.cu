@@ -68,8 +68,26 @@ __device__ __forceinline__ void store_u4(char* row, int j, float4 v, int es) {
 }
 
 // z rows are fp32 with ld a multiple of 4; values beyond J inside the last float4 are ignored.
+// SDCA (dual != nullptr; Section 2.1, "Stochastic DCA"): the factor is the damped dual step
+// du_i = step * (dual_i + g_i) with g_i = softmax(z_i) - onehot(y_i), and dual_i <- dual_i - du_i in place
+// (dual rows: fp32, ldd = J rounded up to 4 values per row, pad values written as zeros).
+__device__ __forceinline__ float4 sdca_step4(float* dual_row, int j, int J, float4 g, float step, bool bad) {
+  float4 d = *reinterpret_cast<const float4*>(dual_row + j);
+  float4 du = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (!bad) {   // a sample with a bad label takes no step: its dual variables stay as they are
+    du.x = step * (d.x + g.x); du.y = step * (d.y + g.y); du.z = step * (d.z + g.z); du.w = step * (d.w + g.w);
+    d.x -= du.x; d.y -= du.y; d.z -= du.z; d.w -= du.w;
+  }
+  if (j + 1 >= J) { du.y = 0.f; d.y = 0.f; }
+  if (j + 2 >= J) { du.z = 0.f; d.z = 0.f; }
+  if (j + 3 >= J) { du.w = 0.f; d.w = 0.f; }
+  *reinterpret_cast<float4*>(dual_row + j) = d;
+  return du;
+}
+
 __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, const int32_t* __restrict__ labels,
-                                                                 int K, int J, int cache_floats, int* dev_status, int nsplit, long long zstride) {
+                                                                 int K, int J, int cache_floats, int* dev_status, int nsplit, long long zstride,
+                                                                 float* __restrict__ dual, float sdca_step) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -137,6 +155,7 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
       if (j + 2 >= J) t.z = 0.f;
       if (j + 3 >= J) t.w = 0.f;
     }
+    if (dual != nullptr && q < J4) t = sdca_step4(dual + (size_t)i * (J4 * 4), j, J, t, sdca_step, bad);
     store_u4(ur, j, t, u.es);
   }
 }
@@ -189,7 +208,8 @@ __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, co
 template <int ES>
 __global__ void __launch_bounds__(256) finish_mlr_fused_kernel(RowMap u, const float2* __restrict__ stats, int n_parts,
                                                                int part_cols, const int32_t* __restrict__ labels, int K,
-                                                               int J, int* dev_status) {
+                                                               int J, int* dev_status, float* __restrict__ dual,
+                                                               float sdca_step) {
   extern __shared__ float scale[];   // [n_parts]
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -234,6 +254,17 @@ __global__ void __launch_bounds__(256) finish_mlr_fused_kernel(RowMap u, const f
       if (j + e == y) r -= 1.f;
       if (j + e >= J || bad) r = 0.f;
       vals[e] = r;
+    }
+    if (dual != nullptr && j < J) {   // SDCA: the factor becomes the dual step, the dual variables move by it
+      float* drow = dual + (size_t)i * (((J + 3) >> 2) * 4);
+#pragma unroll
+      for (int e4 = 0; e4 < PER; e4 += 4) {
+        if (j + e4 < J) {
+          const float4 du = sdca_step4(drow, j + e4, J, make_float4(vals[e4], vals[e4 + 1], vals[e4 + 2], vals[e4 + 3]),
+                                       sdca_step, bad);
+          vals[e4] = du.x; vals[e4 + 1] = du.y; vals[e4 + 2] = du.z; vals[e4 + 3] = du.w;
+        }
+      }
     }
     if (ES == 4) {
       float* f4 = reinterpret_cast<float*>(&raw);
@@ -350,14 +381,15 @@ int fin_cache_floats(int J) {
 }  // namespace
 
 int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
-                      int nsplit, long long split_stride_bytes) {
+                      int nsplit, long long split_stride_bytes, float* dual, float sdca_step) {
   const int cf = fin_cache_floats(J);
   static PerDeviceOnce attr_once;   // function attributes are per device
   if (attr_once.first()) {
     cudaFuncSetAttribute(finish_mlr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
   }
-  finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status, nsplit, split_stride_bytes / 4);
+  finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status, nsplit, split_stride_bytes / 4,
+                                                              dual, sdca_step);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
@@ -409,11 +441,13 @@ int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar
 }
 
 int launch_finish_mlr_fused(cudaStream_t s, RowMap u, const float2* stats, int n_parts, int part_cols,
-                            const int32_t* labels, int K, int J, int* dev_status) {
+                            const int32_t* labels, int K, int J, int* dev_status, float* dual, float sdca_step) {
   const size_t smem = (size_t)n_parts * sizeof(float);
   if (smem > 48 * 1024) return SFB_ERR_SHAPE;
-  if (u.es == 4) finish_mlr_fused_kernel<4><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status);
-  else finish_mlr_fused_kernel<2><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status);
+  if (u.es == 4)
+    finish_mlr_fused_kernel<4><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status, dual, sdca_step);
+  else
+    finish_mlr_fused_kernel<2><<<K, 256, smem, s>>>(u, stats, n_parts, part_cols, labels, K, J, dev_status, dual, sdca_step);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

@@ -27,7 +27,7 @@ namespace sfb {
 
 // extra passes implemented in finish.cu
 int launch_finish_mlr_fused(cudaStream_t s, RowMap u, const float2* stats, int n_parts, int part_cols,
-                            const int32_t* labels, int K, int J, int* dev_status);
+                            const int32_t* labels, int K, int J, int* dev_status, float* dual, float sdca_step);
 
 namespace {
 
@@ -1066,7 +1066,9 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
                                    nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
           return r;
         launches += r;
-        if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride)) < 0) return r;
+        if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride, reinterpret_cast<float*>(aux->dual),
+                                   aux->sdca_step)) < 0)
+          return r;
         launches += r;
       } else {
         int n_parts = 0, part_cols = 0;
@@ -1074,7 +1076,8 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
                                    &part_cols, nullptr, 1, 0, workers)) < 0)
           return r;
         launches += r;
-        if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status)) < 0)
+        if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status,
+                                         reinterpret_cast<float*>(aux->dual), aux->sdca_step)) < 0)
           return r;
         launches += r;
       }
