@@ -973,6 +973,10 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   p.k_splits = may_split ? ks_pick : 1;
   if (k_splits_out != nullptr) *k_splits_out = p.k_splits;
   p.k_per_split = (p.k_blocks + p.k_splits - 1) / p.k_splits;
+  // no empty range: a work item without reduction blocks would never signal its accumulator (and the finishing pass
+  // would add a partial buffer nobody wrote)
+  p.k_splits = (p.k_blocks + p.k_per_split - 1) / p.k_per_split;
+  if (k_splits_out != nullptr) *k_splits_out = p.k_splits;
   p.split_stride = split_stride;
   // the operand that does not fit in L2 should stream from HBM once: consecutive tiles share its slab
   p.m_fastest = ((long long)d.J * d.D > (long long)P * d.B * d.D) ? 1 : 0;

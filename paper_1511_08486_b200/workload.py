@@ -42,11 +42,39 @@ def shard_batch(t: dict, model: str, first_worker: int, n_workers: int, Bsz: int
     return s
 
 
-class DeviceWorkload:
-    """Device copies of the inputs of configuration `cfg`, a context, and the SF buffer."""
+GUARD_BYTES = 4096
 
-    def __init__(self, cfg: dict, inputs: dict, path: str | None = None, device="cuda:0", stream=None):
+
+class Guarded:
+    """A device tensor placed between two guard bands of GUARD_BYTES bytes each, filled with 0xFF (a NaN pattern in
+    fp32 and bf16).  `t` is the usable tensor (128-byte aligned); `intact()` tells whether both bands still hold
+    their pattern.  A stray write lands in a band and is seen there; a stray read that feeds arithmetic turns the
+    result into NaN."""
+
+    def __init__(self, shape, dtype, device, fill=None):
+        n = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        self.raw = torch.full((n + 2 * GUARD_BYTES,), 0xFF, dtype=torch.uint8, device=device)
+        self.n = n
+        self.t = self.raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(*shape)
+        if fill is not None:
+            self.t.copy_(fill)
+        else:
+            self.t.zero_()
+
+    def intact(self) -> bool:
+        lo, hi = self.raw[:GUARD_BYTES], self.raw[GUARD_BYTES + self.n:]
+        return bool((lo == 0xFF).all().item()) and bool((hi == 0xFF).all().item())
+
+
+class DeviceWorkload:
+    """Device copies of the inputs of configuration `cfg`, a context, and the SF buffer.
+
+    guard=True puts every tensor the library writes (W, the SF buffer, U, V) between guard bands
+    (`guards_intact()` checks them) for tests that look for out-of-range accesses."""
+
+    def __init__(self, cfg: dict, inputs: dict, path: str | None = None, device="cuda:0", stream=None, guard=False):
         self.cfg, self.device = cfg, torch.device(device)
+        self._guards = []
         self.path = path or cfg["path"]
         model = cfg["model"]
         self.model = model
@@ -60,7 +88,7 @@ class DeviceWorkload:
         self.ldu, self.ldv = self.ctx.ldu, self.ctx.ldv
         dev = self.device
         self.W0 = torch.from_numpy(inputs["W"]).to(dev)
-        self.W = self.W0.clone()
+        self.W = self._alloc(self.W0.shape, torch.float32, guard, fill=self.W0)
         bf16 = self.path == "bf16"
         self.val_dtype = torch.bfloat16 if bf16 else torch.float32
         self.batches = []
@@ -83,9 +111,19 @@ class DeviceWorkload:
                 t["Xdata"] = torch.from_numpy(inputs["Xdata"][b]).to(dev)
                 t["aux"] = B.make_aux(rowptr=t["rowptr"], idx=t["idx"], val=t["val"], Xdata=t["Xdata"])
             self.batches.append(t)
-        self.sf_buf = torch.zeros(self.ctx.sf_buffer_bytes, dtype=torch.uint8, device=dev)
-        self.U = torch.zeros(self.K, self.ldu, dtype=self.val_dtype, device=dev)
-        self.V = None if sparse else torch.zeros(self.K, self.ldv, dtype=self.val_dtype, device=dev)
+        self.sf_buf = self._alloc((self.ctx.sf_buffer_bytes,), torch.uint8, guard)
+        self.U = self._alloc((self.K, self.ldu), self.val_dtype, guard)
+        self.V = None if sparse else self._alloc((self.K, self.ldv), self.val_dtype, guard)
+
+    def _alloc(self, shape, dtype, guard, fill=None):
+        if not guard:
+            return fill.clone() if fill is not None else torch.zeros(*shape, dtype=dtype, device=self.device)
+        g = Guarded(tuple(shape), dtype, self.device, fill)
+        self._guards.append(g)
+        return g.t
+
+    def guards_intact(self) -> bool:
+        return all(g.intact() for g in self._guards)
 
     def reset(self):
         self.W.copy_(self.W0)

@@ -16,9 +16,9 @@ from tests.util import (MAX_STORAGE_OVER_TOL, MODEL_ID, TOL, assert_lines, batch
 pytestmark = pytest.mark.gpu
 
 
-def _workload(cfg, inputs, path):
+def _workload(cfg, inputs, path, guard=False):
     from paper_1511_08486_b200.workload import DeviceWorkload
-    return DeviceWorkload(cfg, inputs, path=path)
+    return DeviceWorkload(cfg, inputs, path=path, guard=guard)
 
 
 def _wire_dtype(path):
@@ -58,9 +58,10 @@ def _sc_update_from_zero(cfg, U, batch, n_rows=None):
     return orc.delta_w(U[:n], A[:n])
 
 
-def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
+def check_config(cfg, path, eta=None, steps=2, check_v_exact=True, guard=False):
+    """guard: W, the SF buffer, U and V sit between guard bands of NaN patterns that must survive every call."""
     inputs = make_inputs(cfg)
-    wl = _workload(cfg, inputs, path)
+    wl = _workload(cfg, inputs, path, guard=guard)
     tol = TOL[path]
     J, D, K = cfg["J"], cfg["D"], cfg["K"]
     eta = cfg["eta"] if eta is None else eta
@@ -176,6 +177,7 @@ def check_config(cfg, path, eta=None, steps=2, check_v_exact=True):
         h, U_last, _ = orc.unpack(runs[0][1])
         assert h["clock"] == steps - 1 and h["P"] == cfg["P"] and h["J"] == J
         assert wl.ctx.status() == 0
+        assert wl.guards_intact(), "a kernel wrote outside W, the SF buffer, U or V"
         return dict(e_u=e_u, e_dw=e_dw, e_step=e_step)
     finally:
         wl.close()

@@ -30,6 +30,13 @@ def test_x3_pairs_ragged_and_short_streams():
         check_config(_cfg("C1", J=J, D=D, P=P, B=B, pool=1), "tf32x3", eta=0.5, steps=2)
 
 
+def test_x3_reduction_ranges_never_come_out_empty():
+    """42 atoms of reduction cut for 8 ranges give ranges of 6 atoms, of which only 7 exist: the eighth must not be
+    launched (found by the shape sweep as a bounded-wait time-out of the forward pass)."""
+    check_config(_cfg("C1", J=100, D=1312, P=2, B=130, pool=1), "tf32x3", eta=0.5, steps=2)
+    check_config(_cfg("C2", J=2, D=1304, P=2, B=20), "tf32x3", eta=1e-3, steps=1)
+
+
 def test_x3_dml():
     check_config(_cfg("C2", J=72, D=1000, P=3, B=20), "tf32x3", eta=1e-3, steps=2)
     check_config(_cfg("C2", J=600, D=2000, P=8, B=32), "tf32x3", eta=1e-4, steps=2)
