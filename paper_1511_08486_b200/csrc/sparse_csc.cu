@@ -13,6 +13,8 @@
 // in a private 16 x 65 tile, and finally updates W with 64-byte row segments.
 // U is read once and W once per slice; no floating-point atomics; every element of W has one owner and a fixed
 // summation order (bit-reproducible); atoms nobody uses get W + (-eta * 0) = W, bit-identical.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace sfb {
@@ -217,18 +219,26 @@ __global__ void __launch_bounds__(512) csc_apply_kernel(float* __restrict__ W, R
           const int nxt = (base + 32 < stop) ? base + 32 : next_beg;
           if (nxt + lane < nnz) { pre_i = ent_i[nxt + lane]; pre_a = ent_a[nxt + lane]; }
           __syncwarp();
+          // a round holds up to 32 entries; short columns (sparse codes) take the 8- or 16-entry body, so the time of
+          // a column follows its entries, not the round size (the bodies are unrolled: no branch inside them)
+          const int n_here = min(32, stop - base);     // warp-uniform
+          auto body = [&](auto iters) {
 #pragma unroll
-          for (int k = 0; k < 16; k += 2) {
-            const int4 p = strip4[k], q = strip4[k + 1];
-            const float2 u0 = *reinterpret_cast<const float2*>(Us + p.x * 64 + 2 * lane);
-            const float2 u1 = *reinterpret_cast<const float2*>(Us + p.z * 64 + 2 * lane);
-            const float2 u2 = *reinterpret_cast<const float2*>(Us + q.x * 64 + 2 * lane);
-            const float2 u3 = *reinterpret_cast<const float2*>(Us + q.z * 64 + 2 * lane);
-            acc0.x = fmaf(__int_as_float(p.y), u0.x, acc0.x); acc0.y = fmaf(__int_as_float(p.y), u0.y, acc0.y);
-            acc1.x = fmaf(__int_as_float(p.w), u1.x, acc1.x); acc1.y = fmaf(__int_as_float(p.w), u1.y, acc1.y);
-            acc2.x = fmaf(__int_as_float(q.y), u2.x, acc2.x); acc2.y = fmaf(__int_as_float(q.y), u2.y, acc2.y);
-            acc3.x = fmaf(__int_as_float(q.w), u3.x, acc3.x); acc3.y = fmaf(__int_as_float(q.w), u3.y, acc3.y);
-          }
+            for (int k = 0; k < decltype(iters)::value; k += 2) {
+              const int4 p = strip4[k], q = strip4[k + 1];
+              const float2 u0 = *reinterpret_cast<const float2*>(Us + p.x * 64 + 2 * lane);
+              const float2 u1 = *reinterpret_cast<const float2*>(Us + p.z * 64 + 2 * lane);
+              const float2 u2 = *reinterpret_cast<const float2*>(Us + q.x * 64 + 2 * lane);
+              const float2 u3 = *reinterpret_cast<const float2*>(Us + q.z * 64 + 2 * lane);
+              acc0.x = fmaf(__int_as_float(p.y), u0.x, acc0.x); acc0.y = fmaf(__int_as_float(p.y), u0.y, acc0.y);
+              acc1.x = fmaf(__int_as_float(p.w), u1.x, acc1.x); acc1.y = fmaf(__int_as_float(p.w), u1.y, acc1.y);
+              acc2.x = fmaf(__int_as_float(q.y), u2.x, acc2.x); acc2.y = fmaf(__int_as_float(q.y), u2.y, acc2.y);
+              acc3.x = fmaf(__int_as_float(q.w), u3.x, acc3.x); acc3.y = fmaf(__int_as_float(q.w), u3.y, acc3.y);
+            }
+          };
+          if (n_here <= 8) body(std::integral_constant<int, 4>());
+          else if (n_here <= 16) body(std::integral_constant<int, 8>());
+          else body(std::integral_constant<int, 16>());
           __syncwarp();
         }
         T[dd * 65 + 2 * lane] = (acc0.x + acc1.x) + (acc2.x + acc3.x);
