@@ -74,7 +74,9 @@
  *   count and flags bit 1 is set.  Offsets and strides are those of the full buffer: a sender transmits the
  *   first n_sf rows of each block (sfb_wire_bytes counts them), a receiver reads them in place.  sfb_pack and
  *   sfb_step compact, sfb_apply leaves out the reduction blocks that hold only empty slots; W' is the same
- *   sum (bit-identical on SFB_PATH_F32).  Not available with sparse v or sfb_factors_shard.
+ *   sum (bit-identical on SFB_PATH_F32).  In the sharded step every process compacts the streams of its own
+ *   workers (sfb_factors_shard) before the exchange and sfb_commit_header rebuilds the pair counts from the streams
+ *   that arrived.  Not available with sparse v.
  */
 #ifndef SFB_H_
 #define SFB_H_

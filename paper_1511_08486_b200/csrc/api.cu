@@ -581,7 +581,6 @@ int sfb_factors_shard(sfb_ctx* c, const void* W, const void* X, const sfb_aux* a
   if (c == nullptr || W == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
   if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
   const sfb_desc& d = c->d;
-  if (d.compact) return SFB_ERR_UNSUPPORTED;   // the sharded step keeps every slot
   if (first_worker < 0 || n_workers <= 0 || first_worker > d.P - n_workers) return SFB_ERR_ARG;
   int r = check_aux(c, aux);
   if (r != SFB_OK) return r;
@@ -597,12 +596,18 @@ int sfb_factors_shard(sfb_ctx* c, const void* W, const void* X, const sfb_aux* a
                         c->dev_status));
     codes = stream_codes(c, shard);
   }
-  return factors_into(c, W, X, aux, stream_u(c, shard), d.v_sparse ? RowMap() : stream_v(c, shard), codes, n_workers);
+  r = factors_into(c, W, X, aux, stream_u(c, shard), d.v_sparse ? RowMap() : stream_v(c, shard), codes, n_workers);
+  if (r < 0) return r;
+  // a process compacts the streams of its own workers before they are sent
+  if (d.compact) ACC(launch_compact(c->stream, sf_buf, d, c->l, c->compact_ws, first_worker, n_workers));
+  return SFB_OK;
 }
 
 int sfb_commit_header(sfb_ctx* c, void* sf_buf, uint32_t clock) {
   if (c == nullptr || sf_buf == nullptr || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
   ACC(launch_write_header(c->stream, sf_buf, c->d, c->l, clock, nullptr));
+  // compacted streams: the directory is local, its pair counts are rebuilt from what the exchange brought
+  if (c->d.compact) ACC(launch_count_pairs(c->stream, sf_buf, c->d, c->l, c->compact_ws));
   return SFB_OK;
 }
 

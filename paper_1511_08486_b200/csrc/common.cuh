@@ -126,7 +126,10 @@ int launch_pack_csr(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layou
 // its "compacted" flag.  workspace: compact_workspace_bytes(K, P) bytes.  launch_kept_rows lists the slots
 // p * B + r, r < count of worker p, of the first `workers` workers (idx [K], n_out one int; device arrays).
 long long compact_workspace_bytes(int K, int P);
-int launch_compact(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace);
+int launch_compact(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace, int first_worker = 0,
+                   int n_workers = 0);   // n_workers > 0: only those workers' streams (a process's shard)
+// Rebuilds the directory's pair counts (and the header flag) from streams that arrived already compacted.
+int launch_count_pairs(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace);
 int launch_kept_rows(cudaStream_t s, const void* sf_buf, int B, int workers, int* idx, int* n_out);
 
 // Sets SFB_DEV_BAD_HEADER in *dev_status unless the buffer's header matches the descriptor.

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) row_nonzero_kernel(RowMap u, int K, int J
 // One block per worker: dest[i] = new slot of pair i inside its worker (-1: left out); the worker's count goes
 // to counts[p] and to the n_sf field of its directory entry; block 0 sets the header's "compacted" flag.
 __global__ void __launch_bounds__(256) compact_scan_kernel(const uint8_t* __restrict__ flags, int B, int* __restrict__ dest,
-                                                           int* __restrict__ counts, char* buf) {
+                                                           int* __restrict__ counts, char* buf, int first_worker) {
   __shared__ int warp_cnt[8];
   __shared__ int base;
   const int p = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -62,8 +62,8 @@ __global__ void __launch_bounds__(256) compact_scan_kernel(const uint8_t* __rest
   }
   if (threadIdx.x == 0) {
     counts[p] = base;
-    reinterpret_cast<uint32_t*>(buf + 128 + (size_t)p * 32)[1] = (uint32_t)base;   // directory: n_sf
-    if (p == 0) reinterpret_cast<uint32_t*>(buf)[2] |= 2u;                           // header flags, bit 1
+    reinterpret_cast<uint32_t*>(buf + 128 + (size_t)(first_worker + p) * 32)[1] = (uint32_t)base;   // directory: n_sf
+    if (p == 0) reinterpret_cast<uint32_t*>(buf)[2] |= 2u;                                            // header flags, bit 1
   }
 }
 
@@ -123,24 +123,73 @@ __global__ void __launch_bounds__(256) kept_rows_kernel(const char* buf, int B, 
   if (threadIdx.x == 0) *n_out = base;
 }
 
+// One block per worker: n_sf of its directory entry = number of its u rows flagged nonzero (in a compacted stream
+// the kept pairs are exactly the leading rows); block 0 sets the header's "compacted" flag.
+__global__ void __launch_bounds__(256) count_pairs_kernel(const uint8_t* __restrict__ flags, int B, char* buf) {
+  __shared__ int total;
+  if (threadIdx.x == 0) total = 0;
+  __syncthreads();
+  const int p = blockIdx.x;
+  int n = 0;
+  for (int r = threadIdx.x; r < B; r += 256) n += flags[(size_t)p * B + r] != 0 ? 1 : 0;
+  for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+  if ((threadIdx.x & 31) == 0) atomicAdd(&total, n);   // integer: the order does not matter
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    reinterpret_cast<uint32_t*>(buf + 128 + (size_t)p * 32)[1] = (uint32_t)total;
+    if (p == 0) reinterpret_cast<uint32_t*>(buf)[2] |= 2u;
+  }
+}
+
+struct Scratch {
+  uint8_t* flags; int* dest; int* counts;
+};
+// flags [K] bytes, new slots [K] ints, per-worker counts [P] ints; offsets fixed by the full K = P * B
+Scratch scratch(void* workspace, int K) {
+  Scratch w;
+  w.flags = reinterpret_cast<uint8_t*>(workspace);
+  w.dest = reinterpret_cast<int*>(reinterpret_cast<char*>(workspace) + pad_to(K, 256));
+  w.counts = reinterpret_cast<int*>(reinterpret_cast<char*>(w.dest) + pad_to((long long)K * 4, 256));
+  return w;
+}
+
 }  // namespace
 
-long long compact_workspace_bytes(int K, int P) { return pad_to((long long)K, 256) + pad_to((long long)K * 4, 256) + pad_to((long long)P * 4, 256); }
+long long compact_workspace_bytes(int K, int P) {
+  return pad_to((long long)K, 256) + pad_to((long long)K * 4, 256) + pad_to((long long)P * 4, 256);
+}
 
-int launch_compact(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace) {
+// Directory pair counts of a buffer whose streams were compacted elsewhere (each process of a sharded step compacts
+// the streams of its own workers before the exchange; the directory is local and is rebuilt from what arrived).
+int launch_count_pairs(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace) {
   const int K = d.P * d.B;
-  uint8_t* flags = reinterpret_cast<uint8_t*>(workspace);
-  int* dest = reinterpret_cast<int*>(reinterpret_cast<char*>(workspace) + pad_to(K, 256));
-  int* counts = reinterpret_cast<int*>(reinterpret_cast<char*>(dest) + pad_to((long long)K * 4, 256));
+  const Scratch w = scratch(workspace, K);
   char* buf = reinterpret_cast<char*>(sf_buf);
   RowMap u;
   u.base = buf + l.streams_off; u.worker_stride = l.stream_stride; u.ld = l.ldu; u.B = d.B; u.es = l.es;
-  row_nonzero_kernel<<<(K + 7) / 8, 256, 0, s>>>(u, K, d.J, flags);
-  compact_scan_kernel<<<d.P, 256, 0, s>>>(flags, d.B, dest, counts, buf);
+  row_nonzero_kernel<<<(K + 7) / 8, 256, 0, s>>>(u, K, d.J, w.flags);
+  count_pairs_kernel<<<d.P, 256, 0, s>>>(w.flags, d.B, buf);
+  return cudaGetLastError() == cudaSuccess ? 2 : SFB_ERR_CUDA;
+}
+
+// first_worker / n_workers: compact only the streams of those workers (n_workers = 0: all P).  Worker indices
+// inside the kernels are relative to first_worker: streams, directory entries, flags, slots and counts alike
+// (counts[p] of the workspace belongs to worker first_worker + p).
+int launch_compact(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, void* workspace, int first_worker,
+                   int n_workers) {
+  if (n_workers <= 0) { first_worker = 0; n_workers = d.P; }
+  const int K = n_workers * d.B;
+  const Scratch w = scratch(workspace, d.P * d.B);
+  char* buf = reinterpret_cast<char*>(sf_buf);
+  char* streams = buf + l.streams_off + (long long)first_worker * l.stream_stride;
+  RowMap u;
+  u.base = streams; u.worker_stride = l.stream_stride; u.ld = l.ldu; u.B = d.B; u.es = l.es;
+  row_nonzero_kernel<<<(K + 7) / 8, 256, 0, s>>>(u, K, d.J, w.flags);
+  compact_scan_kernel<<<n_workers, 256, 0, s>>>(w.flags, d.B, w.dest, w.counts, buf, first_worker);
   const int u_units = l.ldu * l.es / 16, v_units = l.ldv * l.es / 16;
   const int u_slices = (u_units + SLICE_UNITS - 1) / SLICE_UNITS, v_slices = (v_units + SLICE_UNITS - 1) / SLICE_UNITS;
-  compact_move_kernel<<<dim3(d.P, u_slices + v_slices), 256, 0, s>>>(buf + l.streams_off, l.stream_stride, l.u_bytes, d.B,
-                                                                     u_units, v_units, u_slices, dest, counts);
+  compact_move_kernel<<<dim3(n_workers, u_slices + v_slices), 256, 0, s>>>(streams, l.stream_stride, l.u_bytes, d.B, u_units,
+                                                                           v_units, u_slices, w.dest, w.counts);
   return cudaGetLastError() == cudaSuccess ? 3 : SFB_ERR_CUDA;
 }
 

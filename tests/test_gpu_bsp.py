@@ -137,3 +137,43 @@ def test_bsp_bench_under_a_launcher_runs_the_nccl_exchange():
     assert out["scaling"] == "strong" and out["device_status"] == 0 and out["gpu_launches"] > 0
     assert out["config"]["parallelism"].startswith("bsp sfb")
     assert set(out["stages_ms"]) >= {"factors", "exchange", "apply"}
+
+
+@pytest.mark.parametrize("path,over", [("f32", dict(J=40, D=300, P=4, B=6)), ("f32", dict(J=128, D=1024, P=4, B=64)),
+                                       ("tf32", dict(J=64, D=512, P=4, B=64)), ("tf32x3", dict(J=260, D=1024, P=4, B=100))])
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_sharded_step_with_compaction(path, over, world):
+    """compact = 1: every process compacts the streams of its own workers before the exchange, the directory's pair
+    counts are rebuilt from the streams that arrived: same buffer (byte for byte: the kept pairs, their order and the
+    counts do not depend on who computed them) and same update as the single-process compacted step."""
+    cfg = scaled("C2", **over)
+    cfg["path"] = path
+    cfg["compact"] = 1
+    inputs = make_inputs(cfg)
+    wl = _workload(cfg, inputs, path)
+    try:
+        eta = 1e-3
+        wl.step(0, eta=eta)
+        torch.cuda.synchronize()
+        W_ref, buf_ref = wl.W.clone(), wl.sf_buf.clone()
+        h_ref, U_ref, V_ref = orc.unpack(buf_ref.cpu().numpy())
+        assert h_ref["flags"] == orc.FLAG_COMPACT and 0 < sum(h_ref["n_sf"]) < cfg["K"]
+        wl.reset()
+        wl.sf_buf.zero_()
+        t = wl.batches[0]
+        for rank in range(world):
+            first, n = worker_range(cfg["P"], world, rank)
+            s = shard_batch(t, cfg["model"], first, n, cfg["B"])
+            wl.ctx.factors_shard(wl.W, s["X"], s["aux"], wl.sf_buf, first, n)
+        wl.ctx.commit_header(wl.sf_buf, 0)
+        wl.ctx.apply(wl.W, wl.sf_buf, eta)
+        assert wl.ctx.status() == 0
+        h, U, V = orc.unpack(wl.sf_buf.cpu().numpy())
+        assert h == h_ref and np.array_equal(V, V_ref)
+        assert orc.rel_fro(U, U_ref) <= (1e-6 if path == "f32" else 0.1 * TOL[path])
+        if world == 1:
+            assert torch.equal(wl.sf_buf, buf_ref) and torch.equal(wl.W, W_ref)
+        dW, dW_ref = to_f64(wl.W) - to_f64(wl.W0), to_f64(W_ref) - to_f64(wl.W0)
+        assert orc.rel_fro(dW, dW_ref) <= (1e-5 if path == "f32" else 0.1 * TOL[path])
+    finally:
+        wl.close()

@@ -39,7 +39,7 @@ def _memo(cfg, tag, fn):
     path): computed once.  Keyed by everything that determines the synthetic inputs and the request."""
     key = (tag,) + tuple(sorted((k, repr(v)) for k, v in cfg.items() if k not in ("path", "compact")))
     if key not in _ORACLE_MEMO:
-        if len(_ORACLE_MEMO) > 4:
+        if len(_ORACLE_MEMO) > 8:
             _ORACLE_MEMO.clear()
         _ORACLE_MEMO[key] = fn()
     return _ORACLE_MEMO[key]
