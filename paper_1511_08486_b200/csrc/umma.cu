@@ -8,9 +8,11 @@
 //             the output index ("MN-major"); tcgen05 reads them in that form directly from the SF
 //             buffer's worker streams, no transposed copy is made.
 //
-// Warp roles (320 threads): warp 0 issues TMA loads into a 4-stage shared-memory ring, warp 1 issues
+// Warp roles (320 threads): warp 0 issues TMA loads into a shared-memory ring of 3 to 8 stages, warp 1 issues
 // the MMAs (one thread) into one of two TMEM accumulators, warps 2-9 drain the other accumulator
 // (tcgen05.ld) and run the epilogue, so the write-back of tile t overlaps the MMAs of tile t+1.
+// The error-compensated kernels (SPLIT, fp32-grade results from tf32 MMAs) add warps 10-13, which split every
+// operand stage into what the tensor core sees of it and the exact remainder.
 // Every wait on an mbarrier is bounded; a wait that runs out sets SFB_DEV_TIMEOUT and the CTA leaves
 // through the common exit (TMEM freed) instead of hanging.
 #include <cuda.h>
@@ -815,6 +817,9 @@ constexpr int STAGE_ATOMS = 2;
 // Compensated kernels: 128-byte atoms (32 fp32 reduction steps = 4 MMA instructions) one accumulator may take
 // before its range ends: 40 atoms = 160 roundings toward zero, about 2.6e-6 of the sum.
 constexpr int X3_ATOMS_PER_RANGE = 40;
+// ... and pairs one launch of the compensated apply takes (512 instructions: 8e-6 of the sum at worst, half of it
+// on average over a tile's life); larger updates are applied in several launches.
+constexpr int X3_PAIRS_PER_APPLY = 4096;
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   if (get_encode() == nullptr) return SFB_ERR_CUDA;
@@ -1120,8 +1125,37 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
   return launches + r;
 }
 
+static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows,
+                            float eta, int K, const int* dev_status, const void* directory);
+
 int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
                int K, const int* dev_status, const void* directory) {
+  const sfb_desc& d = pl->d;
+  if (pl->x3 && K > X3_PAIRS_PER_APPLY && K > d.B) {
+    // The accumulator of a tile rounds toward zero once per 8 pairs (about 1.6e-8 of the sum each time), so an update
+    // of very many pairs goes to W in several launches of whole worker streams, each added to W in fp32 by the
+    // epilogue: more traffic on W, an error that stops growing with K.
+    const int workers = K / d.B;
+    int per = X3_PAIRS_PER_APPLY / d.B;
+    if (per < 1) per = 1;
+    int launches = 0;
+    for (int w0 = 0; w0 < workers; w0 += per) {
+      const int n = (workers - w0 < per) ? workers - w0 : per;
+      RowMap u = u_rows, v = v_rows;
+      u.base += (long long)w0 * u.worker_stride;
+      v.base += (long long)w0 * v.worker_stride;
+      const void* dir = directory != nullptr ? reinterpret_cast<const char*>(directory) + (size_t)w0 * 32 : nullptr;
+      const int r = umma_apply_range(pl, s, W, w_shadow, u, v, eta, n * d.B, dev_status, dir);
+      if (r < 0) return r;
+      launches += r;
+    }
+    return launches;
+  }
+  return umma_apply_range(pl, s, W, w_shadow, u_rows, v_rows, eta, K, dev_status, directory);
+}
+
+static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows,
+                            float eta, int K, const int* dev_status, const void* directory) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   const int workers = K / d.B;
