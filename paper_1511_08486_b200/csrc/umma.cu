@@ -788,6 +788,7 @@ int dispatch_gemm(cudaStream_t s, int es, const Variant& v, const CUtensorMap& a
 }  // namespace
 
 constexpr int MAX_SPLITS = 8;   // ranges a forward reduction may be cut into (partial buffers of the plan)
+constexpr int X3_MAX_SPLITS = 16;   // ... on the compensated path, where the count is also tuned to fill whole waves
 
 struct UmmaPlan {
   sfb_desc d;
@@ -837,7 +838,8 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   {   // forward GEMMs whose 128 x 128 tiles do not fill the SMs may split their reduction
     const long long K_ = (long long)d.P * d.B;
     const long long tiles = ((K_ + 127) / 128) * ((d.J + 127) / 128);
-    if ((tiles < p->num_sms || p->x3) && cudaMalloc(&p->part_ws, (size_t)MAX_SPLITS * K_ * p->ldp * 4) != cudaSuccess) {
+    if ((tiles < p->num_sms || p->x3) &&
+        cudaMalloc(&p->part_ws, (size_t)(p->x3 ? X3_MAX_SPLITS : MAX_SPLITS) * K_ * p->ldp * 4) != cudaSuccess) {
       cudaGetLastError();
       delete p;
       return SFB_ERR_ALLOC;
@@ -909,13 +911,21 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
       // Ranges of the reduction, added in fp32 by the finishing pass: enough of them that one accumulator takes
       // at most X3_ATOMS_PER_RANGE atoms (4 instructions each; every instruction rounds the sum toward zero,
       // about 1.6e-8 of it), and enough to give every SM work.
+      // Among the admissible counts the one with the least work on the busiest SM pair is taken: waves of
+      // (tile, range) items times the atoms of a range, plus a little per range for its partial buffer.
       const long long tiles = (long long)((m_units + v.cg - 1) / v.cg) * ((N + 127) / 128);
       const long long slots = pl->num_sms / v.cg;
-      long long ks = (k_atoms + X3_ATOMS_PER_RANGE - 1) / X3_ATOMS_PER_RANGE;
-      if (tiles * ks < slots) ks = (slots + tiles - 1) / tiles;
-      if (ks > max_splits) ks = max_splits;
-      while (ks > 1 && k_atoms < 4 * ks) --ks;
-      *splits = (int)(ks < 1 ? 1 : ks);
+      long long ks_min = (k_atoms + X3_ATOMS_PER_RANGE - 1) / X3_ATOMS_PER_RANGE;
+      if (ks_min > max_splits) ks_min = max_splits;
+      long long best = ks_min < 1 ? 1 : ks_min, best_cost = -1;
+      for (long long ks = best; ks <= max_splits && (ks == best || k_atoms >= 4 * ks); ++ks) {
+        const long long per = (k_atoms + ks - 1) / ks;
+        const long long n_ranges = (k_atoms + per - 1) / per;          // ranges that exist
+        const long long waves = (tiles * n_ranges + slots - 1) / slots;
+        const long long cost = waves * per * 8 + n_ranges * 3;          // in eighths of an atom
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = ks; }
+      }
+      *splits = (int)best;
     }
     return v;
   }
@@ -968,7 +978,8 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   const bool may_split = k_splits_out != nullptr && stats == nullptr && max_splits > 1;
   int ks_pick = 1;
   const Variant v = pick_variant(pl, m_units, d.J, (d.D % CH) == 0 && (a.ld % CH) == 0, (d.D + CH - 1) / CH,
-                                 may_split ? (max_splits < MAX_SPLITS ? max_splits : MAX_SPLITS) : 1, &ks_pick);
+                                 may_split ? (max_splits < (pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS)
+                                                  ? max_splits : (pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS)) : 1, &ks_pick);
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
   p.n_tiles = (d.J + v.bn - 1) / v.bn;
   p.k_blocks = (d.D + CH * v.ka - 1) / (CH * v.ka);
@@ -1020,7 +1031,7 @@ int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMa
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS, sstride, workers)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride)) < 0) return r;
@@ -1072,7 +1083,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
         const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
         int ks = 1;
         if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr,
-                                   nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
+                                   nullptr, &ks, pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS, sstride, workers)) < 0)
           return r;
         launches += r;
         if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride, reinterpret_cast<float*>(aux->dual),
@@ -1113,7 +1124,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, MAX_SPLITS, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS, sstride, workers)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
