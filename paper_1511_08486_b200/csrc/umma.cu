@@ -906,6 +906,15 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
     // kernels, at 43 % tensor-pipe activity, is the shared-memory read path of three MMAs per fp32 operand pair)
     v.bn = 128; v.ka = 1;
     v.cg = m_units >= 2 ? 2 : 1;
+    if (v.cg == 2 && (m_units & 1) && max_splits <= 1) {
+      // An odd number of row units leaves the last pair half empty.  Single CTAs waste nothing there but move about
+      // 192 KB through shared memory per stage where a pair's CTA moves 168 (each loads and splits all of its B tile):
+      // take them when their waves, so weighted, are shorter (600 rows: 3 waves of singles against 4 of pairs).
+      const long long n_tiles = (N + 127) / 128;
+      const long long waves_pair = (((m_units + 1) / 2) * n_tiles + pl->num_sms / 2 - 1) / (pl->num_sms / 2);
+      const long long waves_one = ((long long)m_units * n_tiles + pl->num_sms - 1) / pl->num_sms;
+      if (waves_one * 192 < waves_pair * 168) v.cg = 1;
+    }
     v.fold = v.cg == 2 && dims_chunk_aligned;
     if (splits != nullptr && k_atoms > 0 && max_splits > 1) {
       // Ranges of the reduction, added in fp32 by the finishing pass: enough of them that one accumulator takes

