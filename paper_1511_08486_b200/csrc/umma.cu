@@ -418,15 +418,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
         if (!ok) break;
         uint4* raw = reinterpret_cast<uint4*>(tiles + s * STAGE_BYTES);
-#pragma unroll 8
-        for (int q = lane; q < RAW_BYTES / 16; q += 32) {
-          const uint4 x = raw[q];
-          uint4 lo;
-          lo.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(x.x & 0xFFFFE000u));
-          lo.y = __float_as_uint(__uint_as_float(x.y) - __uint_as_float(x.y & 0xFFFFE000u));
-          lo.z = __float_as_uint(__uint_as_float(x.z) - __uint_as_float(x.z & 0xFFFFE000u));
-          lo.w = __float_as_uint(__uint_as_float(x.w) - __uint_as_float(x.w & 0xFFFFE000u));
-          raw[q + RAW_BYTES / 16] = lo;
+        // eight 16-byte loads in flight per lane before their remainders are computed and stored: the loop is bound
+        // by the shared-memory latency otherwise (the loads and stores go through one pointer, so the compiler keeps
+        // them in program order)
+        constexpr int UNITS = RAW_BYTES / 16;          // a multiple of 256 (tiles of whole 4 KB blocks)
+        static_assert(UNITS % 256 == 0, "stage bytes");
+#pragma unroll 1
+        for (int q0 = lane; q0 < UNITS; q0 += 256) {
+          uint4 x[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) x[j] = raw[q0 + 32 * j];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            uint4 lo;
+            lo.x = __float_as_uint(__uint_as_float(x[j].x) - __uint_as_float(x[j].x & 0xFFFFE000u));
+            lo.y = __float_as_uint(__uint_as_float(x[j].y) - __uint_as_float(x[j].y & 0xFFFFE000u));
+            lo.z = __float_as_uint(__uint_as_float(x[j].z) - __uint_as_float(x[j].z & 0xFFFFE000u));
+            lo.w = __float_as_uint(__uint_as_float(x[j].w) - __uint_as_float(x[j].w & 0xFFFFE000u));
+            raw[q0 + 32 * j + UNITS] = lo;
+          }
         }
         ptx::fence_proxy_async();   // the tensor core reads these tiles through the async proxy
         __syncwarp();
