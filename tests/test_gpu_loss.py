@@ -32,6 +32,10 @@ CASES = [
     ("C3", "f32", dict(J=70, D=333, P=3, B=5, density=0.1)),
     ("C3", "f32", {}),
     ("C3", "tf32", dict(J=512, D=2000, P=4, B=32)),
+    ("C1", "tf32x3", dict(J=200, D=1024, P=4, B=64)),
+    ("C1", "tf32x3", {}),
+    ("C2", "tf32x3", dict(J=64, D=512, P=2, B=64)),
+    ("C3", "tf32x3", dict(J=512, D=2000, P=4, B=32)),
     ("C4", "bf16", dict(J=256, D=512, P=2, B=64, pool=1, labels="uniform")),
     ("C4", "bf16", dict(J=4096, D=2048, P=4, B=128, pool=1)),     # Zipf labels, several tiles per dimension
 ]
