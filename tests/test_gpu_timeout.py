@@ -18,19 +18,20 @@ from tests.test_gpu_parity import _workload
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("over", [
-    dict(J=512, D=4096, P=4, B=128, pool=1, labels="uniform"),       # single-CTA tiles, split reduction
-    dict(J=4096, D=4096, P=8, B=256, pool=1, labels="uniform"),      # CTA pairs, fused softmax epilogue
+@pytest.mark.parametrize("path,over", [
+    ("bf16", dict(J=512, D=4096, P=4, B=128, pool=1, labels="uniform")),       # single-CTA tiles, split reduction
+    ("bf16", dict(J=4096, D=4096, P=8, B=256, pool=1, labels="uniform")),      # CTA pairs, fused softmax epilogue
+    ("tf32x3", dict(J=512, D=2048, P=4, B=128, pool=1, labels="uniform")),     # compensated kernels: the splitter warps leave too
 ])
-def test_lost_signal_times_out_cleanly(over, monkeypatch):
+def test_lost_signal_times_out_cleanly(path, over, monkeypatch):
     from paper_1511_08486_b200 import binding as B
     cfg = scaled("C4", **over)
-    cfg["path"] = "bf16"
+    cfg["path"] = path
     inputs = make_inputs(cfg)
     monkeypatch.setenv("SFB_TEST_LOSE_SIGNAL", "1")
-    wl = _workload(cfg, inputs, "bf16")
+    wl = _workload(cfg, inputs, path)
     monkeypatch.delenv("SFB_TEST_LOSE_SIGNAL")
-    fresh = _workload(cfg, inputs, "bf16")
+    fresh = _workload(cfg, inputs, path)
     try:
         t0 = time.perf_counter()
         wl.step(0, eta=1e-3)
