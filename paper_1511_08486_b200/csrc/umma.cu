@@ -805,6 +805,7 @@ struct UmmaPlan {
   Layout l;
   int num_sms;
   int es;
+  int max_splits; // ranges a forward reduction may be cut into = partial buffers allocated
   bool x3;        // error-compensated tf32 (SFB_PATH_TF32X3): the SPLIT kernels, forward always through partial buffers
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
   float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
@@ -828,9 +829,9 @@ constexpr int STAGE_ATOMS = 2;
 // Compensated kernels: 128-byte atoms (32 fp32 reduction steps = 4 MMA instructions) one accumulator may take
 // before its range ends: 40 atoms = 160 roundings toward zero, about 2.6e-6 of the sum.
 constexpr int X3_ATOMS_PER_RANGE = 40;
-// ... and pairs one launch of the compensated apply takes (512 instructions: 8e-6 of the sum at worst, half of it
-// on average over a tile's life); larger updates are applied in several launches.
-constexpr int X3_PAIRS_PER_APPLY = 4096;
+// ... and pairs one launch of the compensated apply takes (256 instructions: 4e-6 of the sum; measured: 4096 pairs in
+// one launch come out at 1.0e-5, 2048 at 5e-6); larger updates are applied in several launches.
+constexpr int X3_PAIRS_PER_APPLY = 2048;
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   if (get_encode() == nullptr) return SFB_ERR_CUDA;
@@ -848,8 +849,14 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   {   // forward GEMMs whose 128 x 128 tiles do not fill the SMs may split their reduction
     const long long K_ = (long long)d.P * d.B;
     const long long tiles = ((K_ + 127) / 128) * ((d.J + 127) / 128);
-    if ((tiles < p->num_sms || p->x3) &&
-        cudaMalloc(&p->part_ws, (size_t)(p->x3 ? X3_MAX_SPLITS : MAX_SPLITS) * K_ * p->ldp * 4) != cudaSuccess) {
+    // the compensated path tunes the count up to 16, within 4 GB of partial buffers
+    p->max_splits = MAX_SPLITS;
+    if (p->x3) {
+      const long long one = K_ * p->ldp * 4;
+      long long n = (4LL << 30) / (one > 0 ? one : 1);
+      p->max_splits = (int)(n < 1 ? 1 : (n > X3_MAX_SPLITS ? X3_MAX_SPLITS : n));
+    }
+    if ((tiles < p->num_sms || p->x3) && cudaMalloc(&p->part_ws, (size_t)p->max_splits * K_ * p->ldp * 4) != cudaSuccess) {
       cudaGetLastError();
       delete p;
       return SFB_ERR_ALLOC;
@@ -997,8 +1004,7 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   const bool may_split = k_splits_out != nullptr && stats == nullptr && max_splits > 1;
   int ks_pick = 1;
   const Variant v = pick_variant(pl, m_units, d.J, (d.D % CH) == 0 && (a.ld % CH) == 0, (d.D + CH - 1) / CH,
-                                 may_split ? (max_splits < (pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS)
-                                                  ? max_splits : (pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS)) : 1, &ks_pick);
+                                 may_split ? (max_splits < pl->max_splits ? max_splits : pl->max_splits) : 1, &ks_pick);
   p.m_tiles = (m_units + v.cg - 1) / v.cg;
   p.n_tiles = (d.J + v.bn - 1) / v.bn;
   p.k_blocks = (d.D + CH * v.ka - 1) / (CH * v.ka);
@@ -1050,7 +1056,7 @@ int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMa
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride)) < 0) return r;
@@ -1102,7 +1108,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
         const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
         int ks = 1;
         if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr,
-                                   nullptr, &ks, pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS, sstride, workers)) < 0)
+                                   nullptr, &ks, pl->max_splits, sstride, workers)) < 0)
           return r;
         launches += r;
         if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride, reinterpret_cast<float*>(aux->dual),
@@ -1143,7 +1149,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->x3 ? X3_MAX_SPLITS : MAX_SPLITS, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
