@@ -50,7 +50,7 @@
  *                  same wire format as SFB_PATH_TF32.  The tensor core's fp32 accumulator rounds toward zero
  *                  once per instruction of 8 reduction steps, which costs about 1.6e-8 of a sum per
  *                  instruction: forward reductions are cut into ranges that are added in fp32 afterwards, and
- *                  updates of more than 2048 pairs are applied to W in several launches of whole worker streams.
+ *                  updates of more than 1024 pairs are applied to W in several launches of whole worker streams.
  *
  * SF buffer wire format (little-endian; every offset a multiple of 128 bytes)
  *   header, 128 bytes:

@@ -829,9 +829,9 @@ constexpr int STAGE_ATOMS = 2;
 // Compensated kernels: 128-byte atoms (32 fp32 reduction steps = 4 MMA instructions) one accumulator may take
 // before its range ends: 40 atoms = 160 roundings toward zero, about 2.6e-6 of the sum.
 constexpr int X3_ATOMS_PER_RANGE = 40;
-// ... and pairs one launch of the compensated apply takes (256 instructions: 4e-6 of the sum; measured: 4096 pairs in
+// ... and pairs one launch of the compensated apply takes (128 instructions: 2e-6 of the sum; measured: 4096 pairs in
 // one launch come out at 1.0e-5, 2048 at 5e-6); larger updates are applied in several launches.
-constexpr int X3_PAIRS_PER_APPLY = 2048;
+constexpr int X3_PAIRS_PER_APPLY = 1024;
 
 int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   if (get_encode() == nullptr) return SFB_ERR_CUDA;

@@ -30,7 +30,7 @@ def _pair(cfg, inputs, path):
     ("tf32", dict(J=72, D=1000, P=3, B=20), 1e-4),            # several workers share a reduction block: nothing skipped
     ("tf32", dict(J=260, D=1024, P=5, B=200), 1e-4),          # B >= one reduction block: whole blocks are skipped
     ("tf32x3", dict(J=260, D=1024, P=5, B=200), 1e-4),        # compensated path, blocks skipped
-    ("tf32x3", dict(J=128, D=512, P=32, B=256), 1e-4),        # 8192 pairs: four launches of the apply, directory offsets
+    ("tf32x3", dict(J=128, D=512, P=32, B=256), 1e-4),        # 8192 pairs: eight launches of the apply, directory offsets
     ("f32", {}, 1e-5),                                        # full size
     ("tf32", {}, 1e-5),
 ])

@@ -49,7 +49,7 @@ def test_x3_sparse_coding_scaled():
 
 def test_x3_many_pairs_are_applied_in_several_launches():
     """16384 pairs per update: one accumulator would take 2048 roundings toward zero (3e-5 of the sum); the apply goes
-    to W in eight launches of 2048 pairs instead and stays inside 1e-5.  Also with compaction (directory offsets)."""
+    to W in sixteen launches of 1024 pairs instead and stays inside 1e-5.  Also with compaction (directory offsets)."""
     check_config(_cfg("C1", J=128, D=256, P=64, B=256, pool=1), "tf32x3", eta=0.5, steps=1)
     cfg = _cfg("C2", J=128, D=512, P=32, B=256)
     cfg["compact"] = 0
