@@ -372,6 +372,41 @@ __global__ void __launch_bounds__(256) transpose_rows_kernel(RowMap src, float* 
   }
 }
 
+// The same transposition for rows that are whole numbers of 16-byte units (C a multiple of 4, rows 16-byte aligned):
+// 64 x 64 tiles, 16-byte global loads and stores on both sides, and both operands of the forward pass in one launch
+// (blockIdx.z picks the job).
+struct TransposeJob {
+  RowMap src;
+  float* dst;
+  int R, C, ldr;
+  RowMap copy;
+};
+__global__ void __launch_bounds__(256) transpose_rows_vec_kernel(TransposeJob j0, TransposeJob j1) {
+  __shared__ float tile[64][65];
+  const TransposeJob& j = blockIdx.z == 0 ? j0 : j1;
+  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+  if (c0 >= j.C || r0 >= j.ldr) return;
+  const int tq = threadIdx.x & 15, tr = threadIdx.x >> 4;   // 16 x 16
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int rr = tr + 16 * q, r = r0 + rr, c = c0 + tq * 4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (r < j.R && c < j.C) {
+      v = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(j.src.row(r)) + c);
+      if (j.copy.base != nullptr) *reinterpret_cast<float4*>(reinterpret_cast<float*>(j.copy.row(r)) + c) = v;
+    }
+    tile[rr][tq * 4] = v.x; tile[rr][tq * 4 + 1] = v.y; tile[rr][tq * 4 + 2] = v.z; tile[rr][tq * 4 + 3] = v.w;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int cc = tr + 16 * q, c = c0 + cc, r = r0 + tq * 4;
+    if (c < j.C && r < j.ldr)
+      *reinterpret_cast<float4*>(j.dst + (size_t)c * j.ldr + r) =
+          make_float4(tile[tq * 4][cc], tile[tq * 4 + 1][cc], tile[tq * 4 + 2][cc], tile[tq * 4 + 3][cc]);
+  }
+}
+
 }  // namespace
 
 // Few 128 x 128 tiles and a long reduction (e.g. 1024 samples x 1000 classes over 20000 features): the
@@ -448,8 +483,22 @@ int launch_forward_f32_nn(cudaStream_t s, const float* W, RowMap src, RowMap cop
   RowMap wrows;
   wrows.base = const_cast<char*>(reinterpret_cast<const char*>(W));
   wrows.worker_stride = 0; wrows.ld = D; wrows.B = J > 0 ? J : 1; wrows.es = 4;
-  transpose_rows_kernel<<<dim3((D + 31) / 32, (ldk + 31) / 32), 256, 0, s>>>(src, xt, K, D, ldk, copy);
-  transpose_rows_kernel<<<dim3((D + 31) / 32, (ldj + 31) / 32), 256, 0, s>>>(wrows, wt, J, D, ldj, RowMap());
+  const bool vec = (D & 3) == 0 && (src.ld & 3) == 0 && (reinterpret_cast<uintptr_t>(src.base) & 15) == 0 &&
+                   (src.worker_stride & 15) == 0 && (reinterpret_cast<uintptr_t>(W) & 15) == 0 &&
+                   (copy.base == nullptr || ((copy.ld & 3) == 0 && (reinterpret_cast<uintptr_t>(copy.base) & 15) == 0 &&
+                                             (copy.worker_stride & 15) == 0));
+  int transposes = 2;
+  if (vec) {   // both operands in one launch
+    TransposeJob jx, jw;
+    jx.src = src; jx.dst = xt; jx.R = K; jx.C = D; jx.ldr = ldk; jx.copy = copy;
+    jw.src = wrows; jw.dst = wt; jw.R = J; jw.C = D; jw.ldr = ldj; jw.copy = RowMap();
+    const int ry = ((ldk > ldj ? ldk : ldj) + 63) / 64;
+    transpose_rows_vec_kernel<<<dim3((D + 63) / 64, ry, 2), 256, 0, s>>>(jx, jw);
+    transposes = 1;
+  } else {
+    transpose_rows_kernel<<<dim3((D + 31) / 32, (ldk + 31) / 32), 256, 0, s>>>(src, xt, K, D, ldk, copy);
+    transpose_rows_kernel<<<dim3((D + 31) / 32, (ldj + 31) / 32), 256, 0, s>>>(wrows, wt, J, D, ldj, RowMap());
+  }
   int ks = (part.base != nullptr && nsplit_out != nullptr) ? forward_f32_splits(K, J, D) : 1;
   if (ks > max_splits) ks = max_splits;
   if (nsplit_out != nullptr) *nsplit_out = ks;
@@ -464,7 +513,7 @@ int launch_forward_f32_nn(cudaStream_t s, const float* W, RowMap src, RowMap cop
   dim3 grid((J + 127) / 128, (K + 127) / 128, ks);
   sgemm_pipe_kernel<1><<<grid, 256, PIPE * PIPE_STAGE_FLOATS * 4, s>>>(nullptr, a, b, D, K, ldj, 0.f, nullptr,
                                                                        ks > 1 ? part : z, per, split_stride, nullptr, nullptr);
-  return cudaGetLastError() == cudaSuccess ? 3 : SFB_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? transposes + 1 : SFB_ERR_CUDA;
 }
 
 }  // namespace sfb
