@@ -12,7 +12,7 @@ import torch
 from oracle import sfb_oracle as orc
 from sfbgen import get_config, make_inputs, scaled
 from tests.test_gpu_parity import _workload
-from tests.util import MODEL_ID, TOL, assert_lines, batch_of, to_f64
+from tests.util import MODEL_ID, TOL, assert_lines
 
 pytestmark = pytest.mark.gpu
 

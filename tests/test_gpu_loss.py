@@ -1,5 +1,4 @@
 """The device-side minibatch objective (sfb_loss) against the oracle's fp64 losses."""
-import numpy as np
 import pytest
 import torch
 

@@ -5,9 +5,7 @@ MMA tile and single pipeline stage (so a wrong descriptor or swizzle shows up in
 span several tiles, ragged edges handled by TMA zero fill, worker streams shorter than one
 reduction block, and finally the full workload shapes.
 """
-import numpy as np
 import pytest
-import torch
 
 from sfbgen import get_config, scaled
 from tests.test_gpu_parity import check_config
