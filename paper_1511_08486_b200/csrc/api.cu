@@ -45,7 +45,9 @@ struct sfb_ctx {
   cudaEvent_t copied[2], consumed[2];
   bool host_ready;
   uint64_t host_steps;
-  __nv_bfloat16* w_shadow;  // bf16 path: bf16 copy of W, refreshed by the apply
+  // bf16 path: bf16 copy of W, refreshed by the apply.  Compensated tf32 path: W's correction operand
+  // (bf16 [value | remainder] per 32 columns, as many bytes as W), rebuilt before a forward pass when stale.
+  __nv_bfloat16* w_shadow;
   const void* shadow_of;    // W pointer the shadow currently mirrors (nullptr = stale)
   UmmaPlan* umma;           // tensor-core plan (tensor maps), TF32 / BF16 paths
   int64_t launches;
@@ -143,10 +145,19 @@ int check_aux(const sfb_ctx* c, const sfb_aux* a) {
     c->launches += r_;             \
   } while (0)
 
-// Refreshes the bf16 shadow of W if it does not mirror this W.
+bool has_shadow(const sfb_ctx* c) { return c->d.path == SFB_PATH_BF16 || c->d.path == SFB_PATH_TF32X3; }
+
+// Refreshes the shadow of W (bf16 copy, or correction operand) if it does not mirror this W.
 int ensure_shadow(sfb_ctx* c, const void* W) {
-  if (c->d.path != SFB_PATH_BF16 || c->shadow_of == W) return SFB_OK;
-  ACC(launch_cast_bf16(c->stream, reinterpret_cast<const float*>(W), c->w_shadow, (long long)c->d.J * c->d.D));
+  if (!has_shadow(c) || c->shadow_of == W) return SFB_OK;
+  if (c->d.path == SFB_PATH_BF16) {
+    ACC(launch_cast_bf16(c->stream, reinterpret_cast<const float*>(W), c->w_shadow, (long long)c->d.J * c->d.D));
+  } else {
+    RowMap w;
+    w.base = const_cast<char*>(reinterpret_cast<const char*>(W));
+    w.ld = c->d.D; w.B = c->d.J; w.es = 4; w.worker_stride = 0;
+    ACC(launch_split_k(c->stream, w, c->d.J, c->d.D, c->w_shadow, false));
+  }
   c->shadow_of = W;
   return SFB_OK;
 }
@@ -168,7 +179,12 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     // plain tf32: the code values are rounded to nearest tf32 as they are densified; the compensated path keeps
     // them exact (its kernels split every operand into what the tensor core sees and the rest)
     ACC(launch_densify_codes(c->stream, codes, a, K, d.D, c->dev_status, d.path == SFB_PATH_TF32));
-    ACC(umma_forward_sc(c->umma, c->stream, W, a, u, reinterpret_cast<const float*>(aux->Xdata), c->dev_status, workers));
+    {
+      const int r = ensure_shadow(c, W);
+      if (r < 0) return r;
+    }
+    ACC(umma_forward_sc(c->umma, c->stream, W, a, u, reinterpret_cast<const float*>(aux->Xdata), c->dev_status, workers,
+                        c->w_shadow));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {
@@ -198,7 +214,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     return SFB_OK;
   }
   // tensor-core paths
-  if (d.path == SFB_PATH_BF16) {
+  {
     const int r = ensure_shadow(c, W);
     if (r < 0) return r;
   }
@@ -298,6 +314,8 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
     }
   }
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
+  if (ok && desc->path == SFB_PATH_TF32X3)
+    ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * ((desc->D + 31) / 32) * 128) == cudaSuccess;
   if (ok && desc->compact) {
     ok = cudaMalloc(&c->compact_ws, (size_t)compact_workspace_bytes(c->K, desc->P)) == cudaSuccess;
     if (ok && desc->path == SFB_PATH_F32) ok = cudaMalloc(&c->kept_idx, ((size_t)c->K + 1) * 4) == cudaSuccess;
@@ -363,6 +381,7 @@ int sfb_prox(sfb_ctx* c, void* W) {
   if (c == nullptr || W == nullptr || !aligned(W, 16)) return SFB_ERR_ARG;
   if (c->d.model != SFB_SC) return SFB_OK;   // h = 0 for the MLR and DML workloads: identity
   ACC(launch_prox_unit_columns(c->stream, reinterpret_cast<float*>(W), c->d.J, c->d.D));
+  c->shadow_of = nullptr;   // W changed
   return SFB_OK;
 }
 
@@ -399,7 +418,7 @@ int sfb_loss(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, doubl
     if (r < 0) return r;
     const bool bf16 = d.path == SFB_PATH_BF16;
     ACC(umma_forward_rows(c->umma, c->stream, bf16 ? (const void*)c->w_shadow : W, caller_rows(X, d.D, d.B, c->l.es),
-                          rows, c->dev_status));
+                          rows, c->dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, 0, c->w_shadow));
   }
   ACC(launch_sample_loss(c->stream, d.model, rows, aux->labels, aux->similar, d.margin, c->K, d.J, c->loss_i, loss,
                          c->dev_status));
@@ -554,6 +573,7 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
       ACC(launch_densify_codes(c->stream, stream_codes(c, sf_buf), dense_codes(c), K, d.D, c->dev_status,
                                d.path == SFB_PATH_TF32));
     ACC(umma_apply(c->umma, c->stream, W, nullptr, stream_u(c, sf_buf), dense_codes(c), eta, K, c->dev_status));
+    c->shadow_of = nullptr;   // W changed: a correction operand made from it is stale
   } else if (d.path == SFB_PATH_F32) {
     const int* idx = nullptr;
     const int* n_idx = nullptr;
@@ -572,6 +592,7 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
     ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status,
                    d.compact ? reinterpret_cast<const char*>(sf_buf) + 128 : nullptr));
     if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
+    else c->shadow_of = nullptr;                     // W changed: its correction operand is stale
   }
   return SFB_OK;
 }
@@ -615,7 +636,7 @@ int sfb_apply(sfb_ctx* c, void* W, const void* sf_buf, float eta, int32_t K) {
   if (c == nullptr || W == nullptr || sf_buf == nullptr) return SFB_ERR_ARG;
   if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
   if (K <= 0 || K > c->K || (K % c->d.B) != 0) return SFB_ERR_ARG;
-  if (c->d.path == SFB_PATH_BF16 && c->shadow_of != W) c->shadow_of = nullptr;
+  if (has_shadow(c) && c->shadow_of != W) c->shadow_of = nullptr;
   return apply_from(c, W, sf_buf, eta, K, true);
 }
 

@@ -189,5 +189,12 @@ int launch_sample_loss(cudaStream_t s, int model, RowMap rows, const int32_t* la
 
 // W (fp32) -> bf16 shadow, round to nearest even.
 int launch_cast_bf16(cudaStream_t s, const float* W, __nv_bfloat16* Wb, long long n);
+// Correction operands of the error-compensated tf32 kernels (split.cu): bf16 [remainder | value] (A side) or
+// [value | remainder] (B side) of fp32 rows.  K-major: dst[row][atom][64] over `rows` rows of `cols` values.
+// MN-major: dst[block][64][ldc], block = 32 pairs taken as the apply's reduction blocks are (32 rows of one
+// worker, or k_bb rows of each of k_wp workers), ldc a multiple of 64.
+int launch_split_k(cudaStream_t s, RowMap src, int rows, int cols, void* dst, bool a_side);
+int launch_split_mn(cudaStream_t s, RowMap src, int cols, int workers, int k_bb, int k_wp, int k_bpw, int blocks,
+                    void* dst, int ldc, bool a_side);
 
 }  // namespace sfb

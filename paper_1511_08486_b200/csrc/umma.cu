@@ -35,7 +35,6 @@ namespace {
 
 constexpr int BM = 128;          // rows per CTA tile = TMEM lanes
 constexpr int NUM_THREADS = 320;         // TMA warp, MMA warp, 8 epilogue warps
-constexpr int SPLIT_THREADS = 128;       // error-compensated kernels: 4 more warps that split the operand stages
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // one swizzled 32 x 32 fp32 block per epilogue warp
 constexpr int RING_BYTES = 192 * 1024;   // shared memory given to the operand ring
 constexpr int MAX_STAGES = 8;
@@ -70,7 +69,6 @@ struct GemmParams {
 
 struct SharedCtl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
-  uint64_t ready[MAX_STAGES];   // error-compensated kernels: the stage's residual tiles are written (both CTAs of a pair)
   uint32_t tmem_base;
   volatile int abort;
   int k_total;                 // apply: reduction blocks per tile (sum of nb[] when a directory is given)
@@ -130,17 +128,21 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 //          one TMA instruction fills a whole operand stage (needs J, D multiples of CH); otherwise
 //          one 3-D TMA per chunk, with zero fill on every ragged edge.
 //   SPLIT  error-compensated tf32 (ES = 4): the tensor core drops the low 13 mantissa bits of an fp32 operand, so
-//          x = hi + lo with hi = what the tensor core sees of x and lo = x - hi (exact in fp32).  Four extra
-//          warps compute the lo tiles of every operand stage in shared memory, and every reduction step
-//          issues three MMAs: a * b into the main accumulator, lo(a) * b and a * lo(b) into a second one
-//          (lo * lo, about 2^-22 of the product, is dropped).  The accumulators are added in the epilogue.
+//          x = hi + lo with hi = what the tensor core sees of x and lo = x - hi (exact in fp32).  Besides its
+//          fp32 operand tiles a stage then holds the bf16 correction tiles [lo(a) | a] and [b | lo(b)] (a
+//          pre-pass writes them to global memory with the tiling of the fp32 operands, tensor maps tmAc / tmBc;
+//          64 bf16 reduction steps per 128-byte atom of 32 fp32 ones), and every atom issues four tf32
+//          instructions a * b into the main accumulator and four bf16 instructions lo(a) b + a lo(b) into a
+//          second one (lo * lo, about 2^-22 of the product, is dropped; bf16 carries the corrections, themselves
+//          2^-10 of the product, to 2^-18).  The accumulators are added in the epilogue.
 //          Two accumulators because the tensor core's fp32 accumulation rounds toward zero once per
 //          instruction (measured: a sum of n instructions comes out short by about n * 2^-26): the small
-//          corrections must not cost the large sum two more roundings per step.
+//          corrections must not cost the large sum more roundings.
 template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI, bool SPLIT>
-__global__ void __launch_bounds__(NUM_THREADS + (SPLIT ? SPLIT_THREADS : 0), 1)
+__global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
+                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmAc,
+                 const __grid_constant__ CUtensorMap tmBc, const GemmParams p) {
   constexpr int CH = 128 / ES;                 // values per 128-byte chunk
   constexpr int BK = CH * KA;                  // reduction steps per pipeline stage
   constexpr int UMMA_K = 32 / ES;              // reduction steps per instruction (16 bf16 / 8 tf32)
@@ -148,15 +150,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   constexpr int A_STAGE_BYTES = BM * 128 * KA;
   constexpr int B_STAGE_BYTES = BNC * 128 * KA;
   constexpr int RAW_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;     // what TMA brings per stage
-  constexpr int STAGE_BYTES = RAW_BYTES * (SPLIT ? 2 : 1);     // SPLIT: the lo tiles follow, same layout
+  constexpr int STAGE_BYTES = RAW_BYTES * (SPLIT ? 2 : 1);     // SPLIT: the correction tiles follow, same sizes
   constexpr int NACC = SPLIT ? 2 : 1;                          // accumulators per tile (main, corrections)
   constexpr int ACC_COLS = BN * NACC;
+  constexpr int NBUF = (2 * ACC_COLS <= 512) ? 2 : 1;          // accumulator sets in the 512 columns of tensor memory
   static_assert(!SPLIT || (ES == 4 && EPI == 0), "error compensation is for fp32 operands and plain stores");
-  // whose "full" barrier a CTA's loads are credited to: its own (single CTAs; and SPLIT pairs, where each CTA's
-  // splitter warps wait for their own CTA's bytes), or the even CTA's (plain pairs: one barrier for the MMA issuer)
-  constexpr bool OWN = (CG == 1) || SPLIT;
+  // whose "full" barrier a CTA's loads are credited to: its own, or the even CTA's (pairs: one barrier for the
+  // MMA issuer)
+  constexpr bool OWN = (CG == 1);
   constexpr int STAGES = (RING_BYTES / STAGE_BYTES) < MAX_STAGES ? (RING_BYTES / STAGE_BYTES) : MAX_STAGES;
   constexpr uint32_t IDESC = ptx::instr_desc(ES == 2 ? 1u : 2u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM * CG, BN);
+  constexpr uint32_t IDESC_C = ptx::instr_desc(1u, APPLY ? 1u : 0u, APPLY ? 1u : 0u, BM * CG, BN);   // SPLIT: bf16 corrections
+  static_assert(!SPLIT || KA == 1, "the correction tiles hold one atom of the reduction");
   static_assert(STAGES >= 2, "ring too shallow");
 
   extern __shared__ uint8_t smem_raw[];
@@ -174,7 +179,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&ctl->full[s], 1);
       ptx::mbar_init(&ctl->empty[s], 1);
-      ptx::mbar_init(&ctl->ready[s], CG);   // one arrival per CTA: the splitter warp that took the stage
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->tmem_full[b], 1);
@@ -197,9 +201,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmA);
     ptx::prefetch_tmap(&tmB);
+    if (SPLIT) { ptx::prefetch_tmap(&tmAc); ptx::prefetch_tmap(&tmBc); }
   }
   if (warp == 1) {
-    ptx::tmem_alloc<CG>(&ctl->tmem_base, 2 * ACC_COLS);
+    ptx::tmem_alloc<CG>(&ctl->tmem_base, NBUF * ACC_COLS);
     ptx::tmem_relinquish<CG>();
   }
   ptx::tc_fence_before();
@@ -244,7 +249,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           uint64_t* bar = &ctl->full[s];
           uint32_t full_addr = ptx::smem_u32(bar);
           if (CG == 2) full_addr = ptx::map_to_cta(full_addr, 0);
-          if (OWN) ptx::mbar_expect_tx(bar, RAW_BYTES);
+          if (OWN) ptx::mbar_expect_tx(bar, STAGE_BYTES);
           else if (rank == 0) ptx::mbar_expect_tx(bar, CG * STAGE_BYTES);
           if (!APPLY) {
             if (FOLD) {   // dims (value-in-atom, row, worker, atom): one box = KA atoms of 128 rows
@@ -291,6 +296,32 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
         }
+        if (SPLIT && lane == 0) {
+          // correction tiles: same coordinates as the fp32 ones, in units of their own tiling
+          uint8_t* ac_dst = tiles + s * STAGE_BYTES + RAW_BYTES;
+          uint8_t* bc_dst = ac_dst + A_STAGE_BYTES;
+          uint64_t* bar = &ctl->full[s];
+          uint32_t full_addr = ptx::smem_u32(bar);
+          if (CG == 2) full_addr = ptx::map_to_cta(full_addr, 0);
+          if (!APPLY) {   // dims (value-in-atom, row, worker, atom)
+            if (OWN) {
+              ptx::tma_load_4d_hint(ac_dst, &tmAc, bar, 0, slot0, mp0, kb, pol_a);
+              ptx::tma_load_4d_hint(bc_dst, &tmBc, bar, 0, ncol0, 0, kb, pol_b);
+            } else {
+              ptx::tma_load_4d_hint_pair(ac_dst, &tmAc, full_addr, 0, slot0, mp0, kb, pol_a);
+              ptx::tma_load_4d_hint_pair(bc_dst, &tmBc, full_addr, 0, ncol0, 0, kb, pol_b);
+            }
+          } else {        // dims (value-in-chunk of 64, line, chunk): 64 lines per reduction block
+            const int blk = (p.B >= BK) ? kp0 * p.k_bpw + row0 / BK : kp0 / p.k_wp;
+            if (OWN) {
+              ptx::tma_load_3d_hint(ac_dst, &tmAc, bar, 0, blk * 64, (mt * BM) / 64, pol_a);
+              ptx::tma_load_3d_hint(bc_dst, &tmBc, bar, 0, blk * 64, ncol0 / 64, pol_b);
+            } else {
+              ptx::tma_load_3d_hint_pair(ac_dst, &tmAc, full_addr, 0, blk * 64, (mt * BM) / 64, pol_a);
+              ptx::tma_load_3d_hint_pair(bc_dst, &tmBc, full_addr, 0, blk * 64, ncol0 / 64, pol_b);
+            }
+          }
+        }
         if (APPLY) {   // next reduction block: next BK rows of this worker, or the next group of workers
           if (p.B >= BK) {
             row0 += BK;
@@ -328,15 +359,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int work = cluster_id; work < total_work && ok; work += num_clusters, ++it) {
       const int split = work % p.k_splits;
       const int kb_begin = split * k_per_split, kb_end = min(kb_begin + k_per_split, k_blocks);
-      const int buf = it & 1;
-      const uint32_t acc_ph = (it >> 1) & 1u;
+      const int buf = it % NBUF;
+      const uint32_t acc_ph = (uint32_t)(it / NBUF) & 1u;
       ok = wait_or_abort(&ctl->tmem_empty[buf], acc_ph ^ 1u, ctl, p.status);
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
       const uint32_t d_lo = d_tmem + BN;              // SPLIT: accumulator of the correction products
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        ok = wait_or_abort(SPLIT ? &ctl->ready[s] : &ctl->full[s], ph, ctl, p.status, SPLIT && CG == 2);
+        ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
         if (!ok) break;
         ptx::tc_fence_after();
         if (lane == 0) {
@@ -354,10 +385,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const uint32_t acc = (kb > kb_begin || a > 0 || k > 0) ? 1u : 0u;
                 if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
                 else ptx::mma_tf32<CG>(d_tmem, a_desc + k * 2, b_desc + k * 2, IDESC, acc);
-                if (SPLIT) {   // lo(a) * b + a * lo(b): the lo tiles sit RAW_BYTES behind the raw ones
-                  ptx::mma_tf32<CG>(d_lo, a_desc + (RAW_BYTES >> 4) + k * 2, b_desc + k * 2, IDESC, acc);
-                  ptx::mma_tf32<CG>(d_lo, a_desc + k * 2, b_desc + (RAW_BYTES >> 4) + k * 2, IDESC, 1u);
-                }
+              }
+              if (SPLIT) {
+                // corrections: the bf16 tiles RAW_BYTES behind the fp32 ones, [lo(a) | a] times [b | lo(b)] over 64
+                // reduction steps = lo(a) b + a lo(b) of the atom's 32; four instructions of 16
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  ptx::mma_f16<CG>(d_lo, a_desc + (RAW_BYTES >> 4) + k * 2, b_desc + (RAW_BYTES >> 4) + k * 2, IDESC_C,
+                                   (kb > kb_begin || k > 0) ? 1u : 0u);
               }
             }
           } else {
@@ -372,10 +407,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               const uint32_t acc = (kb > kb_begin || k > 0) ? 1u : 0u;
               if (ES == 2) ptx::mma_f16<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
               else ptx::mma_tf32<CG>(d_tmem, a_desc + k * STEP, b_desc + k * STEP, IDESC, acc);
-              if (SPLIT) {
-                ptx::mma_tf32<CG>(d_lo, a_desc + (RAW_BYTES >> 4) + k * STEP, b_desc + k * STEP, IDESC, acc);
-                ptx::mma_tf32<CG>(d_lo, a_desc + k * STEP, b_desc + (RAW_BYTES >> 4) + k * STEP, IDESC, 1u);
-              }
+            }
+            if (SPLIT) {
+              // corrections: bf16 tiles of 64 reduction lines ([lo(a) ; a] and [b ; lo(b)]) in 128-byte chunks of 64
+              // values, 8192 B apart, 128-byte swizzle; sixteen lines per instruction
+              const uint64_t ac_desc = ptx::smem_desc(a_addr + RAW_BYTES, 64 * 128, 1024, 2);
+              const uint64_t bc_desc = ptx::smem_desc(b_addr + RAW_BYTES, 64 * 128, 1024, 2);
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                ptx::mma_f16<CG>(d_lo, ac_desc + k * 128, bc_desc + k * 128, IDESC_C, (kb > kb_begin || k > 0) ? 1u : 0u);
             }
           }
           // (test hook: one lost signal, so that the producer's bounded wait runs out and the abort path is taken)
@@ -391,59 +431,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         __syncwarp();
         if (++s == STAGES) { s = 0; ph ^= 1u; }
-      }
-    }
-  } else if (SPLIT && warp >= NUM_THREADS / 32) {
-    // ------------------------------------------------------------------ operand splitter (warps 10..13, every CTA)
-    // For every stage that has landed: lo = x - (x with the low 13 mantissa bits cleared), element by element, into
-    // the second half of the stage (the swizzled layout is the same, so the tiles are walked as flat memory).
-    // Each of the four warps takes its own stages of the ring and splits them alone, so up to four stages are in the works at a
-    // time: the chain "wait for the bytes, read, subtract, write, fence, signal" of one stage is longer than the
-    // tensor core needs for the stage's MMAs, but four of them overlap.
-    constexpr int NSPLIT = SPLIT_THREADS / 32;
-    const int sw = warp - NUM_THREADS / 32;
-    long long n_stage = 0;     // running count of reduction blocks over all of this CTA's tiles
-    bool ok = true;
-    uint32_t ready_addr = ptx::smem_u32(&ctl->ready[0]);
-    if (CG == 2) ready_addr = ptx::map_to_cta(ready_addr, 0);
-    for (int work = cluster_id; work < total_work && ok; work += num_clusters) {
-      const int split = work % p.k_splits;
-      const int kb_begin = split * k_per_split, kb_end = min(kb_begin + k_per_split, k_blocks);
-      for (int kb = kb_begin; kb < kb_end; ++kb, ++n_stage) {
-        // a warp owns whole stages of the ring (stage s belongs to warp s mod 4), so it meets every phase of its
-        // stages' barriers in order; parity waits cannot tell phases two apart
-        const int s = (int)(n_stage % STAGES);
-        if (s % NSPLIT != sw) continue;
-        const uint32_t ph = (uint32_t)((n_stage / STAGES) & 1);
-        ok = wait_or_abort(&ctl->full[s], ph, ctl, p.status);
-        if (!ok) break;
-        uint4* raw = reinterpret_cast<uint4*>(tiles + s * STAGE_BYTES);
-        // eight 16-byte loads in flight per lane before their remainders are computed and stored: the loop is bound
-        // by the shared-memory latency otherwise (the loads and stores go through one pointer, so the compiler keeps
-        // them in program order)
-        constexpr int UNITS = RAW_BYTES / 16;          // a multiple of 256 (tiles of whole 4 KB blocks)
-        static_assert(UNITS % 256 == 0, "stage bytes");
-#pragma unroll 1
-        for (int q0 = lane; q0 < UNITS; q0 += 256) {
-          uint4 x[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) x[j] = raw[q0 + 32 * j];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            uint4 lo;
-            lo.x = __float_as_uint(__uint_as_float(x[j].x) - __uint_as_float(x[j].x & 0xFFFFE000u));
-            lo.y = __float_as_uint(__uint_as_float(x[j].y) - __uint_as_float(x[j].y & 0xFFFFE000u));
-            lo.z = __float_as_uint(__uint_as_float(x[j].z) - __uint_as_float(x[j].z & 0xFFFFE000u));
-            lo.w = __float_as_uint(__uint_as_float(x[j].w) - __uint_as_float(x[j].w & 0xFFFFE000u));
-            raw[q0 + 32 * j + UNITS] = lo;
-          }
-        }
-        ptx::fence_proxy_async();   // the tensor core reads these tiles through the async proxy
-        __syncwarp();
-        if (lane == 0) {
-          if (CG == 1) ptx::mbar_arrive(&ctl->ready[s]);
-          else ptx::mbar_arrive_cluster(ready_addr + (uint32_t)(s * sizeof(uint64_t)));
-        }
       }
     }
   } else {
@@ -464,8 +451,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int mt, nt;
       tile_coords(p, tile, mt, nt);
       mt = mt * CG + (int)rank;
-      const int buf = it & 1;
-      const uint32_t acc_ph = (it >> 1) & 1u;
+      const int buf = it % NBUF;
+      const uint32_t acc_ph = (uint32_t)(it / NBUF) & 1u;
       // destination rows of the 8 row groups this lane touches (row = quarter*32 + 4*g + lrow)
       float* rowp[8];
 #pragma unroll
@@ -575,9 +562,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float4 wn[8];   // next block of W, in flight while this block is combined and stored
 #pragma unroll
         for (int g = 0; g < 8; ++g) wn[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-        // (the compensated kernels have registers for one block of W only: they fetch the next one afterwards;
-        // their reduction loop is three times as long, so the epilogue has the time)
-        if (APPLY && !SPLIT && cc + 1 < BN / 64) {
+        if (APPLY && cc + 1 < BN / 64) {
 #pragma unroll
           for (int g = 0; g < 8; ++g)
             if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
@@ -619,11 +604,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
         }
-        if (APPLY && SPLIT && cc + 1 < BN / 64) {
-#pragma unroll
-          for (int g = 0; g < 8; ++g)
-            if (rowp[g] != nullptr && c + 32 < ncols) wn[g] = __ldcs(reinterpret_cast<const float4*>(rowp[g] + c + 32));
-        }
 #pragma unroll
         for (int g = 0; g < 8; ++g) wv[g] = wn[g];
         if (APPLY) {   // the 32 x 32 block of new W sits in the staging block, swizzled as the tensor map expects
@@ -652,7 +632,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (CG == 2) ptx::cluster_sync();   // nobody leaves while its pair may still signal it or read its tiles
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc<CG>(tmem_base, 2 * ACC_COLS);
+    ptx::tmem_dealloc<CG>(tmem_base, NBUF * ACC_COLS);
   }
 }
 
@@ -709,10 +689,10 @@ int pow2_at_least(int n) {
 }
 
 template <int ES, bool APPLY, int BN, int CG, int KA, bool FOLD, int EPI, bool SPLIT = false>
-int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w, const GemmParams& p,
-                int num_sms) {
+int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w, const CUtensorMap& ac,
+                const CUtensorMap& bc, const GemmParams& p, int num_sms) {
   constexpr int stage_bytes = (BM + BN / CG) * 128 * KA * (SPLIT ? 2 : 1);
-  constexpr int threads = NUM_THREADS + (SPLIT ? SPLIT_THREADS : 0);
+  constexpr int threads = NUM_THREADS;
   constexpr int stages = (RING_BYTES / stage_bytes) < MAX_STAGES ? (RING_BYTES / stage_bytes) : MAX_STAGES;
   constexpr int smem = stages * stage_bytes + EPI_STAGE_BYTES + 1024 + (int)sizeof(SharedCtl);
   auto kernel = umma_gemm_kernel<ES, APPLY, BN, CG, KA, FOLD, EPI, SPLIT>;
@@ -740,7 +720,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
   const int tiles = p.m_tiles * p.n_tiles * p.k_splits;
   if (CG == 1) {
     const int grid = tiles < num_sms ? tiles : num_sms;
-    kernel<<<grid, threads, smem, s>>>(a, b, w, p);
+    kernel<<<grid, threads, smem, s>>>(a, b, w, ac, bc, p);
   } else {
     const int clusters = tiles < max_clusters ? tiles : max_clusters;
     cudaLaunchConfig_t cfg;
@@ -753,7 +733,7 @@ int launch_gemm(cudaStream_t s, const CUtensorMap& a, const CUtensorMap& b, cons
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cfg.attrs = at; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kernel, a, b, w, p) != cudaSuccess) return SFB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kernel, a, b, w, ac, bc, p) != cudaSuccess) return SFB_ERR_CUDA;
   }
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
@@ -766,33 +746,61 @@ struct Variant {
   bool split;   // error-compensated tf32: 128-column tiles, one atom per stage, lo tiles made in shared memory
 };
 
+// ac / bc: tensor maps of the correction operands (compensated kernels only; the others get the plain maps again)
 template <int ES, bool APPLY, int EPI>
 int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& w,
-                const GemmParams& p, int num_sms) {
+                const CUtensorMap& ac, const CUtensorMap& bc, const GemmParams& p, int num_sms) {
   if (v.split) {
     if (ES == 4 && EPI == 0) {   // the only instantiations: fp32 operands, plain stores / W write-back
-      if (v.cg == 2 && v.fold) return launch_gemm<4, APPLY, 128, 2, 1, true, 0, true>(s, a, b, w, p, num_sms);
-      if (v.cg == 2) return launch_gemm<4, APPLY, 128, 2, 1, false, 0, true>(s, a, b, w, p, num_sms);
-      return launch_gemm<4, APPLY, 128, 1, 1, false, 0, true>(s, a, b, w, p, num_sms);
+      if (v.cg == 2 && v.fold) return launch_gemm<4, APPLY, 128, 2, 1, true, 0, true>(s, a, b, w, ac, bc, p, num_sms);
+      if (v.cg == 2) return launch_gemm<4, APPLY, 128, 2, 1, false, 0, true>(s, a, b, w, ac, bc, p, num_sms);
+      return launch_gemm<4, APPLY, 128, 1, 1, false, 0, true>(s, a, b, w, ac, bc, p, num_sms);
     }
     return SFB_ERR_UNSUPPORTED;
   }
   if (v.cg == 2) {
-    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, w, p, num_sms);
-    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, w, p, num_sms);
-    if (v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, false, EPI>(s, a, b, w, p, num_sms);
-    return launch_gemm<ES, APPLY, 256, 2, 1, false, EPI>(s, a, b, w, p, num_sms);
+    if (v.fold && v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, true, EPI>(s, a, b, w, a, b, p, num_sms);
+    if (v.fold) return launch_gemm<ES, APPLY, 256, 2, 1, true, EPI>(s, a, b, w, a, b, p, num_sms);
+    if (v.ka == 2) return launch_gemm<ES, APPLY, 256, 2, 2, false, EPI>(s, a, b, w, a, b, p, num_sms);
+    return launch_gemm<ES, APPLY, 256, 2, 1, false, EPI>(s, a, b, w, a, b, p, num_sms);
   }
-  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false, EPI>(s, a, b, w, p, num_sms);
-  if (v.ka == 2) return launch_gemm<ES, APPLY, 128, 1, 2, false, EPI>(s, a, b, w, p, num_sms);
-  return launch_gemm<ES, APPLY, 128, 1, 1, false, EPI>(s, a, b, w, p, num_sms);
+  if (v.bn == 256) return launch_gemm<ES, APPLY, 256, 1, 1, false, EPI>(s, a, b, w, a, b, p, num_sms);
+  if (v.ka == 2) return launch_gemm<ES, APPLY, 128, 1, 2, false, EPI>(s, a, b, w, a, b, p, num_sms);
+  return launch_gemm<ES, APPLY, 128, 1, 1, false, EPI>(s, a, b, w, a, b, p, num_sms);
 }
 
 template <bool APPLY, int EPI>
 int dispatch_gemm(cudaStream_t s, int es, const Variant& v, const CUtensorMap& a, const CUtensorMap& b,
-                  const CUtensorMap& w, const GemmParams& p, int num_sms) {
-  return es == 2 ? dispatch_es<2, APPLY, EPI>(s, v, a, b, w, p, num_sms)
-                 : dispatch_es<4, APPLY, EPI>(s, v, a, b, w, p, num_sms);
+                  const CUtensorMap& w, const CUtensorMap& ac, const CUtensorMap& bc, const GemmParams& p, int num_sms) {
+  return es == 2 ? dispatch_es<2, APPLY, EPI>(s, v, a, b, w, ac, bc, p, num_sms)
+                 : dispatch_es<4, APPLY, EPI>(s, v, a, b, w, ac, bc, p, num_sms);
+}
+
+// Tensor maps of the correction operands (bf16, 128-byte swizzle, always whole 128-byte atoms).
+// K-major: dst[row][atom][64] as (value, row, worker, atom), rows of all workers consecutive.
+bool encode_corr_k_map(CUtensorMap* m, const void* base, long long rows_per_worker, long long workers, long long atoms,
+                       int box_rows, int box_workers) {
+  auto fn = get_encode();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[4] = {64, (cuuint64_t)rows_per_worker, (cuuint64_t)workers, (cuuint64_t)atoms};
+  cuuint64_t strides[3] = {(cuuint64_t)atoms * 128, (cuuint64_t)rows_per_worker * atoms * 128, 128};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_workers, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// MN-major: dst[line][ldc] as (value within a chunk of 64, line, chunk); a box is 64 lines of box_chunks chunks.
+bool encode_corr_mn_map(CUtensorMap* m, const void* base, long long ldc, long long lines, int box_chunks) {
+  auto fn = get_encode();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {64, (cuuint64_t)lines, (cuuint64_t)(ldc / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)ldc * 2, 128};
+  cuuint32_t box[3] = {64, 64, (cuuint32_t)box_chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -808,6 +816,12 @@ struct UmmaPlan {
   int max_splits; // ranges a forward reduction may be cut into = partial buffers allocated
   bool x3;        // error-compensated tf32 (SFB_PATH_TF32X3): the SPLIT kernels, forward always through partial buffers
   float2* stats;  // MLR: (max, sum of exps) per (sample, half tile) from the forward GEMM's epilogue
+  // compensated kernels: correction operands of the sample rows (forward) and of the factor rows (apply),
+  // rewritten by a pre-pass before every GEMM launch
+  void* xc;
+  void* uc;
+  void* vc;
+  int ldcu, ldcv;               // padded row lengths (multiples of 64) of uc / vc
   float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
   int ldp;
   // MLR: the factor v is a copy of x that nothing in the factor stage reads, so it runs on a side stream
@@ -845,6 +859,9 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   const char* ls = getenv("SFB_TEST_LOSE_SIGNAL");
   p->lose_signal = (ls != nullptr && ls[0] == '1') ? 1 : 0;
   p->part_ws = nullptr;
+  p->xc = p->uc = p->vc = nullptr;
+  p->ldcu = (int)pad_to(d.J, 64);
+  p->ldcv = (int)pad_to(d.D, 64);
   p->ldp = (int)pad_to(d.J, 4);
   {   // forward GEMMs whose 128 x 128 tiles do not fill the SMs may split their reduction
     const long long K_ = (long long)d.P * d.B;
@@ -858,6 +875,23 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
     }
     if ((tiles < p->num_sms || p->x3) && cudaMalloc(&p->part_ws, (size_t)p->max_splits * K_ * p->ldp * 4) != cudaSuccess) {
       cudaGetLastError();
+      delete p;
+      return SFB_ERR_ALLOC;
+    }
+  }
+  if (p->x3) {
+    const size_t K_ = (size_t)d.P * d.B;
+    // reduction blocks of 32 pairs as the apply takes them: whole blocks per worker, or several workers per block
+    const size_t blocks = d.B >= 32 ? (size_t)d.P * ((d.B + 31) / 32) : ((size_t)d.P + 32 / pow2_at_least(d.B) - 1) / (32 / pow2_at_least(d.B));
+    const bool ok = cudaMalloc(&p->xc, K_ * ((d.D + 31) / 32) * 128) == cudaSuccess &&
+                    cudaMalloc(&p->uc, blocks * 64 * p->ldcu * 2) == cudaSuccess &&
+                    cudaMalloc(&p->vc, blocks * 64 * p->ldcv * 2) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      if (p->xc) cudaFree(p->xc);
+      if (p->uc) cudaFree(p->uc);
+      if (p->vc) cudaFree(p->vc);
+      if (p->part_ws) cudaFree(p->part_ws);
       delete p;
       return SFB_ERR_ALLOC;
     }
@@ -884,6 +918,9 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
     if (cudaMalloc(&p->stats, (size_t)d.P * d.B * parts * sizeof(float2)) != cudaSuccess) {
       cudaGetLastError();
       if (p->part_ws) cudaFree(p->part_ws);
+      if (p->xc) cudaFree(p->xc);
+      if (p->uc) cudaFree(p->uc);
+      if (p->vc) cudaFree(p->vc);
       delete p;
       return SFB_ERR_ALLOC;
     }
@@ -901,6 +938,9 @@ void umma_plan_destroy(UmmaPlan* p) {
   }
   if (p->stats) cudaFree(p->stats);
   if (p->part_ws) cudaFree(p->part_ws);
+  if (p->xc) cudaFree(p->xc);
+  if (p->uc) cudaFree(p->uc);
+  if (p->vc) cudaFree(p->vc);
   delete p;
 }
 
@@ -917,10 +957,7 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
     // Compensated kernels: 256 x 128 pair tiles (128 x 128 for a single row unit), one atom per stage.
     v.split = true;
     // 128 columns: main and correction accumulators of two tiles fill the 512 columns of tensor memory, so the
-    // epilogue of a tile overlaps the MMAs of the next (256-column tiles with a single set and an exposed epilogue
-    // were measured 6 % slower at 4096 x 10000, K = 1024, in spite of a third less shared-memory traffic per flop;
-    // two warps per stage instead of one stage per warp in the splitter changed nothing either: what bounds these
-    // kernels, at 43 % tensor-pipe activity, is the shared-memory read path of three MMAs per fp32 operand pair)
+    // epilogue of a tile overlaps the MMAs of the next.
     v.bn = 128; v.ka = 1;
     v.cg = m_units >= 2 ? 2 : 1;
     if (v.cg == 2 && (m_units & 1) && max_splits <= 1) {
@@ -990,7 +1027,7 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
 int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
                       float2* stats, int* n_parts_out, int* part_cols_out, int* k_splits_out, int max_splits,
-                      long long split_stride, int workers) {
+                      long long split_stride, int workers, const void* w_corr) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   const int P = workers > 0 ? workers : d.P;     // a shard of the workers, or all of them
@@ -1040,13 +1077,27 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
   if (!encode_rows_map(&tb, es, Wop, d.D, d.J, 1, (long long)d.D * es, (long long)d.D * es * d.J, v.bn / v.cg, 1,
                        v.fold, v.ka, false))
     return SFB_ERR_CUDA;
-  return stats != nullptr ? dispatch_gemm<false, 1>(s, es, v, ta, tb, ta, p, pl->num_sms)
-                          : dispatch_gemm<false, 0>(s, es, v, ta, tb, ta, p, pl->num_sms);
+  CUtensorMap tac = ta, tbc = tb;
+  int launches = 0;
+  if (pl->x3) {
+    // correction operands: the sample rows' are written here, W's come from the caller (it knows when W changed)
+    if (w_corr == nullptr) return SFB_ERR_ARG;
+    const int atoms = (d.D + 31) / 32;
+    const int r = launch_split_k(s, a, P * d.B, d.D, pl->xc, true);
+    if (r < 0) return r;
+    launches += r;
+    if (!encode_corr_k_map(&tac, pl->xc, d.B, P, atoms, p.m_bb, p.m_wp) ||
+        !encode_corr_k_map(&tbc, w_corr, d.J, 1, atoms, v.bn / v.cg, 1))
+      return SFB_ERR_CUDA;
+  }
+  const int r = stats != nullptr ? dispatch_gemm<false, 1>(s, es, v, ta, tb, ta, tac, tbc, p, pl->num_sms)
+                                 : dispatch_gemm<false, 0>(s, es, v, ta, tb, ta, tac, tbc, p, pl->num_sms);
+  return r < 0 ? r : launches + r;
 }
 
 // Sparse coding on the tensor cores: u rows = dense code rows `a` times W^T, minus the data rows.
 int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
-                    int workers) {
+                    int workers, const void* w_corr) {
   const sfb_desc& d = pl->d;
   const int K = (workers > 0 ? workers : d.P) * d.B;
   int r, launches = 0;
@@ -1056,13 +1107,14 @@ int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMa
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers,
+                               w_corr)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride)) < 0) return r;
     return launches + r;
   }
-  if ((r = umma_forward_rows(pl, s, W, a, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers)) < 0) return r;
+  if ((r = umma_forward_rows(pl, s, W, a, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers, w_corr)) < 0) return r;
   launches += r;
   if ((r = launch_finish_sc(s, u, u, Xdata, K, d.J)) < 0) return r;
   return launches + r;
@@ -1108,7 +1160,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
         const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
         int ks = 1;
         if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, pz, dev_status, nullptr, nullptr,
-                                   nullptr, &ks, pl->max_splits, sstride, workers)) < 0)
+                                   nullptr, &ks, pl->max_splits, sstride, workers, pl->x3 ? w_shadow : nullptr)) < 0)
           return r;
         launches += r;
         if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride, reinterpret_cast<float*>(aux->dual),
@@ -1118,7 +1170,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
       } else {
         int n_parts = 0, part_cols = 0;
         if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
-                                   &part_cols, nullptr, 1, 0, workers)) < 0)
+                                   &part_cols, nullptr, 1, 0, workers, pl->x3 ? w_shadow : nullptr)) < 0)
           return r;
         launches += r;
         if ((r = launch_finish_mlr_fused(s, u, pl->stats, n_parts, part_cols, aux->labels, K, d.J, dev_status,
@@ -1149,13 +1201,16 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     pz.worker_stride = (long long)d.B * pl->ldp * 4;
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
-    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers)) < 0)
+    if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers,
+                               pl->x3 ? w_shadow : nullptr)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
     return launches + r;
   }
-  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers)) < 0) return r;
+  if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers,
+                             pl->x3 ? w_shadow : nullptr)) < 0)
+    return r;
   launches += r;
   if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
   return launches + r;
@@ -1247,7 +1302,22 @@ static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return SFB_ERR_CUDA;
   }
-  return dispatch_gemm<true, 0>(s, es, v, tu, tv, tw, p, pl->num_sms);
+  CUtensorMap tuc = tu, tvc = tv;
+  int launches = 0;
+  if (pl->x3) {
+    // correction operands of this launch's factor rows, block by block as the kernel takes them (BK = 32 pairs)
+    int r = launch_split_mn(s, u_rows, d.J, workers, p.k_bb, p.k_wp, p.k_bpw, p.k_blocks, pl->uc, pl->ldcu, true);
+    if (r < 0) return r;
+    launches += r;
+    r = launch_split_mn(s, v_rows, d.D, workers, p.k_bb, p.k_wp, p.k_bpw, p.k_blocks, pl->vc, pl->ldcv, false);
+    if (r < 0) return r;
+    launches += r;
+    if (!encode_corr_mn_map(&tuc, pl->uc, pl->ldcu, (long long)p.k_blocks * 64, BM / 64) ||
+        !encode_corr_mn_map(&tvc, pl->vc, pl->ldcv, (long long)p.k_blocks * 64, (v.bn / v.cg) / 64))
+      return SFB_ERR_CUDA;
+  }
+  const int r = dispatch_gemm<true, 0>(s, es, v, tu, tv, tw, tuc, tvc, p, pl->num_sms);
+  return r < 0 ? r : launches + r;
 }
 
 }  // namespace sfb

@@ -17,13 +17,16 @@ int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16
                  const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers = 0);
 
 // Z rows (fp32) = A rows (the path's value type) times Wop^T on the tensor cores; no epilogue beyond the store.
+// w_corr: on the compensated path, W's correction operand (launch_split_k of W's rows, B side); w_shadow plays
+// that part in umma_forward.
 int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
                       float2* stats = nullptr, int* n_parts_out = nullptr, int* part_cols_out = nullptr,
-                      int* k_splits_out = nullptr, int max_splits = 1, long long split_stride = 0, int workers = 0);
+                      int* k_splits_out = nullptr, int max_splits = 1, long long split_stride = 0, int workers = 0,
+                      const void* w_corr = nullptr);
 
 // Sparse coding: u rows = dense code rows `a` (fp32) times W^T minus the data rows Xdata [K][J].
 int umma_forward_sc(UmmaPlan* p, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
-                    int workers = 0);
+                    int workers = 0, const void* w_corr = nullptr);
 
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
 // u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).

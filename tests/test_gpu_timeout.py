@@ -21,7 +21,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("path,over", [
     ("bf16", dict(J=512, D=4096, P=4, B=128, pool=1, labels="uniform")),       # single-CTA tiles, split reduction
     ("bf16", dict(J=4096, D=4096, P=8, B=256, pool=1, labels="uniform")),      # CTA pairs, fused softmax epilogue
-    ("tf32x3", dict(J=512, D=2048, P=4, B=128, pool=1, labels="uniform")),     # compensated kernels: the splitter warps leave too
+    ("tf32x3", dict(J=512, D=2048, P=4, B=128, pool=1, labels="uniform")),     # compensated kernels (four operand tiles per stage)
 ])
 def test_lost_signal_times_out_cleanly(path, over, monkeypatch):
     from paper_1511_08486_b200 import binding as B
