@@ -315,7 +315,9 @@ int sfb_create(const sfb_desc* desc, void* cuda_stream, sfb_ctx** out) {
   }
   if (ok && desc->path == SFB_PATH_BF16) ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * desc->D * 2) == cudaSuccess;
   if (ok && desc->path == SFB_PATH_TF32X3)
-    ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * ((desc->D + 31) / 32) * 128) == cudaSuccess;
+    ok = cudaMalloc(&c->w_shadow, (size_t)desc->J * ((desc->D + 31) / 32) * 128) == cudaSuccess &&
+         // columns beyond D inside the last atom are zeros for good: nothing writes them again
+         cudaMemset(c->w_shadow, 0, (size_t)desc->J * ((desc->D + 31) / 32) * 128) == cudaSuccess;
   if (ok && desc->compact) {
     ok = cudaMalloc(&c->compact_ws, (size_t)compact_workspace_bytes(c->K, desc->P)) == cudaSuccess;
     if (ok && desc->path == SFB_PATH_F32) ok = cudaMalloc(&c->kept_idx, ((size_t)c->K + 1) * 4) == cudaSuccess;
@@ -572,8 +574,9 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
     if (check)
       ACC(launch_densify_codes(c->stream, stream_codes(c, sf_buf), dense_codes(c), K, d.D, c->dev_status,
                                d.path == SFB_PATH_TF32));
-    ACC(umma_apply(c->umma, c->stream, W, nullptr, stream_u(c, sf_buf), dense_codes(c), eta, K, c->dev_status));
-    c->shadow_of = nullptr;   // W changed: a correction operand made from it is stale
+    ACC(umma_apply(c->umma, c->stream, W, has_shadow(c) ? c->w_shadow : nullptr, stream_u(c, sf_buf), dense_codes(c), eta,
+                   K, c->dev_status));
+    if (has_shadow(c)) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
   } else if (d.path == SFB_PATH_F32) {
     const int* idx = nullptr;
     const int* n_idx = nullptr;
@@ -591,8 +594,10 @@ static int apply_from(sfb_ctx* c, void* W, const void* sf_buf, float eta, int K,
   } else {
     ACC(umma_apply(c->umma, c->stream, W, c->w_shadow, stream_u(c, sf_buf), stream_v(c, sf_buf), eta, K, c->dev_status,
                    d.compact ? reinterpret_cast<const char*>(sf_buf) + 128 : nullptr));
-    if (d.path == SFB_PATH_BF16) c->shadow_of = W;   // the apply epilogue rewrote the shadow from the new W
-    else c->shadow_of = nullptr;                     // W changed: its correction operand is stale
+    // The apply epilogue rewrote the shadow from the new W.  (A compacted buffer without a single pair launches no
+    // tile: W and a shadow that mirrored it stay as they were; a stale shadow stays stale.)
+    if (has_shadow(c) && (!d.compact || c->shadow_of == W)) c->shadow_of = W;
+    else c->shadow_of = nullptr;
   }
   return SFB_OK;
 }

@@ -53,7 +53,10 @@ struct GemmParams {
   int k_bb, k_wp, k_bpw;    // apply: a reduction block is k_bb rows x k_wp workers; blocks per worker
   int Mvalid, Nvalid;       // apply: (J, D)
   float* W;                 // apply: fp32 master, row stride ldw
-  __nv_bfloat16* shadow;    // apply: bf16 copy of the new W (or nullptr)
+  // apply: bf16 copy of the new W (or nullptr); compensated kernels: W's correction operand for the next forward
+  // pass, [row][atom of 32 columns][32 values | 32 remainders], w_atoms atoms per row
+  __nv_bfloat16* shadow;
+  int w_atoms;
   long long ldw;
   float eta;
   RowMap z;                 // forward: output rows (fp32 products, or exps in the factor's storage type)
@@ -592,7 +595,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               // the new fp32 W goes out by a TMA bulk store of the whole staging block (below): fewer store
               // instructions than per-thread 16-byte stores
               *reinterpret_cast<float4*>(stage + lr * 32 + ((lq ^ (lr & 7)) << 2)) = w;
-              if (p.shadow != nullptr) {
+              if (SPLIT && p.shadow != nullptr) {
+                // the correction operand of the new W (B side: values, then remainders of what the tensor core sees)
+                const float rx = w.x - __uint_as_float(__float_as_uint(w.x) & 0xFFFFE000u);
+                const float ry = w.y - __uint_as_float(__float_as_uint(w.y) & 0xFFFFE000u);
+                const float rz = w.z - __uint_as_float(__float_as_uint(w.z) & 0xFFFFE000u);
+                const float rw = w.w - __uint_as_float(__float_as_uint(w.w) & 0xFFFFE000u);
+                __nv_bfloat162 v0 = __floats2bfloat162_rn(w.x, w.y), v1 = __floats2bfloat162_rn(w.z, w.w);
+                __nv_bfloat162 r0 = __floats2bfloat162_rn(rx, ry), r1 = __floats2bfloat162_rn(rz, rw);
+                const long long j = mt * BM + quarter * 32 + lr;
+                uint2* dst = reinterpret_cast<uint2*>(p.shadow + (j * p.w_atoms + (c >> 5)) * 64 + (c & 31));
+                __stcs(dst, make_uint2(*reinterpret_cast<uint32_t*>(&v0), *reinterpret_cast<uint32_t*>(&v1)));
+                __stcs(dst + 8, make_uint2(*reinterpret_cast<uint32_t*>(&r0), *reinterpret_cast<uint32_t*>(&r1)));
+              } else if (p.shadow != nullptr) {
                 __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
                 uint2 pk;
                 pk.x = *reinterpret_cast<uint32_t*>(&lo);
@@ -752,6 +767,8 @@ int dispatch_es(cudaStream_t s, const Variant& v, const CUtensorMap& a, const CU
                 const CUtensorMap& ac, const CUtensorMap& bc, const GemmParams& p, int num_sms) {
   if (v.split) {
     if (ES == 4 && EPI == 0) {   // the only instantiations: fp32 operands, plain stores / W write-back
+      if (v.cg == 2 && v.bn == 256 && v.fold) return launch_gemm<4, APPLY, 256, 2, 1, true, 0, true>(s, a, b, w, ac, bc, p, num_sms);
+      if (v.cg == 2 && v.bn == 256) return launch_gemm<4, APPLY, 256, 2, 1, false, 0, true>(s, a, b, w, ac, bc, p, num_sms);
       if (v.cg == 2 && v.fold) return launch_gemm<4, APPLY, 128, 2, 1, true, 0, true>(s, a, b, w, ac, bc, p, num_sms);
       if (v.cg == 2) return launch_gemm<4, APPLY, 128, 2, 1, false, 0, true>(s, a, b, w, ac, bc, p, num_sms);
       return launch_gemm<4, APPLY, 128, 1, 1, false, 0, true>(s, a, b, w, ac, bc, p, num_sms);
@@ -954,42 +971,55 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
   v.split = false;
   if (splits != nullptr) *splits = 1;
   if (pl->x3) {
-    // Compensated kernels: 256 x 128 pair tiles (128 x 128 for a single row unit), one atom per stage.
+    // Compensated kernels: one atom of the reduction per stage (fp32 tiles and their bf16 correction tiles).  These
+    // kernels run at the rate L2 delivers their operands, so a candidate shape costs the bytes its busiest SM loads:
+    //   256 x 128 pair tiles: 48 KB per stage and CTA; the accumulators (main, corrections) of two tiles fill the
+    //     512 columns of tensor memory, so a tile's epilogue overlaps the MMAs of the next;
+    //   256 x 256 pair tiles: 64 KB per stage for twice the work, but one accumulator set: the epilogue is exposed
+    //     (about 8 stages' worth per tile, measured at 4096 x 10000, K = 1024);
+    //   128 x 128 single tiles (64 KB per stage): for a single row unit, or when an odd number of row units would
+    //     leave the last pair half empty and waves of singles are shorter (an apply of 600 rows).
+    // With a split reduction (forward; ranges added in fp32 by the finishing pass) the number of ranges is chosen
+    // with the shape: enough of them that one accumulator takes at most X3_ATOMS_PER_RANGE atoms (every instruction
+    // rounds the sum toward zero, about 1.6e-8 of it), and the count with the least cost among the admissible ones
+    // (a little is added per range for its partial buffer).
     v.split = true;
-    // 128 columns: main and correction accumulators of two tiles fill the 512 columns of tensor memory, so the
-    // epilogue of a tile overlaps the MMAs of the next.
-    v.bn = 128; v.ka = 1;
-    v.cg = m_units >= 2 ? 2 : 1;
-    if (v.cg == 2 && (m_units & 1) && max_splits <= 1) {
-      // An odd number of row units leaves the last pair half empty.  Single CTAs waste nothing there but move about
-      // 192 KB through shared memory per stage where a pair's CTA moves 168 (each loads and splits all of its B tile):
-      // take them when their waves, so weighted, are shorter (600 rows: 3 waves of singles against 4 of pairs).
-      const long long n_tiles = (N + 127) / 128;
-      const long long waves_pair = (((m_units + 1) / 2) * n_tiles + pl->num_sms / 2 - 1) / (pl->num_sms / 2);
-      const long long waves_one = ((long long)m_units * n_tiles + pl->num_sms - 1) / pl->num_sms;
-      if (waves_one * 192 < waves_pair * 168) v.cg = 1;
+    v.ka = 1;
+    const bool ranged = splits != nullptr && k_atoms > 0 && max_splits > 1;
+    const long long k_len = k_atoms > 0 ? k_atoms : 32;          // atoms of the reduction (apply: 32 pairs each)
+    long long best_cost = -1;
+    auto consider = [&](int bn, int cg) {
+      const long long stage_kb = (BM + bn / cg) * 256 / 1024;    // fp32 + correction tiles of one CTA
+      const long long epi = (4 * bn > 512) ? 8 * stage_kb : 0;   // exposed epilogue, in KB loaded
+      const long long tiles = (long long)((m_units + cg - 1) / cg) * ((N + bn - 1) / bn);
+      const long long slots = pl->num_sms / cg;
+      long long ks_lo = 1, ks_hi = 1;
+      if (ranged) {
+        ks_lo = (k_len + X3_ATOMS_PER_RANGE - 1) / X3_ATOMS_PER_RANGE;
+        if (ks_lo > max_splits) ks_lo = max_splits;
+        if (ks_lo < 1) ks_lo = 1;
+        ks_hi = max_splits;
+      }
+      for (long long ks = ks_lo; ks <= ks_hi && (ks == ks_lo || k_len >= 4 * ks); ++ks) {
+        const long long per = (k_len + ks - 1) / ks;
+        const long long n_ranges = (k_len + per - 1) / per;          // ranges that exist
+        const long long waves = (tiles * n_ranges + slots - 1) / slots;
+        const long long cost = waves * (per * stage_kb + epi) + (ranged ? n_ranges * stage_kb * 3 / 8 : 0);
+        if (best_cost < 0 || cost < best_cost) {
+          best_cost = cost;
+          v.bn = bn; v.cg = cg;
+          if (splits != nullptr) *splits = (int)ks;
+        }
+      }
+    };
+    if (m_units >= 2) {
+      consider(128, 2);
+      if (N > 128) consider(256, 2);
+      if ((m_units & 1) && !ranged) consider(128, 1);
+    } else {
+      consider(128, 1);
     }
     v.fold = v.cg == 2 && dims_chunk_aligned;
-    if (splits != nullptr && k_atoms > 0 && max_splits > 1) {
-      // Ranges of the reduction, added in fp32 by the finishing pass: enough of them that one accumulator takes
-      // at most X3_ATOMS_PER_RANGE atoms (4 instructions each; every instruction rounds the sum toward zero,
-      // about 1.6e-8 of it), and enough to give every SM work.
-      // Among the admissible counts the one with the least work on the busiest SM pair is taken: waves of
-      // (tile, range) items times the atoms of a range, plus a little per range for its partial buffer.
-      const long long tiles = (long long)((m_units + v.cg - 1) / v.cg) * ((N + 127) / 128);
-      const long long slots = pl->num_sms / v.cg;
-      long long ks_min = (k_atoms + X3_ATOMS_PER_RANGE - 1) / X3_ATOMS_PER_RANGE;
-      if (ks_min > max_splits) ks_min = max_splits;
-      long long best = ks_min < 1 ? 1 : ks_min, best_cost = -1;
-      for (long long ks = best; ks <= max_splits && (ks == best || k_atoms >= 4 * ks); ++ks) {
-        const long long per = (k_atoms + ks - 1) / ks;
-        const long long n_ranges = (k_atoms + per - 1) / per;          // ranges that exist
-        const long long waves = (tiles * n_ranges + slots - 1) / slots;
-        const long long cost = waves * per * 8 + n_ranges * 3;          // in eighths of an atom
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = ks; }
-      }
-      *splits = (int)best;
-    }
     return v;
   }
   v.bn = (N > 128 && (long long)m_units * ((N + 255) / 256) >= pl->num_sms) ? 256 : 128;
@@ -1259,7 +1289,7 @@ static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16
   // stream (the next row, or the stream's V block: always inside the buffer), which only feeds accumulator rows
   // j >= J, and those are never written.  (The V block of the last stream ends the buffer, hence no such
   // licence for D.)
-  const Variant v = pick_variant(pl, m_units, d.D, (d.D % CH) == 0);
+  const Variant v = pick_variant(pl, m_units, d.D, (d.D % CH) == 0, pl->x3 ? (K + 31) / 32 : 0);
   const int BK = CH * v.ka;
   if (d.B >= BK) { p.k_bb = BK; p.k_wp = 1; p.k_bpw = (d.B + BK - 1) / BK; p.k_blocks = workers * p.k_bpw; }
   else { p.k_bb = pow2_at_least(d.B); p.k_wp = BK / p.k_bb; p.k_bpw = 1; p.k_blocks = (workers + p.k_wp - 1) / p.k_wp; }
@@ -1275,7 +1305,8 @@ static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16
   p.b_policy = p.m_fastest ? 0 : 2;
   p.group = APPLY_GROUP;
   p.W = reinterpret_cast<float*>(W);
-  p.shadow = (d.path == SFB_PATH_BF16) ? w_shadow : nullptr;
+  p.shadow = (d.path == SFB_PATH_BF16 || pl->x3) ? w_shadow : nullptr;
+  p.w_atoms = (d.D + 31) / 32;
   p.ldw = d.D;
   p.eta = eta;
   p.status_ro = dev_status;
