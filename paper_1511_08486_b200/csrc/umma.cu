@@ -823,7 +823,7 @@ bool encode_corr_mn_map(CUtensorMap* m, const void* base, long long ldc, long lo
 }  // namespace
 
 constexpr int MAX_SPLITS = 8;   // ranges a forward reduction may be cut into (partial buffers of the plan)
-constexpr int X3_MAX_SPLITS = 16;   // ... on the compensated path, where the count is also tuned to fill whole waves
+constexpr int X3_MAX_SPLITS = 32;   // ... on the compensated path, where the count is also tuned to fill whole waves
 
 struct UmmaPlan {
   sfb_desc d;
