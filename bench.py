@@ -44,11 +44,12 @@ BURST_REGION_S = 1.0
 
 def tensor_peak(peaks, path, region_s):
     """(peak TFLOP/s, label) for a tensor-core kernel timed inside a region of `region_s` seconds."""
-    # tf32 nominal rate is half of bf16; the compensated path spends three tensor-core products per algorithmic one
-    scale = {"bf16": 1.0, "tf32": 0.5, "tf32x3": 0.5 / 3.0}[path]
+    # tf32 nominal rate is half of bf16; the compensated path spends, per algorithmic product, one tf32 product and
+    # one bf16 product of twice the reduction length (as long as a tf32 one): two tf32 products' worth
+    scale = {"bf16": 1.0, "tf32": 0.5, "tf32x3": 0.5 / 2.0}[path]
     kind = "burst" if region_s < BURST_REGION_S else "sustained"
     base = peaks["bf16"] if kind == "burst" else peaks["bf16_sustained"]
-    label = (f"{peaks['source']} cuBLAS bf16 {kind} ({base:.1f})" + {"bf16": "", "tf32": " x 0.5 (tf32)", "tf32x3": " x 0.5 (tf32) / 3 (three products per multiply-add)"}[path] +
+    label = (f"{peaks['source']} cuBLAS bf16 {kind} ({base:.1f})" + {"bf16": "", "tf32": " x 0.5 (tf32)", "tf32x3": " x 0.5 (tf32) / 2 (a tf32 product and a bf16 correction product of the same length per multiply-add)"}[path] +
              f": timed region {region_s * 1e3:.0f} ms")
     return base * scale, label, scale
 
@@ -553,7 +554,7 @@ def main():
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": {"f32": "f32", "tf32": "tf32", "bf16": "bf16", "tf32x3": "tf32x3 (fp32 operands as three tf32 products)"}[path],
+            "scaling": "weak", "vs_baseline": None, "dtype": {"f32": "f32", "tf32": "tf32", "bf16": "bf16", "tf32x3": "tf32x3 (fp32 operands: tf32 product + bf16 correction product, fp32 accumulate)"}[path],
             "data": "synthetic",
             "config": {"workload": workload_name(cfg, path), "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "per-step footprint larger than L2" if flush is None else "L2 flushed between steps",

@@ -44,10 +44,13 @@
  *                  bf16 in memory; W stays an fp32 master and the context keeps a bf16 shadow of
  *                  it that the apply refreshes.
  *   SFB_PATH_TF32X3  tensor cores with error compensation, for fp32-grade results (the tolerance class of
- *                  SFB_PATH_F32): every fp32 operand is split, inside the kernel, into the part the tensor core
- *                  sees (its top 10 mantissa bits) and the exact remainder, and each product is formed from
- *                  three tensor-core multiplications (a b ~ hi hi + lo hi + hi lo); X, U, V fp32 in memory,
- *                  same wire format as SFB_PATH_TF32.  The tensor core's fp32 accumulator rounds toward zero
+ *                  SFB_PATH_F32): every fp32 operand x is the part the tensor core sees (its top 10 mantissa
+ *                  bits, hi) plus an exact remainder lo, and a product is formed as a b ~ hi hi + lo b + a lo:
+ *                  hi hi by a tf32 multiplication of the operands as they are, the two corrections by one bf16
+ *                  multiplication of "correction operands" [lo(a) | a] and [b | lo(b)] that a pre-pass (and,
+ *                  for W, the apply's write-back) keeps in the context's workspace; X, U, V fp32 in memory,
+ *                  same wire format as SFB_PATH_TF32.  The context caches W's correction operand like the
+ *                  bf16 shadow (sfb_invalidate).  The tensor core's fp32 accumulator rounds toward zero
  *                  once per instruction of 8 reduction steps, which costs about 1.6e-8 of a sum per
  *                  instruction: forward reductions are cut into ranges that are added in fp32 afterwards, and
  *                  updates of more than 1024 pairs are applied to W in several launches of whole worker streams.
@@ -257,7 +260,8 @@ int sfb_active_pairs(sfb_ctx* ctx, int32_t* n);
  * padding is not counted.  Synchronises the stream (reads the directory back). */
 int sfb_wire_bytes(sfb_ctx* ctx, const void* sf_buf, uint64_t* bytes);
 
-/* Tells the context that W was changed by someone else, so a cached bf16 shadow is stale. */
+/* Tells the context that W was changed by someone else, so what it caches of W (the bf16 shadow of
+ * SFB_PATH_BF16, the correction operand of SFB_PATH_TF32X3) is stale. */
 int sfb_invalidate(sfb_ctx* ctx);
 
 /* Synchronises the stream, returns the sticky device status word in *device_status and clears it. */
