@@ -164,8 +164,10 @@ int ensure_shadow(sfb_ctx* c, const void* W) {
 
 // Factors of one minibatch written through the row maps u / v (v.base == nullptr: v not wanted).
 // workers > 0: the minibatch holds only that many workers' samples and u / v / codes start at the first of them.
+// for_apply: the apply of exactly these rows (all K pairs, no compaction in between) follows in the same call, so
+// the compensated path may write the apply's correction operands while it writes the factors.
 int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, RowMap u, RowMap v, CsrView codes,
-                 int workers = 0) {
+                 int workers = 0, bool for_apply = false) {
   const sfb_desc& d = c->d;
   const int K = workers > 0 ? workers * d.B : c->K;
   const float* Wf = reinterpret_cast<const float*>(W);
@@ -184,7 +186,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
       if (r < 0) return r;
     }
     ACC(umma_forward_sc(c->umma, c->stream, W, a, u, reinterpret_cast<const float*>(aux->Xdata), c->dev_status, workers,
-                        c->w_shadow));
+                        c->w_shadow, for_apply));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {
@@ -218,7 +220,7 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     const int r = ensure_shadow(c, W);
     if (r < 0) return r;
   }
-  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, c->dev_status, workers));
+  ACC(umma_forward(c->umma, c->stream, W, c->w_shadow, X, aux, u, v, c->dev_status, workers, for_apply));
   return SFB_OK;
 }
 
@@ -701,7 +703,8 @@ int sfb_step(sfb_ctx* c, void* W, const void* X, const sfb_aux* aux, void* sf_bu
     join_aux();
     return SFB_ERR_CUDA;
   }
-  r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes);
+  r = factors_into(c, W, X, aux, stream_u(c, sf_buf), d.v_sparse ? RowMap() : stream_v(c, sf_buf), codes, 0,
+                   d.path == SFB_PATH_TF32X3 && !d.compact && K == c->K);
   if (forked && cudaStreamWaitEvent(c->stream, c->aux_join, 0) != cudaSuccess) return SFB_ERR_CUDA;
   if (r < 0) return r;
   // pairs whose u came out as zero are dropped from the message before it is "sent" (and applied)

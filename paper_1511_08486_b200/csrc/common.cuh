@@ -32,6 +32,47 @@ struct Layout {
 
 static inline long long pad_to(long long n, long long a) { return (n + a - 1) / a * a; }
 
+// Optional extra outputs of a kernel that writes fp32 factor rows on the compensated tf32 path: the rows'
+// bf16 correction operands (split.cu), so that no separate pass has to read the rows again.
+//   mn: for the apply (MN-major), [block of 32 pairs][64 lines][ldc]; pair (worker w, row r) sits in block
+//       w * k_bpw + r / 32, line r % 32 (k_wp == 1: whole blocks per worker), or in block w / k_wp, line
+//       (w % k_wp) * k_bb + r (k_bb rows of each of k_wp workers per block); a_side: remainder lines first.
+//   km: for the forward (K-major A side), [pair][atom][32 remainders | 32 values].
+struct CorrOut {
+  char* mn;
+  char* km;
+  int ldc, k_bb, k_wp, k_bpw, a_side, atoms;
+  __host__ __device__ CorrOut() : mn(nullptr), km(nullptr), ldc(0), k_bb(32), k_wp(1), k_bpw(1), a_side(0), atoms(0) {}
+};
+#ifdef __CUDACC__
+// values t of pair i (B pairs per worker) at columns j .. j + 3, j a multiple of 4
+__device__ __forceinline__ void corr_store4(const CorrOut& c, int i, int B, int j, float4 t) {
+  const float rx = t.x - __uint_as_float(__float_as_uint(t.x) & 0xFFFFE000u);
+  const float ry = t.y - __uint_as_float(__float_as_uint(t.y) & 0xFFFFE000u);
+  const float rz = t.z - __uint_as_float(__float_as_uint(t.z) & 0xFFFFE000u);
+  const float rw = t.w - __uint_as_float(__float_as_uint(t.w) & 0xFFFFE000u);
+  const __nv_bfloat162 v0 = __floats2bfloat162_rn(t.x, t.y), v1 = __floats2bfloat162_rn(t.z, t.w);
+  const __nv_bfloat162 r0 = __floats2bfloat162_rn(rx, ry), r1 = __floats2bfloat162_rn(rz, rw);
+  const uint2 val = make_uint2(*reinterpret_cast<const uint32_t*>(&v0), *reinterpret_cast<const uint32_t*>(&v1));
+  const uint2 rem = make_uint2(*reinterpret_cast<const uint32_t*>(&r0), *reinterpret_cast<const uint32_t*>(&r1));
+  if (c.mn != nullptr && j < c.ldc) {
+    const int w = i / B, r = i - w * B;
+    long long blk;
+    int line;
+    if (c.k_wp == 1) { blk = (long long)w * c.k_bpw + (r >> 5); line = r & 31; }
+    else { blk = w / c.k_wp; line = (w % c.k_wp) * c.k_bb + r; }
+    char* base = c.mn + ((blk * 64) * c.ldc + j) * 2;
+    *reinterpret_cast<uint2*>(base + (long long)(c.a_side ? line : 32 + line) * c.ldc * 2) = rem;
+    *reinterpret_cast<uint2*>(base + (long long)(c.a_side ? 32 + line : line) * c.ldc * 2) = val;
+  }
+  if (c.km != nullptr && (j >> 5) < c.atoms) {
+    char* atom = c.km + (((long long)i * c.atoms + (j >> 5)) * 64 + (j & 31)) * 2;
+    *reinterpret_cast<uint2*>(atom) = rem;
+    *reinterpret_cast<uint2*>(atom + 64) = val;
+  }
+}
+#endif
+
 static inline Layout make_layout(const sfb_desc& d) {
   Layout l;
   l.es = (d.path == SFB_PATH_BF16) ? 2 : 4;
@@ -78,7 +119,7 @@ struct PerDeviceOnce {
 // with few tiles has its reduction cut into *nsplit_out ranges whose partial products go to `part` instead
 // of `z` (the finishing pass sums them in range order); forward_f32_splits tells how many in advance.
 // v rows = Xa rows - Xb rows, one fp32 subtraction per element, pad columns zero (the DML factor v).
-int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D);
+int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D, CorrOut corr = CorrOut());
 int forward_f32_splits(int K, int J, int D);
 // The same contraction through transposed copies of both operands (two transposing passes, then the pipelined
 // large-tile kernel).  src: operand rows a_i behind a row map; copy (optional): those rows also written there;
@@ -101,17 +142,18 @@ int launch_apply_f32(cudaStream_t s, float* W, RowMap u, RowMap v, int K, int J,
 // dual (optional, SDCA): fp32 dual variables of the K samples, [K][J rounded up to 4], updated in place; the factor
 // written to u is then the dual step sdca_step * (dual + softmax - onehot).
 int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
-                      int nsplit = 1, long long split_stride_bytes = 0, float* dual = nullptr, float sdca_step = 0.f);
+                      int nsplit = 1, long long split_stride_bytes = 0, float* dual = nullptr, float sdca_step = 0.f,
+                      CorrOut corr = CorrOut());
 
 // DML epilogue: u = +z (similar) or -z * [|z|^2 < margin] (dissimilar).
 // active (optional, [K] bytes): 1 where the pair contributes (similar, or dissimilar inside the margin), 0 where u_i = 0.
 int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
-                      int nsplit = 1, long long split_stride_bytes = 0, uint8_t* active = nullptr);
+                      int nsplit = 1, long long split_stride_bytes = 0, uint8_t* active = nullptr, CorrOut corr = CorrOut());
 // idx[0 .. *n_out) = ascending list of the samples i < K with active[i] != 0 (device arrays; one ordered block).
 int launch_compact_active(cudaStream_t s, const uint8_t* active, int K, int* idx, int* n_out);
 
 // Copies K rows of `cols` values from src to dst rows (same value type), zero-filling dst pad columns.
-int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols);
+int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols, CorrOut corr = CorrOut());
 
 // Writes header and directory of the SF buffer.  `rowptr` (global CSR row pointers) only for sparse v.
 int launch_write_header(cudaStream_t s, void* sf_buf, const sfb_desc& d, const Layout& l, uint32_t clock,
@@ -178,7 +220,7 @@ int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, 
 // SC epilogue on dense products: u = z - x in place (u rows hold z), pad columns zero.
 // z: products (possibly `nsplit` partials); u = sum of partials - x.
 int launch_finish_sc(cudaStream_t s, RowMap z, RowMap u, const float* Xdata, int K, int J, int nsplit = 1,
-                     long long split_stride_bytes = 0);
+                     long long split_stride_bytes = 0, CorrOut corr = CorrOut());
 
 // Column-norm projection: every column of W with 2-norm above 1 is divided by its norm (in place).
 int launch_prox_unit_columns(cudaStream_t s, float* W, int J, int D);

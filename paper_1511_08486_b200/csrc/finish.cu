@@ -87,7 +87,7 @@ __device__ __forceinline__ float4 sdca_step4(float* dual_row, int j, int J, floa
 
 __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, const int32_t* __restrict__ labels,
                                                                  int K, int J, int cache_floats, int* dev_status, int nsplit, long long zstride,
-                                                                 float* __restrict__ dual, float sdca_step) {
+                                                                 float* __restrict__ dual, float sdca_step, CorrOut corr) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -157,12 +157,13 @@ __global__ void __launch_bounds__(1024) finish_mlr_kernel(RowMap z, RowMap u, co
     }
     if (dual != nullptr && q < J4) t = sdca_step4(dual + (size_t)i * (J4 * 4), j, J, t, sdca_step, bad);
     store_u4(ur, j, t, u.es);
+    if (corr.mn != nullptr) corr_store4(corr, i, u.B, j, t);
   }
 }
 
 __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, const uint8_t* __restrict__ similar,
                                                                  float margin, int K, int J, int cache_floats, int nsplit, long long zstride,
-                                                                 uint8_t* __restrict__ active) {
+                                                                 uint8_t* __restrict__ active, CorrOut corr) {
   extern __shared__ __align__(16) float cache[];
   __shared__ float red[32];
   const int i = blockIdx.x;
@@ -199,6 +200,7 @@ __global__ void __launch_bounds__(1024) finish_dml_kernel(RowMap z, RowMap u, co
       if (j + 3 >= J) t.w = 0.f;
     }
     store_u4(ur, j, t, u.es);
+    if (corr.mn != nullptr) corr_store4(corr, i, u.B, j, t);
   }
 }
 
@@ -309,7 +311,7 @@ __global__ void __launch_bounds__(256) prox_unit_columns_kernel(float* __restric
 }
 
 // 16-byte-vectorised row copy; rows are whole numbers of 16-byte units on both sides.
-__global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, int K, int cols) {
+__global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, int K, int cols, CorrOut corr) {
   const int units_dst = dst.ld * dst.es / 16;
   const int per = 16 / dst.es;
   const long long total = (long long)K * units_dst;
@@ -333,12 +335,15 @@ __global__ void __launch_bounds__(256) copy_rows_kernel(RowMap src, RowMap dst, 
       }
     }
     *reinterpret_cast<uint4*>(dst.row(i) + (size_t)q * 16) = val;
+    if (corr.mn != nullptr || corr.km != nullptr)   // fp32 rows only (the compensated path)
+      corr_store4(corr, i, dst.B, c, make_float4(__uint_as_float(val.x), __uint_as_float(val.y), __uint_as_float(val.z),
+                                                 __uint_as_float(val.w)));
   }
 }
 
 // v rows = Xa - Xb (one fp32 subtraction per element), pad columns zero; 4 values per thread.
 __global__ void __launch_bounds__(256) diff_rows_kernel(const float* __restrict__ Xa, const float* __restrict__ Xb, RowMap v,
-                                                        int K, int D) {
+                                                        int K, int D, CorrOut corr) {
   const int units = v.ld >> 2;
   const long long total = (long long)K * units;
   for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
@@ -355,6 +360,7 @@ __global__ void __launch_bounds__(256) diff_rows_kernel(const float* __restrict_
         if (c + q < D) e[q] = __fsub_rn(Xa[(size_t)i * D + c + q], Xb[(size_t)i * D + c + q]);
     }
     *reinterpret_cast<float4*>(v.row(i) + (size_t)c * 4) = r;
+    if (corr.mn != nullptr || corr.km != nullptr) corr_store4(corr, i, v.B, c, r);
   }
 }
 
@@ -381,7 +387,7 @@ int fin_cache_floats(int J) {
 }  // namespace
 
 int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels, int K, int J, int* dev_status,
-                      int nsplit, long long split_stride_bytes, float* dual, float sdca_step) {
+                      int nsplit, long long split_stride_bytes, float* dual, float sdca_step, CorrOut corr) {
   const int cf = fin_cache_floats(J);
   static PerDeviceOnce attr_once;   // function attributes are per device
   if (attr_once.first()) {
@@ -389,7 +395,7 @@ int launch_finish_mlr(cudaStream_t s, RowMap z, RowMap u, const int32_t* labels,
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
   }
   finish_mlr_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, labels, K, J, cf, dev_status, nsplit, split_stride_bytes / 4,
-                                                              dual, sdca_step);
+                                                              dual, sdca_step, corr);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
@@ -428,7 +434,7 @@ int launch_compact_active(cudaStream_t s, const uint8_t* active, int K, int* idx
 }
 
 int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar, float margin, int K, int J,
-                      int nsplit, long long split_stride_bytes, uint8_t* active) {
+                      int nsplit, long long split_stride_bytes, uint8_t* active, CorrOut corr) {
   const int cf = fin_cache_floats(J);
   static PerDeviceOnce attr_once;   // function attributes are per device
   if (attr_once.first()) {
@@ -436,7 +442,7 @@ int launch_finish_dml(cudaStream_t s, RowMap z, RowMap u, const uint8_t* similar
     cudaFuncSetAttribute(finish_dml_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ROW_CACHE_FLOATS * 4);
   }
   finish_dml_kernel<<<K, fin_threads(J), (size_t)cf * 4, s>>>(z, u, similar, margin, K, J, cf, nsplit, split_stride_bytes / 4,
-                                                              active);
+                                                              active, corr);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
@@ -456,18 +462,18 @@ int launch_prox_unit_columns(cudaStream_t s, float* W, int J, int D) {
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
-int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols) {
+int launch_copy_rows(cudaStream_t s, RowMap src, RowMap dst, int K, int cols, CorrOut corr) {
   const long long total = (long long)K * (dst.ld * dst.es / 16);
   if (total == 0) return 0;
   const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
-  copy_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, K, cols);
+  copy_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, K, cols, corr);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 
-int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D) {
+int launch_diff_rows(cudaStream_t s, const float* Xa, const float* Xb, RowMap v, int K, int D, CorrOut corr) {
   const long long total = (long long)K * (v.ld >> 2);
   const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
-  diff_rows_kernel<<<blocks, 256, 0, s>>>(Xa, Xb, v, K, D);
+  diff_rows_kernel<<<blocks, 256, 0, s>>>(Xa, Xb, v, K, D, corr);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

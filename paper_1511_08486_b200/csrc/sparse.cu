@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, i
 }
 
 __global__ void __launch_bounds__(256) finish_sc_kernel(RowMap zr, RowMap u, const float* __restrict__ Xdata, int K, int J,
-                                                        int nsplit, long long zstride) {
+                                                        int nsplit, long long zstride, CorrOut corr) {
   const int units = u.ld >> 2;
   const long long total = (long long)K * units;
   for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(256) finish_sc_kernel(RowMap zr, RowMap u, con
     z.z = (j + 2 < J) ? z.z - x[j + 2] : 0.f;
     z.w = (j + 3 < J) ? z.w - x[j + 3] : 0.f;
     *p = z;
+    if (corr.mn != nullptr) corr_store4(corr, i, u.B, j, z);
   }
 }
 
@@ -334,10 +335,10 @@ int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, 
 }
 
 int launch_finish_sc(cudaStream_t s, RowMap z, RowMap u, const float* Xdata, int K, int J, int nsplit,
-                     long long split_stride_bytes) {
+                     long long split_stride_bytes, CorrOut corr) {
   const long long total = (long long)K * (u.ld >> 2);
   const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
-  finish_sc_kernel<<<blocks, 256, 0, s>>>(z, u, Xdata, K, J, nsplit, split_stride_bytes / 4);
+  finish_sc_kernel<<<blocks, 256, 0, s>>>(z, u, Xdata, K, J, nsplit, split_stride_bytes / 4, corr);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

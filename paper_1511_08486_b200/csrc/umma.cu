@@ -839,6 +839,12 @@ struct UmmaPlan {
   void* uc;
   void* vc;
   int ldcu, ldcv;               // padded row lengths (multiples of 64) of uc / vc
+  // Set by a factor stage that wrote uc / vc itself, beside the factors (its finishing pass, its copy of v): the
+  // rows they were made from and how many pairs.  The next apply of exactly those rows skips its pre-pass; any
+  // other call clears them.
+  const void* fresh_u;
+  const void* fresh_v;
+  int fresh_K;
   float* part_ws;               // partial products of a split reduction, [MAX_SPLITS][K][ldp] fp32 (small forward GEMMs only)
   int ldp;
   // MLR: the factor v is a copy of x that nothing in the factor stage reads, so it runs on a side stream
@@ -877,6 +883,8 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
   p->lose_signal = (ls != nullptr && ls[0] == '1') ? 1 : 0;
   p->part_ws = nullptr;
   p->xc = p->uc = p->vc = nullptr;
+  p->fresh_u = p->fresh_v = nullptr;
+  p->fresh_K = 0;
   p->ldcu = (int)pad_to(d.J, 64);
   p->ldcv = (int)pad_to(d.D, 64);
   p->ldp = (int)pad_to(d.J, 4);
@@ -900,9 +908,14 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out) {
     const size_t K_ = (size_t)d.P * d.B;
     // reduction blocks of 32 pairs as the apply takes them: whole blocks per worker, or several workers per block
     const size_t blocks = d.B >= 32 ? (size_t)d.P * ((d.B + 31) / 32) : ((size_t)d.P + 32 / pow2_at_least(d.B) - 1) / (32 / pow2_at_least(d.B));
+    // zeroed once: what no writer touches (columns beyond a row's padded length, lines of rows that do not exist,
+    // the tail of a row's last atom) must read as zeros, as the fp32 operands' out-of-range elements do
     const bool ok = cudaMalloc(&p->xc, K_ * ((d.D + 31) / 32) * 128) == cudaSuccess &&
                     cudaMalloc(&p->uc, blocks * 64 * p->ldcu * 2) == cudaSuccess &&
-                    cudaMalloc(&p->vc, blocks * 64 * p->ldcv * 2) == cudaSuccess;
+                    cudaMalloc(&p->vc, blocks * 64 * p->ldcv * 2) == cudaSuccess &&
+                    cudaMemset(p->xc, 0, K_ * ((d.D + 31) / 32) * 128) == cudaSuccess &&
+                    cudaMemset(p->uc, 0, blocks * 64 * p->ldcu * 2) == cudaSuccess &&
+                    cudaMemset(p->vc, 0, blocks * 64 * p->ldcv * 2) == cudaSuccess;
     if (!ok) {
       cudaGetLastError();
       if (p->xc) cudaFree(p->xc);
@@ -1057,7 +1070,7 @@ static Variant pick_variant(const UmmaPlan* pl, int m_units, int N, bool dims_ch
 // Z rows (fp32, through `z`) = A rows (through `a`, the path's value type) times W^T.
 int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
                       float2* stats, int* n_parts_out, int* part_cols_out, int* k_splits_out, int max_splits,
-                      long long split_stride, int workers, const void* w_corr) {
+                      long long split_stride, int workers, const void* w_corr, bool a_corr_ready) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   const int P = workers > 0 ? workers : d.P;     // a shard of the workers, or all of them
@@ -1113,9 +1126,11 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
     // correction operands: the sample rows' are written here, W's come from the caller (it knows when W changed)
     if (w_corr == nullptr) return SFB_ERR_ARG;
     const int atoms = (d.D + 31) / 32;
-    const int r = launch_split_k(s, a, P * d.B, d.D, pl->xc, true);
-    if (r < 0) return r;
-    launches += r;
+    if (!a_corr_ready) {   // (the kernel that made the rows may have written their correction operand with them)
+      const int r = launch_split_k(s, a, P * d.B, d.D, pl->xc, true);
+      if (r < 0) return r;
+      launches += r;
+    }
     if (!encode_corr_k_map(&tac, pl->xc, d.B, P, atoms, p.m_bb, p.m_wp) ||
         !encode_corr_k_map(&tbc, w_corr, d.J, 1, atoms, v.bn / v.cg, 1))
       return SFB_ERR_CUDA;
@@ -1126,11 +1141,27 @@ int umma_forward_rows(UmmaPlan* pl, cudaStream_t s, const void* Wop, RowMap a, R
 }
 
 // Sparse coding on the tensor cores: u rows = dense code rows `a` times W^T, minus the data rows.
+// Geometry of the apply's reduction blocks (32 pairs each) for a kernel that writes a correction operand.
+static CorrOut apply_corr(const UmmaPlan* pl, void* dst, int ldc, bool a_side) {
+  CorrOut c;
+  c.mn = reinterpret_cast<char*>(dst);
+  c.ldc = ldc;
+  c.a_side = a_side ? 1 : 0;
+  const int B = pl->d.B;
+  if (B >= 32) { c.k_bb = 32; c.k_wp = 1; c.k_bpw = (B + 31) / 32; }
+  else { c.k_bb = pow2_at_least(B); c.k_wp = 32 / c.k_bb; c.k_bpw = 1; }
+  return c;
+}
+
 int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
-                    int workers, const void* w_corr) {
+                    int workers, const void* w_corr, bool for_apply) {
   const sfb_desc& d = pl->d;
   const int K = (workers > 0 ? workers : d.P) * d.B;
   int r, launches = 0;
+  pl->fresh_u = pl->fresh_v = nullptr;
+  pl->fresh_K = 0;
+  const bool emit = pl->x3 && for_apply && workers == 0;
+  const CorrOut cu = emit ? apply_corr(pl, pl->uc, pl->ldcu, true) : CorrOut();
   if (pl->part_ws != nullptr) {   // reduction in ranges (few tiles, or the compensated path): summed by the finishing pass
     RowMap pz;
     pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
@@ -1141,20 +1172,29 @@ int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMa
                                w_corr)) < 0)
       return r;
     launches += r;
-    if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride)) < 0) return r;
+    if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride, cu)) < 0) return r;
+    if (emit) { pl->fresh_u = u.base; pl->fresh_K = K; }
     return launches + r;
   }
   if ((r = umma_forward_rows(pl, s, W, a, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers, w_corr)) < 0) return r;
   launches += r;
-  if ((r = launch_finish_sc(s, u, u, Xdata, K, d.J)) < 0) return r;
+  if ((r = launch_finish_sc(s, u, u, Xdata, K, d.J, 1, 0, cu)) < 0) return r;
+  if (emit) { pl->fresh_u = u.base; pl->fresh_K = K; }
   return launches + r;
 }
 
 int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
-                 const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers) {
+                 const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers, bool for_apply) {
   const sfb_desc& d = pl->d;
   const int K = (workers > 0 ? workers : d.P) * d.B;
   int launches = 0, r;
+  pl->fresh_u = pl->fresh_v = nullptr;
+  pl->fresh_K = 0;
+  // compensated path, apply of these very rows to follow: the kernels that write u and v also write the apply's
+  // correction operands
+  const bool emit = pl->x3 && for_apply && workers == 0;
+  const CorrOut cu = emit ? apply_corr(pl, pl->uc, pl->ldcu, true) : CorrOut();
+  CorrOut cv = emit ? apply_corr(pl, pl->vc, pl->ldcv, false) : CorrOut();
   RowMap x_rows;
   x_rows.base = const_cast<char*>(reinterpret_cast<const char*>(X));
   x_rows.ld = d.D; x_rows.B = d.B; x_rows.es = pl->es;
@@ -1177,7 +1217,7 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     };
     auto body = [&]() -> int {
       if (forked) {
-        if ((r = launch_copy_rows(pl->side, x_rows, v, K, d.D)) < 0) return r;
+        if ((r = launch_copy_rows(pl->side, x_rows, v, K, d.D, cv)) < 0) return r;
         launches += r;
       }
       // the GEMM epilogue leaves exp(z - local max) in u and (max, sum) per half tile; the finishing
@@ -1194,9 +1234,10 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
           return r;
         launches += r;
         if ((r = launch_finish_mlr(s, pz, u, aux->labels, K, d.J, dev_status, ks, sstride, reinterpret_cast<float*>(aux->dual),
-                                   aux->sdca_step)) < 0)
+                                   aux->sdca_step, cu)) < 0)
           return r;
         launches += r;
+        if (emit) { pl->fresh_u = u.base; pl->fresh_K = K; }
       } else {
         int n_parts = 0, part_cols = 0;
         if ((r = umma_forward_rows(pl, s, bf16 ? (const void*)w_shadow : W, x_rows, u, dev_status, pl->stats, &n_parts,
@@ -1209,20 +1250,26 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
         launches += r;
       }
       if (!forked && v.base != nullptr) {
-        if ((r = launch_copy_rows(s, x_rows, v, K, d.D)) < 0) return r;
+        if ((r = launch_copy_rows(s, x_rows, v, K, d.D, cv)) < 0) return r;
         launches += r;
       }
       return 0;
     };
     const int rb = body();
     const int rj = join_side();
+    if (rb < 0 || rj < 0) pl->fresh_u = nullptr;
     if (rb < 0) return rb;
     if (rj < 0) return rj;
+    if (pl->fresh_u != nullptr && v.base != nullptr) pl->fresh_v = v.base;
     return launches;
   }
   // DML (TF32): the pair differences are the factor v and the GEMM operand
   if (v.base == nullptr) return SFB_ERR_ARG;
-  if ((r = launch_diff_rows(s, reinterpret_cast<const float*>(X), reinterpret_cast<const float*>(aux->Xb), v, K, d.D)) < 0)
+  if (pl->x3) {   // ... and the forward's own correction operand of the differences
+    cv.km = reinterpret_cast<char*>(pl->xc);
+    cv.atoms = (d.D + 31) / 32;
+  }
+  if ((r = launch_diff_rows(s, reinterpret_cast<const float*>(X), reinterpret_cast<const float*>(aux->Xb), v, K, d.D, cv)) < 0)
     return r;
   launches += r;
   if (pl->part_ws != nullptr) {
@@ -1232,27 +1279,38 @@ int umma_forward(UmmaPlan* pl, cudaStream_t s, const void* W, const __nv_bfloat1
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
     if ((r = umma_forward_rows(pl, s, W, v, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers,
-                               pl->x3 ? w_shadow : nullptr)) < 0)
+                               pl->x3 ? w_shadow : nullptr, pl->x3)) < 0)
       return r;
     launches += r;
-    if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride)) < 0) return r;
+    if ((r = launch_finish_dml(s, pz, u, aux->similar, d.margin, K, d.J, ks, sstride, nullptr, cu)) < 0) return r;
+    if (emit) { pl->fresh_u = u.base; pl->fresh_v = v.base; pl->fresh_K = K; }
     return launches + r;
   }
   if ((r = umma_forward_rows(pl, s, W, v, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers,
-                             pl->x3 ? w_shadow : nullptr)) < 0)
+                             pl->x3 ? w_shadow : nullptr, pl->x3)) < 0)
     return r;
   launches += r;
-  if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J)) < 0) return r;
+  if ((r = launch_finish_dml(s, u, u, aux->similar, d.margin, K, d.J, 1, 0, nullptr, cu)) < 0) return r;
+  if (emit) { pl->fresh_u = u.base; pl->fresh_v = v.base; pl->fresh_K = K; }
   return launches + r;
 }
 
+// blk0: first reduction block of these rows inside the plan's correction operands; have_u / have_v: the factor stage
+// already wrote them there
 static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows,
-                            float eta, int K, const int* dev_status, const void* directory);
+                            float eta, int K, const int* dev_status, const void* directory, long long blk0, bool have_u,
+                            bool have_v);
 
 int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
                int K, const int* dev_status, const void* directory) {
   const sfb_desc& d = pl->d;
-  if (pl->x3 && K > X3_PAIRS_PER_APPLY && K > d.B) {
+  // correction operands left by the factor stage of the same step, for exactly these rows (one use)
+  const bool chunked = pl->x3 && K > X3_PAIRS_PER_APPLY && K > d.B;
+  const bool usable = pl->x3 && directory == nullptr && pl->fresh_K == K && (!chunked || d.B >= 32);
+  const bool have_u = usable && pl->fresh_u == u_rows.base, have_v = usable && pl->fresh_v == v_rows.base;
+  pl->fresh_u = pl->fresh_v = nullptr;
+  pl->fresh_K = 0;
+  if (chunked) {
     // The accumulator of a tile rounds toward zero once per 8 pairs (about 1.6e-8 of the sum each time), so an update
     // of very many pairs goes to W in several launches of whole worker streams, each added to W in fp32 by the
     // epilogue: more traffic on W, an error that stops growing with K.
@@ -1266,17 +1324,19 @@ int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, R
       u.base += (long long)w0 * u.worker_stride;
       v.base += (long long)w0 * v.worker_stride;
       const void* dir = directory != nullptr ? reinterpret_cast<const char*>(directory) + (size_t)w0 * 32 : nullptr;
-      const int r = umma_apply_range(pl, s, W, w_shadow, u, v, eta, n * d.B, dev_status, dir);
+      const long long blk0 = d.B >= 32 ? (long long)w0 * ((d.B + 31) / 32) : 0;
+      const int r = umma_apply_range(pl, s, W, w_shadow, u, v, eta, n * d.B, dev_status, dir, blk0, have_u, have_v);
       if (r < 0) return r;
       launches += r;
     }
     return launches;
   }
-  return umma_apply_range(pl, s, W, w_shadow, u_rows, v_rows, eta, K, dev_status, directory);
+  return umma_apply_range(pl, s, W, w_shadow, u_rows, v_rows, eta, K, dev_status, directory, 0, have_u, have_v);
 }
 
 static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows,
-                            float eta, int K, const int* dev_status, const void* directory) {
+                            float eta, int K, const int* dev_status, const void* directory, long long blk0, bool have_u,
+                            bool have_v) {
   const sfb_desc& d = pl->d;
   const int es = pl->es, CH = 128 / es;
   const int workers = K / d.B;
@@ -1337,14 +1397,19 @@ static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16
   int launches = 0;
   if (pl->x3) {
     // correction operands of this launch's factor rows, block by block as the kernel takes them (BK = 32 pairs)
-    int r = launch_split_mn(s, u_rows, d.J, workers, p.k_bb, p.k_wp, p.k_bpw, p.k_blocks, pl->uc, pl->ldcu, true);
-    if (r < 0) return r;
-    launches += r;
-    r = launch_split_mn(s, v_rows, d.D, workers, p.k_bb, p.k_wp, p.k_bpw, p.k_blocks, pl->vc, pl->ldcv, false);
-    if (r < 0) return r;
-    launches += r;
-    if (!encode_corr_mn_map(&tuc, pl->uc, pl->ldcu, (long long)p.k_blocks * 64, BM / 64) ||
-        !encode_corr_mn_map(&tvc, pl->vc, pl->ldcv, (long long)p.k_blocks * 64, (v.bn / v.cg) / 64))
+    char* uc = reinterpret_cast<char*>(pl->uc) + blk0 * 64 * pl->ldcu * 2;
+    char* vc = reinterpret_cast<char*>(pl->vc) + blk0 * 64 * pl->ldcv * 2;
+    int r;
+    if (!have_u) {
+      if ((r = launch_split_mn(s, u_rows, d.J, workers, p.k_bb, p.k_wp, p.k_bpw, p.k_blocks, uc, pl->ldcu, true)) < 0) return r;
+      launches += r;
+    }
+    if (!have_v) {
+      if ((r = launch_split_mn(s, v_rows, d.D, workers, p.k_bb, p.k_wp, p.k_bpw, p.k_blocks, vc, pl->ldcv, false)) < 0) return r;
+      launches += r;
+    }
+    if (!encode_corr_mn_map(&tuc, uc, pl->ldcu, (long long)p.k_blocks * 64, BM / 64) ||
+        !encode_corr_mn_map(&tvc, vc, pl->ldcv, (long long)p.k_blocks * 64, (v.bn / v.cg) / 64))
       return SFB_ERR_CUDA;
   }
   const int r = dispatch_gemm<true, 0>(s, es, v, tu, tv, tw, tuc, tvc, p, pl->num_sms);

@@ -12,9 +12,11 @@ int umma_plan_create(const sfb_desc& d, const Layout& l, UmmaPlan** out);
 void umma_plan_destroy(UmmaPlan* p);
 
 // z = W a on the tensor cores followed by the model epilogue; factors go through u / v row maps.
+// for_apply (compensated path): umma_apply of exactly these u / v rows, all K pairs, follows before anything else
+// changes them: the kernels that write the factors also write the apply's correction operands (one use).
 // workers > 0: only that many workers' samples (X, aux, u, v start at the first of them).
 int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16* w_shadow, const void* X,
-                 const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers = 0);
+                 const sfb_aux* aux, RowMap u, RowMap v, int* dev_status, int workers = 0, bool for_apply = false);
 
 // Z rows (fp32) = A rows (the path's value type) times Wop^T on the tensor cores; no epilogue beyond the store.
 // w_corr: on the compensated path, W's correction operand (launch_split_k of W's rows, B side); w_shadow plays
@@ -22,11 +24,11 @@ int umma_forward(UmmaPlan* p, cudaStream_t s, const void* W, const __nv_bfloat16
 int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, RowMap z, int* dev_status,
                       float2* stats = nullptr, int* n_parts_out = nullptr, int* part_cols_out = nullptr,
                       int* k_splits_out = nullptr, int max_splits = 1, long long split_stride = 0, int workers = 0,
-                      const void* w_corr = nullptr);
+                      const void* w_corr = nullptr, bool a_corr_ready = false);
 
 // Sparse coding: u rows = dense code rows `a` (fp32) times W^T minus the data rows Xdata [K][J].
 int umma_forward_sc(UmmaPlan* p, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
-                    int workers = 0, const void* w_corr = nullptr);
+                    int workers = 0, const void* w_corr = nullptr, bool for_apply = false);
 
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
 // u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).
