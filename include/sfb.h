@@ -31,7 +31,9 @@
  *   - sfb_compute_factors, sfb_pack, sfb_apply, sfb_step, sfb_factors_shard and sfb_commit_header only enqueue
  *     kernels (and event fork / join with a side stream of the context); after one ordinary call, which does
  *     the one-time kernel attribute set-up, a call may be recorded into a CUDA graph by capturing the context's
- *     stream and replayed (pointers and the clock are then the recorded ones).
+ *     stream and replayed (pointers and the clock are then the recorded ones, and so is the decision whether
+ *     the context's cached copy of W, see sfb_invalidate, had to be rebuilt first: record a call that follows an
+ *     ordinary call on the same W, and do not replay it after W was changed from outside).
  *   - "allocates only in sfb_create" has two stated exceptions, both on first use: the staging buffers
  *     of sfb_step_host and the workspace of sfb_loss.
  *   - W is J x D, row-major fp32, updated in place.  Samples are rows: X is [K][D].
