@@ -644,6 +644,7 @@ int sfb_apply(sfb_ctx* c, void* W, const void* sf_buf, float eta, int32_t K) {
   if (!aligned(W, 16) || !aligned(sf_buf, 128)) return SFB_ERR_ARG;
   if (K <= 0 || K > c->K || (K % c->d.B) != 0) return SFB_ERR_ARG;
   if (has_shadow(c) && c->shadow_of != W) c->shadow_of = nullptr;
+  if (c->umma != nullptr) umma_drop_corr(c->umma);   // the buffer is the caller's: nothing prepared for it counts
   return apply_from(c, W, sf_buf, eta, K, true);
 }
 

@@ -1301,6 +1301,11 @@ static int umma_apply_range(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16
                             float eta, int K, const int* dev_status, const void* directory, long long blk0, bool have_u,
                             bool have_v);
 
+void umma_drop_corr(UmmaPlan* pl) {
+  pl->fresh_u = pl->fresh_v = nullptr;
+  pl->fresh_K = 0;
+}
+
 int umma_apply(UmmaPlan* pl, cudaStream_t s, void* W, __nv_bfloat16* w_shadow, RowMap u_rows, RowMap v_rows, float eta,
                int K, const int* dev_status, const void* directory) {
   const sfb_desc& d = pl->d;

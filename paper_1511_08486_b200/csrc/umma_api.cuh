@@ -30,6 +30,9 @@ int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, Ro
 int umma_forward_sc(UmmaPlan* p, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
                     int workers = 0, const void* w_corr = nullptr, bool for_apply = false);
 
+// Forgets correction operands a factor stage left for "its" apply (a caller that applies a buffer of its own).
+void umma_drop_corr(UmmaPlan* p);
+
 // W <- W - eta * U^T V on the tensor cores with the write-back (and bf16 shadow refresh) fused.
 // u_rows / v_rows: the factor rows (normally the U and V blocks of the SF buffer's worker streams).
 // directory (optional): the SF buffer's directory (sf_buf + 128) of a compacted buffer, whose rows behind each
