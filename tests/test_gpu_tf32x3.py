@@ -56,6 +56,39 @@ def test_x3_many_pairs_are_applied_in_several_launches():
     check_config(cfg, "tf32x3", eta=1e-4, steps=1)
 
 
+@pytest.mark.parametrize("name,over,eta", [
+    ("C1", dict(J=300, D=260, P=5, B=8, pool=1), 0.5),          # reduction blocks of the apply span four workers
+    ("C1", dict(J=257, D=1000, P=2, B=100, pool=1), 0.5),       # ragged last block of every worker
+    ("C1", dict(J=128, D=256, P=16, B=256, pool=1), 0.5),       # 4096 pairs: the apply goes to W in four launches
+    ("C2", dict(J=600, D=2000, P=8, B=32), 1e-4),
+    ("C3", dict(J=512, D=2000, P=4, B=32), 1e-3),
+])
+def test_x3_step_and_separate_calls_give_the_same_bits(name, over, eta):
+    """Inside sfb_step the kernels that write the factors also write the apply's correction operands, and the apply's
+    epilogue leaves W's correction operand for the next forward pass; sfb_compute_factors + sfb_pack + sfb_apply
+    build all of them by their own passes.  Same operands, same GEMMs: W and the buffer must agree bit for bit,
+    step after step."""
+    import torch
+    from sfbgen import make_inputs
+    from tests.test_gpu_parity import _workload
+    cfg = _cfg(name, **over)
+    inputs = make_inputs(cfg)
+    a, b = _workload(cfg, inputs, "tf32x3"), _workload(cfg, inputs, "tf32x3")
+    try:
+        for t in range(3):
+            a.step(t, eta=eta)
+            b.compute_factors(t)
+            b.pack(t, clock=t)
+            b.apply(eta)
+            torch.cuda.synchronize()
+            assert torch.equal(a.W, b.W), f"step {t}: W differs"
+            assert torch.equal(a.sf_buf, b.sf_buf), f"step {t}: SF buffer differs"
+        assert a.ctx.status() == 0 and b.ctx.status() == 0
+    finally:
+        a.close()
+        b.close()
+
+
 def test_x3_c1_full():
     print("C1 tf32x3 margins:", check_config(_cfg("C1"), "tf32x3", eta=1.0, steps=2))
 
