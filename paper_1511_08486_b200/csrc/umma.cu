@@ -578,6 +578,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int q = 0; q < 32; ++q) v[q] = __float_as_uint(__uint_as_float(v[q]) + __uint_as_float(lo[q]));
         }
+        if (cc == BN / 64 - 1) {   // the last of this warp's accumulator columns are in registers: the MMAs may go on
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if (CG == 1 || rank == 0) ptx::mbar_arrive(&ctl->tmem_empty[buf]);
+            else ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[buf]), 0));
+          }
+        }
 #pragma unroll
         for (int q = 0; q < 8; ++q)
           *reinterpret_cast<uint4*>(stage + lane * 32 + ((q ^ (lane & 7)) << 2)) =
@@ -632,11 +640,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         __syncwarp();
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {   // this warp's part of the accumulator is drained
-        if (CG == 1 || rank == 0) ptx::mbar_arrive(&ctl->tmem_empty[buf]);
-        else ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[buf]), 0));
+      if (!APPLY && EPI == 1) {   // (the other epilogues signal from inside their last block)
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {   // this warp's part of the accumulator is drained
+          if (CG == 1 || rank == 0) ptx::mbar_arrive(&ctl->tmem_empty[buf]);
+          else ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[buf]), 0));
+        }
       }
     }
   }
