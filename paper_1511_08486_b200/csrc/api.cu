@@ -180,13 +180,17 @@ int factors_into(sfb_ctx* c, const void* W, const void* X, const sfb_aux* aux, R
     const RowMap a = dense_codes(c);
     // plain tf32: the code values are rounded to nearest tf32 as they are densified; the compensated path keeps
     // them exact (its kernels split every operand into what the tensor core sees and the rest)
-    ACC(launch_densify_codes(c->stream, codes, a, K, d.D, c->dev_status, d.path == SFB_PATH_TF32));
+    // compensated path: the same kernel writes the rows' correction operands (when a row fits in shared memory)
+    const bool with_corr = d.path == SFB_PATH_TF32X3 && workers == 0 && densify_corr_fits(a.ld);
+    const CorrOut a_corr = with_corr ? umma_codes_corr(c->umma, for_apply) : CorrOut();
+    if (with_corr) ACC(launch_densify_codes_corr(c->stream, codes, a, K, d.D, c->dev_status, a_corr));
+    else ACC(launch_densify_codes(c->stream, codes, a, K, d.D, c->dev_status, d.path == SFB_PATH_TF32));
     {
       const int r = ensure_shadow(c, W);
       if (r < 0) return r;
     }
     ACC(umma_forward_sc(c->umma, c->stream, W, a, u, reinterpret_cast<const float*>(aux->Xdata), c->dev_status, workers,
-                        c->w_shadow, for_apply));
+                        c->w_shadow, for_apply, with_corr ? &a_corr : nullptr));
     return SFB_OK;
   }
   if (d.path == SFB_PATH_F32) {

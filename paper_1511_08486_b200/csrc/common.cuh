@@ -216,6 +216,10 @@ int launch_sc_csc_apply(cudaStream_t s, float* W, RowMap u, int K, int J, int D,
 // Dense fp32 rows a_i of the CSR codes (zeros elsewhere), for the tensor-core sparse-coding path.
 // round_tf32: values rounded to the nearest tf32 (the plain tf32 path, whose tensor cores would truncate them).
 int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status, bool round_tf32 = true);
+// The same (exact values) with the rows' correction operands written beside them; a row of ld floats must fit in
+// shared memory (densify_corr_fits).
+bool densify_corr_fits(int ld);
+int launch_densify_codes_corr(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status, CorrOut corr);
 
 // SC epilogue on dense products: u = z - x in place (u rows hold z), pad columns zero.
 // z: products (possibly `nsplit` partials); u = sum of partials - x.

@@ -141,6 +141,30 @@ __global__ void __launch_bounds__(256) densify_kernel(CsrView codes, RowMap a, i
   }
 }
 
+// The same through shared memory (one block per sample, the dense row of a.ld floats staged there), for the
+// compensated path: the row goes out in whole 16-byte units together with its correction operands.
+__global__ void __launch_bounds__(256) densify_corr_kernel(CsrView codes, RowMap a, int K, int D, int* dev_status,
+                                                           CorrOut corr) {
+  extern __shared__ __align__(16) float dense[];
+  const int i = blockIdx.x;
+  const int units = a.ld >> 2;
+  for (int q = threadIdx.x; q < units; q += 256) reinterpret_cast<float4*>(dense)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncthreads();
+  const CsrRow row = csr_row(codes, i);
+  for (int k = threadIdx.x; k < row.len; k += 256) {
+    const uint32_t c = row.idx[k];
+    if (c >= (uint32_t)D || (k > 0 && row.idx[k - 1] >= c)) atomicOr(dev_status, SFB_DEV_BAD_INDEX);   // entry skipped
+    else dense[c] = row.val[k];
+  }
+  __syncthreads();
+  float4* dst = reinterpret_cast<float4*>(a.row(i));
+  for (int q = threadIdx.x; q < units; q += 256) {
+    const float4 t = reinterpret_cast<const float4*>(dense)[q];
+    dst[q] = t;
+    corr_store4(corr, i, a.B, q * 4, t);
+  }
+}
+
 __global__ void __launch_bounds__(256) finish_sc_kernel(RowMap zr, RowMap u, const float* __restrict__ Xdata, int K, int J,
                                                         int nsplit, long long zstride, CorrOut corr) {
   const int units = u.ld >> 2;
@@ -331,6 +355,17 @@ int launch_sc_forward_ws(cudaStream_t s, const float* W, float* Wt, CsrView code
 
 int launch_densify_codes(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status, bool round_tf32) {
   densify_kernel<<<K, 256, 0, s>>>(codes, a, K, D, dev_status, round_tf32);
+  return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
+}
+
+bool densify_corr_fits(int ld) { return (size_t)ld * 4 <= 200 * 1024; }
+
+int launch_densify_codes_corr(cudaStream_t s, CsrView codes, RowMap a, int K, int D, int* dev_status, CorrOut corr) {
+  const size_t smem = (size_t)a.ld * 4;
+  static PerDeviceOnce attr_once;   // function attributes are per device
+  if (attr_once.first())
+    cudaFuncSetAttribute(densify_corr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  densify_corr_kernel<<<K, 256, smem, s>>>(codes, a, K, D, dev_status, corr);
   return cudaGetLastError() == cudaSuccess ? 1 : SFB_ERR_CUDA;
 }
 

@@ -1163,8 +1163,16 @@ static CorrOut apply_corr(const UmmaPlan* pl, void* dst, int ldc, bool a_side) {
   return c;
 }
 
+CorrOut umma_codes_corr(UmmaPlan* pl, bool for_apply) {
+  if (!pl->x3) return CorrOut();
+  CorrOut c = for_apply ? apply_corr(pl, pl->vc, pl->ldcv, false) : CorrOut();
+  c.km = reinterpret_cast<char*>(pl->xc);
+  c.atoms = (pl->d.D + 31) / 32;
+  return c;
+}
+
 int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
-                    int workers, const void* w_corr, bool for_apply) {
+                    int workers, const void* w_corr, bool for_apply, const CorrOut* a_corr) {
   const sfb_desc& d = pl->d;
   const int K = (workers > 0 ? workers : d.P) * d.B;
   int r, launches = 0;
@@ -1172,6 +1180,9 @@ int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMa
   pl->fresh_K = 0;
   const bool emit = pl->x3 && for_apply && workers == 0;
   const CorrOut cu = emit ? apply_corr(pl, pl->uc, pl->ldcu, true) : CorrOut();
+  // the kernel that made the code rows wrote their correction operands: the forward's, and perhaps the apply's
+  const bool a_ready = pl->x3 && a_corr != nullptr && a_corr->km == reinterpret_cast<char*>(pl->xc);
+  const void* v_fresh = (emit && a_corr != nullptr && a_corr->mn == reinterpret_cast<char*>(pl->vc)) ? a.base : nullptr;
   if (pl->part_ws != nullptr) {   // reduction in ranges (few tiles, or the compensated path): summed by the finishing pass
     RowMap pz;
     pz.base = reinterpret_cast<char*>(pl->part_ws); pz.ld = pl->ldp; pz.B = d.B; pz.es = 4;
@@ -1179,17 +1190,19 @@ int umma_forward_sc(UmmaPlan* pl, cudaStream_t s, const void* W, RowMap a, RowMa
     const long long sstride = (long long)d.P * d.B * pl->ldp * 4;
     int ks = 1;
     if ((r = umma_forward_rows(pl, s, W, a, pz, dev_status, nullptr, nullptr, nullptr, &ks, pl->max_splits, sstride, workers,
-                               w_corr)) < 0)
+                               w_corr, a_ready)) < 0)
       return r;
     launches += r;
     if ((r = launch_finish_sc(s, pz, u, Xdata, K, d.J, ks, sstride, cu)) < 0) return r;
-    if (emit) { pl->fresh_u = u.base; pl->fresh_K = K; }
+    if (emit) { pl->fresh_u = u.base; pl->fresh_v = v_fresh; pl->fresh_K = K; }
     return launches + r;
   }
-  if ((r = umma_forward_rows(pl, s, W, a, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers, w_corr)) < 0) return r;
+  if ((r = umma_forward_rows(pl, s, W, a, u, dev_status, nullptr, nullptr, nullptr, nullptr, 1, 0, workers, w_corr,
+                             a_ready)) < 0)
+    return r;
   launches += r;
   if ((r = launch_finish_sc(s, u, u, Xdata, K, d.J, 1, 0, cu)) < 0) return r;
-  if (emit) { pl->fresh_u = u.base; pl->fresh_K = K; }
+  if (emit) { pl->fresh_u = u.base; pl->fresh_v = v_fresh; pl->fresh_K = K; }
   return launches + r;
 }
 

@@ -27,8 +27,12 @@ int umma_forward_rows(UmmaPlan* p, cudaStream_t s, const void* Wop, RowMap a, Ro
                       const void* w_corr = nullptr, bool a_corr_ready = false);
 
 // Sparse coding: u rows = dense code rows `a` (fp32) times W^T minus the data rows Xdata [K][J].
+// a_corr: what umma_codes_corr returned, if the kernel that made the rows `a` has written it.
 int umma_forward_sc(UmmaPlan* p, cudaStream_t s, const void* W, RowMap a, RowMap u, const float* Xdata, int* dev_status,
-                    int workers = 0, const void* w_corr = nullptr, bool for_apply = false);
+                    int workers = 0, const void* w_corr = nullptr, bool for_apply = false, const CorrOut* a_corr = nullptr);
+// Compensated path: where the kernel that makes the dense code rows may write their correction operands (the
+// forward's; with for_apply also the apply's, for which the code rows are the v rows).  Empty on other paths.
+CorrOut umma_codes_corr(UmmaPlan* p, bool for_apply);
 
 // Forgets correction operands a factor stage left for "its" apply (a caller that applies a buffer of its own).
 void umma_drop_corr(UmmaPlan* p);
