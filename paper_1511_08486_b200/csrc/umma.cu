@@ -78,10 +78,9 @@ struct SharedCtl {
   uint16_t nb[MAX_DIR_WORKERS];   // apply with a directory: reduction blocks of each worker
 };
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int* status,
-                                              bool cluster_scope = false) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int* status) {
   for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-    if (cluster_scope ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)) return true;
+    if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && ctl->abort) return false;
   }
   ctl->abort = 1;
